@@ -1,0 +1,409 @@
+#!/usr/bin/env python
+"""Benchmark of the Speculative-Streaming decode hot path on B200.
+
+A step = one pass of the whole hot path over one batch of synthetic input: the attention of every
+layer (plain tree-masked layers, then the N_s multi-stream layers), greedy tree verification and
+KV compaction over all layers.  Default workload: the 7B-class shape the headline metric is quoted
+on (32 layers, 32 heads x 128, L = 2048, 64-node tree, gamma = 4).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 7b] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` is achieved HBM GB/s: the step's algorithmic bytes (each
+input and output byte counted once) divided by the device time of the step, inputs resident in HBM.
+For N > 1 every rank runs an independent replica on its own GPU (the path has no exchange step);
+time is the max over ranks and value sums the bytes of all ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "msa_tree_attention_step_hbm_throughput"
+UNIT = "GB/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="7b")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            d = json.load(fh)
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json, copy kernel)"
+    return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+# ---- clocks --------------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc, self.thread = index, [], None, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0])); smax.append(float(r[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower() == "active":
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---- oracle timing (CPU baseline / reference arm) -----------------------------------------------------
+def oracle_sample(st, heads_per_layer: int = 2):
+    """Times the oracle, as it stands, on a bounded sample of the workload: `heads_per_layer` heads of
+    one plain and one MSA layer (sequence 0), the whole verification of sequence 0, and the compaction
+    of sequence 0 over 4 layers.  Returns (bytes_processed, seconds, description, threads)."""
+    import oracle
+    c = st.cfg
+    H, d, T, g = c.n_heads, c.head_dim, c.n_nodes, c.gamma
+    L = int(st.kv_len[0])
+    n_plain = c.n_layers - c.n_msa_layers
+    layers = ([0] if n_plain > 0 else []) + [c.n_layers - 1]
+    hp = min(heads_per_layer, H)
+    inputs = [st.layer(l) for l in layers]
+    lg = st.logits()
+    s0, cap = int(st.kv_start[0]), int(st.kv_capacity[0])
+    nbytes = 0
+    t0 = time.perf_counter()
+    for ly in inputs:
+        gg = g if ly.is_msa else 0
+        oracle.msa_attention(st.parent[0], L, gg, st.sm_scale, ly.q_main[0], ly.k_cache[s0:s0 + cap],
+                             ly.v_cache[s0:s0 + cap], None if gg == 0 else ly.q_spec[0],
+                             None if gg == 0 else ly.k_spec[0], None if gg == 0 else ly.v_spec[0], heads=(0, hp))
+        nbytes += (4 * L * d + 4 * T * d + 4 * T * gg * d + 4 * T * (1 + gg) * d) * hp
+    r = oracle.tree_verify(lg[0], st.draft_tokens[0], st.parent[0], path_cap=64)
+    nbytes += 4 * T * c.vocab
+    k4 = np.stack([inputs[-1].k_cache[s0:s0 + cap]] * 4)
+    oracle.kv_compact(k4, k4, L, r["accept_len"], r["path"])
+    nbytes += 2 * 2 * r["accept_len"] * H * d * 2 * 4
+    dt = time.perf_counter() - t0
+    desc = ("sequence 0: %d of %d heads of %d attention layer(s) (one plain, one multi-stream), full verification, "
+            "compaction over 4 layers" % (hp, H, len(inputs)))
+    return nbytes, dt, desc, oracle.max_threads()
+
+
+def run_reference(args):
+    """Reference arm: the CPU oracle timed on host cores, on bounded samples of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2402_11131_b200 import workloads as W
+    st = W.make_step(W.CONFIGS[args.workload])
+    steps = max(1, min(args.steps, 5))
+    warm = max(0, min(args.warmup, 1))
+    for _ in range(warm):
+        oracle_sample(st)
+    tot_b, tot_t, desc, thr = 0, 0.0, "", 1
+    for _ in range(steps):
+        b, t, desc, thr = oracle_sample(st)
+        tot_b += b; tot_t += t
+    val = tot_b / tot_t / 1e9
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+            "warmup": warm, "ms_per_step": tot_t / steps * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "note": "CPU oracle on a bounded sample per step"},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": thr, "kind": "oracle", "sample": desc},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ---- our arm -----------------------------------------------------------------------------------------
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    from paper_2402_11131_b200 import api, build, workloads as W
+    from paper_2402_11131_b200.step import DeviceStep
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+    api.lib()
+
+    cfg = W.CONFIGS[args.workload]
+    st = W.make_step(cfg)
+    distinct = 2 if cfg.batch > 1 else None       # the ragged batch reuses two host-generated slabs
+    dev = DeviceStep(st, distinct_slabs=distinct, pinned_host=not args.no_e2e)
+    stream = torch.cuda.Stream()
+    nl = len(dev.layers)
+
+    # bytes of one step (each byte once)
+    with torch.cuda.stream(stream):
+        dev.run_verify(stream)
+    stream.synchronize()
+    acc = dev.accept_len.cpu().numpy()
+    attn_bytes = sum(dev.attention_bytes(i) for i in range(nl))
+    step_bytes = attn_bytes + dev.verify_bytes() + dev.compact_bytes(acc)
+    attn_flops = sum(dev.attention_flops(i) for i in range(nl))
+
+    # ---- capture the step, and the attention layers alone, into CUDA graphs -----------------------
+    def capture(fn):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            fn(stream)                           # warm (lazy kernel attributes are set outside capture)
+            stream.synchronize()
+            with torch.cuda.graph(g, stream=stream):
+                n = fn(stream)
+        return g, n
+
+    g_step, launches_per_step = capture(dev.run_step)
+    g_attn, _ = capture(dev.run_attention)
+    plain_idx = [i for i in range(nl) if not dev.is_msa[i]]
+    msa_idx = [i for i in range(nl) if dev.is_msa[i]]
+    g_plain = capture(lambda s: dev.run_attention(s, only=plain_idx))[0] if plain_idx else None
+    g_msa = capture(lambda s: dev.run_attention(s, only=msa_idx))[0] if msa_idx else None
+    g_verify, _ = capture(dev.run_verify)
+    g_compact, _ = capture(dev.run_compact)
+
+    def time_graph(g, reps, warm):
+        with torch.cuda.stream(stream):
+            for _ in range(warm):
+                g.replay()
+            stream.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(reps):
+                g.replay()
+            e1.record(stream)
+            stream.synchronize()
+        return e0.elapsed_time(e1) / reps     # ms per replay
+
+    # ---- the timed region ----------------------------------------------------------------------
+    K, Wm = args.steps, max(args.warmup, 3)
+    with torch.cuda.stream(stream):
+        for _ in range(Wm):
+            g_step.replay()
+    stream.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for _ in range(K):
+            g_step.replay()
+        e1.record(stream)
+    stream.synchronize()
+    torch.cuda.synchronize()
+    step_ms = e0.elapsed_time(e1) / K
+    # component timings (same graphs' kernels, timed alone) while the clock sampler still runs
+    attn_ms = time_graph(g_attn, K, 3)
+    plain_ms = time_graph(g_plain, K, 3) if g_plain else None
+    msa_ms = time_graph(g_msa, K, 3) if g_msa else None
+    verify_ms = time_graph(g_verify, K, 3)
+    compact_ms = time_graph(g_compact, K, 3)
+    clocks = sampler.stop() if rank == 0 else None
+    if world > 1:
+        t = torch.tensor([step_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        step_ms = float(t.item())
+        dist.barrier()
+    status = api.ss_status(dev.attn_ws, stream) or api.ss_status(dev.verify_ws, stream)
+    if status != 0:
+        raise RuntimeError("device status %d after the timed region" % status)
+
+    # ---- end to end: per-step inputs from pinned host memory, results read back ------------------
+    e2e = None
+    if not args.no_e2e:
+        e2e = time_e2e(dev, stream, max(3, min(K, 50)), world)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_src = measured_peaks()
+    value = world * step_bytes / (step_ms * 1e-3) / 1e9
+    attn_launch_us = attn_ms * 1e3 / nl
+    achieved = (attn_bytes / nl) / (attn_launch_us * 1e-6) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "batch": cfg.batch, "n_layers": cfg.n_layers,
+                   "n_msa_layers": cfg.n_msa_layers, "n_heads": cfg.n_heads, "head_dim": cfg.head_dim,
+                   "prefix_len": [int(x) for x in st.kv_len] if cfg.batch > 1 else int(st.kv_len[0]),
+                   "tree_nodes": cfg.n_nodes, "gamma": cfg.gamma, "vocab": cfg.vocab,
+                   "parallelism": "replicas" if world > 1 else "single_gpu",
+                   "l2": "every layer streams its own KV slab; a step touches %.0f MB, far more than the 126 MB L2"
+                         % (step_bytes / 1e6),
+                   "launch": "whole step replayed as one CUDA graph"},
+        "step_bytes": step_bytes, "pct_of_8TBs": value / world / 8000.0 * 100,
+        "us_per_layer": attn_ms * 1e3 / nl,
+        "us_plain_layer": None if plain_ms is None else plain_ms * 1e3 / len(plain_idx),
+        "us_msa_layer": None if msa_ms is None else msa_ms * 1e3 / len(msa_idx),
+        "us_verify": verify_ms * 1e3, "us_compact": compact_ms * 1e3,
+        "mean_accept_len": float(acc.mean()),
+        "attention_tflops": attn_flops / (attn_ms * 1e-3) / 1e12,
+        "gpu_launches": launches_per_step * K,
+        "clocks": clocks,
+        "roofline": {"kernel": "msa_attention_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
+                     "bytes_per_launch": attn_bytes / nl, "us_per_launch": attn_launch_us, "traffic": ncu_traffic()},
+        "e2e": e2e,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        b, t, desc, thr = oracle_sample(st)
+        line["cpu_baseline"] = {"value": b / t / 1e9, "unit": UNIT, "cores": thr, "kind": "oracle", "sample": desc,
+                                "seconds": t}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def ncu_traffic():
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if present."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            return json.load(fh).get("msa_attention_kernel_dram_bytes_per_launch")
+    return None
+
+
+def time_e2e(dev, stream, reps, world):
+    """The same step driven through the public API with the step's inputs in pinned HOST memory:
+    every step copies the queries, the stream K/V, the tree nodes' K/V, the logits, the draft tokens
+    and the tree descriptors to the device, runs the C-ABI calls, and reads the verification result
+    back.  The KV prefix is the cache, i.e. state left in HBM by earlier steps, not a step input."""
+    import torch
+    import torch.distributed as dist
+    from paper_2402_11131_b200 import api
+    st, c = dev.st, dev.cfg
+    B, T = c.batch, c.n_nodes
+    nl = len(dev.layers)
+    # pinned host staging of the per-step inputs
+    h_logits = dev.logits.cpu().pin_memory()
+    h_tokens = dev.tokens.cpu().pin_memory()
+    h_trees = dev.trees.cpu().pin_memory()
+    h_tree_kv = []
+    for b in range(B):
+        lo = int(st.kv_start[b]) + int(st.kv_len[b])
+        h_tree_kv.append((lo, dev.k_all[:, lo:lo + T].cpu().pin_memory(), dev.v_all[:, lo:lo + T].cpu().pin_memory()))
+    h_out = {k: torch.empty_like(getattr(dev, k), device="cpu").pin_memory()
+             for k in ("accept_len", "accept_path", "bonus_token", "last_node", "kv_len_out")}
+    h2d = h_logits.numel() * 4 + h_tokens.numel() * 4 + h_trees.numel()
+    for lo, hk, hv in h_tree_kv:
+        h2d += 2 * hk.numel() * 2
+    for h in dev.host_inputs:
+        h2d += sum(t.numel() * 2 for t in h.values())
+    d2h = sum(t.numel() * 4 for t in h_out.values())
+
+    def one_step():
+        with torch.cuda.stream(stream):
+            dev.logits.copy_(h_logits, non_blocking=True)
+            dev.tokens.copy_(h_tokens, non_blocking=True)
+            dev.trees.copy_(h_trees, non_blocking=True)
+            for lo, hk, hv in h_tree_kv:
+                dev.k_all[:, lo:lo + T].copy_(hk, non_blocking=True)
+                dev.v_all[:, lo:lo + T].copy_(hv, non_blocking=True)
+            for i, h in enumerate(dev.host_inputs):
+                dev.q_main[i].copy_(h["q_main"], non_blocking=True)
+                if "q_spec" in h:
+                    dev.q_spec[i].copy_(h["q_spec"], non_blocking=True)
+                    dev.k_spec[i].copy_(h["k_spec"], non_blocking=True)
+                    dev.v_spec[i].copy_(h["v_spec"], non_blocking=True)
+            dev.run_step(stream)
+            for k, t in h_out.items():
+                t.copy_(getattr(dev, k), non_blocking=True)
+        stream.synchronize()
+
+    for _ in range(3):
+        one_step()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        one_step()
+    torch.cuda.synchronize()
+    dt = (time.perf_counter() - t0) / reps
+    if world > 1:
+        t = torch.tensor([dt], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dt = float(t.item())
+    acc = dev.accept_len.cpu().numpy()
+    step_bytes = (sum(dev.attention_bytes(i) for i in range(nl)) + dev.verify_bytes() + dev.compact_bytes(acc))
+    return {"value": world * step_bytes / dt / 1e9, "unit": UNIT, "ms_per_step": dt * 1e3,
+            "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": reps,
+            "note": "per-step inputs (queries, stream K/V, tree K/V, logits, tokens, trees) copied from pinned host "
+                    "memory; the KV prefix is resident cache state; results read back to the host"}
+
+
+if __name__ == "__main__":
+    main()

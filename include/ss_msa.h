@@ -1,0 +1,177 @@
+/*
+ * ss_msa.h -- C ABI of the Speculative-Streaming decode hot path on NVIDIA B200 (sm_100a).
+ *
+ * One decode step of Speculative Streaming verifies the tree draft of the previous pass and
+ * speculates the next one in the same forward pass (Sec. 3.2.2).  This library implements the
+ * attention of that pass, the verification and the cache backtracking:
+ *
+ *   ss_tree_build      parent array -> depth / ancestor-bitmask descriptor       (host, pure)
+ *   ss_msa_attention   one layer of tree-masked multi-stream attention           (Eq. 1, Eq. 2)
+ *   ss_tree_verify     greedy verification of the tree draft                     (Sec. 3.2.2, App. A.1)
+ *   ss_kv_compact      lazy KV-cache backtracking of the accepted path           (App. A.1)
+ *   ss_status          read back the device status word
+ *
+ * Conventions
+ *   - Every call returns an int32 status: SS_OK or a negative SS_ERR_* code.  No exceptions.
+ *   - All buffers are caller-owned.  Unless a parameter says "host", a pointer is a DEVICE pointer.
+ *   - Device calls validate their host-visible arguments first (an error means nothing was
+ *     launched), then enqueue kernels on `stream` (a cudaStream_t passed as void*; NULL = the
+ *     default stream) and return without synchronising.  They never allocate or free memory and
+ *     never read device memory back to the host, so they can be captured into a CUDA graph.
+ *   - bf16 tensors are raw 16-bit patterns; the innermost (head_dim) axis is contiguous and every
+ *     tensor base, and every K/V row, must be 16-byte aligned.
+ *   - A workspace must be zero-filled once (cudaMemset) before its first use; each call leaves
+ *     it ready for the next.  Word 0 of a workspace is the device status word: a kernel that
+ *     detects a broken invariant (sequence over capacity, a wait that ran out) stores its
+ *     SS_ERR_* code there and returns instead of faulting.
+ *   - Two calls that share a workspace must not overlap on the device.
+ */
+#ifndef SS_MSA_H_
+#define SS_MSA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SS_MAX_NODES 64      /* tree nodes per sequence (one 64-bit ancestor word per node) */
+#define SS_MAX_GAMMA 4       /* speculative streams per node */
+#define SS_PATH_STRIDE SS_MAX_NODES /* entries per sequence in accept_path */
+
+enum {
+    SS_OK = 0,
+    SS_ERR_INVALID_ARG = -1,    /* null pointer, non-positive size, misaligned buffer */
+    SS_ERR_BAD_TREE = -2,       /* parent[0] != -1 or parent[i] outside [0, i) */
+    SS_ERR_UNSUPPORTED = -3,    /* head_dim not in {64, 80, 128}, too many nodes or streams */
+    SS_ERR_WORKSPACE = -4,      /* workspace smaller than the *_workspace_bytes() answer */
+    SS_ERR_CAPACITY = -5,       /* kv_len + n_nodes exceeds the sequence's slot capacity */
+    SS_ERR_CUDA = -6,           /* a CUDA runtime/driver call failed (launch, tensor-map encode) */
+    SS_ERR_DEVICE_TIMEOUT = -7  /* a bounded device-side wait ran out */
+};
+
+/* Tree / mask descriptor.  Plain data, identical on host and device.
+ * Node 0 is the root (the correction token issued by the main stream in the previous pass,
+ * App. A.1); nodes are flattened root-first so that parent[i] < i.  anc_mask[t] has bit a set
+ * iff a is t or lies on the path from the root to t: a node attends to all its predecessors
+ * starting from the root, and to itself (attention-mask figure of App. A). */
+typedef struct ss_tree_desc {
+    int32_t n_nodes;                 /* T, 1..SS_MAX_NODES */
+    int32_t gamma;                   /* streams per node the tree was built for (informative) */
+    int32_t max_depth;               /* depth(root) = 0 */
+    int32_t reserved;
+    int32_t parent[SS_MAX_NODES];    /* parent[0] = -1; entries >= n_nodes are -1 */
+    int32_t depth[SS_MAX_NODES];
+    uint64_t anc_mask[SS_MAX_NODES];
+} ss_tree_desc;
+
+/* Builds the descriptor of one tree on the HOST (all pointers are host pointers).
+ * Errors: SS_ERR_INVALID_ARG (null), SS_ERR_UNSUPPORTED (n_nodes > SS_MAX_NODES or gamma outside
+ * [0, SS_MAX_GAMMA]), SS_ERR_BAD_TREE (n_nodes < 1, parent[0] != -1, parent[i] not in [0, i)).
+ * Pure and reentrant.  The mask is constant for a fixed tree shape (Sec. 3.2.2), so a caller
+ * may build it once and reuse it. */
+int32_t ss_tree_build(const int32_t* parent, int32_t n_nodes, int32_t gamma, ss_tree_desc* out);
+
+/* One layer of attention for a batch of sequences, each with its own tree draft.
+ *
+ * Main-stream row of node t (Eq. 1): attends the sequence's cached prefix (slots 0..L-1) plus the
+ * tree nodes on its root path, itself included.  Speculative-stream row (t, j), 1 <= j <= gamma
+ * (Eq. 2): attends the same main-stream keys plus the stream keys (t,1)..(t,j) of the same node.
+ * Only main-stream K/V live in the cache; stream K/V are transient inputs (Sec. 3.2.1).
+ * gamma = 0 gives a plain tree-masked layer (the N - N_s lower layers); the *_spec pointers are
+ * then ignored.
+ *
+ * Layouts (bf16, element strides):
+ *   q_main, o_main                 [batch][max_nodes][n_heads][head_dim]
+ *   q_spec, k_spec, v_spec, o_spec [batch][max_nodes][gamma][n_heads][head_dim]
+ *   k_cache, v_cache               this layer's slab: slot s, head h at
+ *                                  base + s*kv_slot_stride + h*kv_head_stride, kv_total_slots slots.
+ *                                  Sequence b owns slots kv_start[b] .. ; its prefix sits at
+ *                                  +0..L_b-1 and the caller has already written the K/V of tree node
+ *                                  t at slot kv_start[b] + L_b + t.
+ *   kv_start int64[batch], kv_len int32[batch] (= L_b), kv_capacity int32[batch] (may be NULL):
+ *                                  device arrays, read by the kernel (the host never needs L_b).
+ *   trees                          device array of `batch` descriptors; rows of nodes >= n_nodes of a
+ *                                  sequence are neither read nor written.
+ *   lse_main float[batch][max_nodes][n_heads], lse_spec float[batch][max_nodes][gamma][n_heads]:
+ *                                  optional natural-log sum-exp of the scaled scores (NULL to skip).
+ * Scores are sm_scale * <q, k>; softmax statistics and both products accumulate in fp32.
+ * Reads nothing past slot kv_start[b]+L_b+T_b-1; writes only o_*, lse_* and the workspace.
+ * If kv_capacity is given and L_b + T_b > kv_capacity[b], sequence b is skipped and the status word
+ * is set to SS_ERR_CAPACITY.
+ * Errors (nothing launched): SS_ERR_INVALID_ARG, SS_ERR_UNSUPPORTED, SS_ERR_WORKSPACE, SS_ERR_CUDA. */
+typedef struct ss_attn_params {
+    int32_t batch, n_heads, head_dim, gamma;
+    int32_t max_nodes;              /* row stride (in nodes) of the q/o/lse arrays, <= SS_MAX_NODES */
+    float sm_scale;
+    const void* q_main;
+    void* o_main;
+    const void* q_spec;
+    const void* k_spec;
+    const void* v_spec;
+    void* o_spec;
+    const void* k_cache;
+    const void* v_cache;
+    int64_t kv_slot_stride, kv_head_stride, kv_total_slots;
+    const int64_t* kv_start;
+    const int32_t* kv_len;
+    const int32_t* kv_capacity;
+    const ss_tree_desc* trees;
+    float* lse_main;
+    float* lse_spec;
+    void* workspace;
+    size_t workspace_bytes;
+} ss_attn_params;
+
+/* Bytes of workspace ss_msa_attention needs for these shapes (pointers in *p are not read). */
+size_t ss_msa_attention_workspace_bytes(const ss_attn_params* p);
+int32_t ss_msa_attention(const ss_attn_params* p, void* stream);
+
+/* Greedy ("hard" matching, App. A.2) verification of each sequence's tree draft (Sec. 3.2.2,
+ * App. A.1).  am[t] = lowest index maximising logits[b][t][.]; the root is always accepted; node c
+ * is valid iff its parent is valid and draft_tokens[c] == am[parent[c]]; the deepest valid node
+ * wins, the lowest node index among equally deep ones.
+ *   logits        float [batch][max_nodes][vocab]   main-stream logits of every tree node
+ *   draft_tokens  int32 [batch][max_nodes]
+ *   accept_len    int32 [batch]      nodes on the accepted path, root included (1 .. max_depth+1)
+ *   accept_path   int32 [batch][SS_PATH_STRIDE]  node indices root-first, padded with -1
+ *   last_node     int32 [batch]      last accepted node
+ *   bonus_token   int32 [batch]      am[last_node]: the correction token, root of the next draft
+ *   node_argmax   int32 [batch][max_nodes] or NULL
+ * Bit-exact by definition (comparisons of fp32 values only). */
+size_t ss_tree_verify_workspace_bytes(int32_t batch, int32_t max_nodes, int32_t vocab);
+int32_t ss_tree_verify(const float* logits, const int32_t* draft_tokens, const ss_tree_desc* trees,
+                       int32_t batch, int32_t max_nodes, int32_t vocab, int32_t* accept_len,
+                       int32_t* accept_path, int32_t* last_node, int32_t* bonus_token,
+                       int32_t* node_argmax, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Cache layout shared by all layers: layer l, slot s, head h, element c of K sits at
+ * k_cache_all + l*layer_stride + s*slot_stride + h*head_stride + c (strides in elements). */
+typedef struct ss_cache_layout {
+    int32_t n_layers, n_heads, head_dim, reserved;
+    int64_t layer_stride, slot_stride, head_stride;
+} ss_cache_layout;
+
+/* Lazy KV backtracking (App. A.1): in every layer and for every sequence b, the K and V of accepted
+ * node accept_path[b][i] move from slot kv_start[b]+L_b+path[i] to slot kv_start[b]+L_b+i, in place,
+ * for i < accept_len[b]; kv_len_out[b] = L_b + accept_len[b] (kv_len_out may alias kv_len_in).
+ * Prefix slots are never written; slots at or past L_b + accept_len[b] are unspecified afterwards.
+ * Stream K/V are never cached, so nothing else moves (Sec. 3.2.1).
+ * accept_len / accept_path are the device outputs of ss_tree_verify: no host round trip. */
+int32_t ss_kv_compact(void* k_cache_all, void* v_cache_all, const ss_cache_layout* layout, int32_t batch,
+                      const int64_t* kv_start, const int32_t* kv_len_in, const int32_t* accept_len,
+                      const int32_t* accept_path, int32_t* kv_len_out, void* stream);
+
+/* Synchronises `stream`, copies the status word of `workspace` to *device_status_out (host) and
+ * clears it.  Returns SS_ERR_CUDA if the stream reports an error. */
+int32_t ss_status(void* workspace, void* stream, int32_t* device_status_out);
+
+/* Library version (major*10000 + minor*100 + patch) and a short human-readable error string. */
+int32_t ss_version(void);
+const char* ss_error_string(int32_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SS_MSA_H_ */

@@ -125,8 +125,8 @@ class LayerInputs:
     q_spec: Optional[np.ndarray]
     k_spec: Optional[np.ndarray]
     v_spec: Optional[np.ndarray]
-    k_cache: np.ndarray
-    v_cache: np.ndarray
+    k_cache: Optional[np.ndarray]
+    v_cache: Optional[np.ndarray]
 
 
 @dataclass
@@ -141,7 +141,11 @@ class StepInputs:
     p_accept: np.ndarray        # float64 [B]
     sm_scale: float
     q_scale: float
+    n_nodes_b: Optional[np.ndarray] = None   # per-sequence tree sizes T_b <= T (default: all T)
     _logits: Optional[np.ndarray] = field(default=None, repr=False)
+
+    def nodes(self, b: int) -> int:
+        return self.cfg.n_nodes if self.n_nodes_b is None else int(self.n_nodes_b[b])
 
     # ---- per-step tensors -------------------------------------------------------------
     def logits(self) -> np.ndarray:
@@ -169,10 +173,10 @@ class StepInputs:
     def is_msa_layer(self, layer: int) -> bool:
         return layer >= self.cfg.n_layers - self.cfg.n_msa_layers
 
-    def layer(self, layer: int, slab_seed: Optional[int] = None) -> LayerInputs:
+    def layer(self, layer: int, slab_seed: Optional[int] = None, with_slab: bool = True) -> LayerInputs:
         """Draw the tensors of one layer.  `slab_seed` (default: the layer index) selects the
         random substream of the KV slab, so a caller may reuse a few distinct slabs for many
-        layers when host memory is short."""
+        layers when host memory is short; with_slab=False skips the slab (k_cache = v_cache = None)."""
         c = self.cfg
         B, T, H, d, g = c.batch, c.n_nodes, c.n_heads, c.head_dim, c.gamma
         msa = self.is_msa_layer(layer)
@@ -183,8 +187,10 @@ class StepInputs:
             ks = _normal_bf16(_rng(c.seed, _TID_KS, layer), (B, T, g, H, d))
             vs = _normal_bf16(_rng(c.seed, _TID_VS, layer), (B, T, g, H, d))
         s = layer if slab_seed is None else slab_seed
-        kc = _normal_bf16(_rng(c.seed, _TID_K, s), (self.total_slots, H, d))
-        vc = _normal_bf16(_rng(c.seed, _TID_V, s), (self.total_slots, H, d))
+        kc = vc = None
+        if with_slab:
+            kc = _normal_bf16(_rng(c.seed, _TID_K, s), (self.total_slots, H, d))
+            vc = _normal_bf16(_rng(c.seed, _TID_V, s), (self.total_slots, H, d))
         return LayerInputs(layer, msa and g > 0, qm, qs, ks, vs, kc, vc)
 
 
