@@ -43,6 +43,9 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--profile", action="store_true",
+                    help="small run for ncu: W warm-up + K steps launched directly (no CUDA graph), "
+                         "no component timings, no end-to-end leg, no CPU baseline")
     return ap.parse_args()
 
 
@@ -194,6 +197,9 @@ def main():
 
     cfg = W.CONFIGS[args.workload]
     st = W.make_step(cfg)
+    if args.profile:
+        run_profile(args, st)
+        return
     distinct = 2 if cfg.batch > 1 else None       # the ragged batch reuses two host-generated slabs
     dev = DeviceStep(st, distinct_slabs=distinct, pinned_host=not args.no_e2e)
     stream = torch.cuda.Stream()
@@ -325,6 +331,29 @@ def main():
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_profile(args, st):
+    """The step launched directly K times after W warm-up steps: the command ncu wraps."""
+    import torch
+    from paper_2402_11131_b200 import api
+    from paper_2402_11131_b200.step import DeviceStep
+    dev = DeviceStep(st, distinct_slabs=2 if st.cfg.batch > 1 else None)
+    stream = torch.cuda.Stream()
+    for _ in range(args.warmup):
+        dev.run_step(stream)
+    stream.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    n = 0
+    for _ in range(args.steps):
+        n += dev.run_step(stream)
+    e1.record(stream)
+    stream.synchronize()
+    status = api.ss_status(dev.attn_ws, stream) or api.ss_status(dev.verify_ws, stream)
+    print(json.dumps({"profile_run": True, "workload": args.workload, "steps": args.steps, "warmup": args.warmup,
+                      "ms_per_step_direct_launch": e0.elapsed_time(e1) / max(1, args.steps), "gpu_launches": n,
+                      "device_status": status}))
 
 
 def ncu_traffic():
