@@ -146,6 +146,27 @@ int32_t ss_tree_verify(const float* logits, const int32_t* draft_tokens, const s
                        int32_t* accept_path, int32_t* last_node, int32_t* bonus_token,
                        int32_t* node_argmax, void* workspace, size_t workspace_bytes, void* stream);
 
+/* ss_tree_verify for callers that cannot provide scratch memory.  (The paper has no counterpart:
+ * this is a property of the library, not of the method.)
+ * Who needs it: code that must not allocate device memory where it calls this library, for example a
+ * plug-in that owns no allocator, a serving loop whose memory was fixed at start-up, or a section in
+ * which cudaMalloc is not permitted.  The scratch that ss_tree_verify takes as `workspace` lives here
+ * in a fixed array of SS_VERIFY_STATIC_SCRATCH_BYTES bytes inside the library's device image; every
+ * GPU that loads the library holds that array until the process exits.  The call allocates and frees
+ * nothing.  Same arguments, outputs and results as ss_tree_verify, minus the workspace.
+ *   - Sizes whose scratch need (ss_tree_verify_workspace_bytes) exceeds the fixed array are rejected
+ *     with SS_ERR_WORKSPACE and nothing is launched.
+ *   - The first call on a device looks up the array's device address (once per device, with that
+ *     device current); make that first call before starting any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; each call
+ *     clears the words that must start at zero (on `stream`, before its kernel).  Calls that overlap
+ *     on the same device (different streams, or several host threads) race: serialise them. */
+#define SS_VERIFY_STATIC_SCRATCH_BYTES (1u << 20)
+int32_t ss_tree_verify_static(const float* logits, const int32_t* draft_tokens, const ss_tree_desc* trees,
+                              int32_t batch, int32_t max_nodes, int32_t vocab, int32_t* accept_len,
+                              int32_t* accept_path, int32_t* last_node, int32_t* bonus_token,
+                              int32_t* node_argmax, void* stream);
+
 /* Cache layout shared by all layers: layer l, slot s, head h, element c of K sits at
  * k_cache_all + l*layer_stride + s*slot_stride + h*head_stride + c (strides in elements). */
 typedef struct ss_cache_layout {

@@ -63,8 +63,9 @@ class CacheLayout(C.Structure):
 
 
 EXPORTS = ("ss_tree_build", "ss_msa_attention_workspace_bytes", "ss_msa_attention",
-           "ss_tree_verify_workspace_bytes", "ss_tree_verify", "ss_kv_compact", "ss_status", "ss_version",
-           "ss_error_string")
+           "ss_tree_verify_workspace_bytes", "ss_tree_verify", "ss_tree_verify_static", "ss_kv_compact", "ss_status",
+           "ss_version", "ss_error_string")
+SS_VERIFY_STATIC_SCRATCH_BYTES = 1 << 20
 
 
 def lib() -> C.CDLL:
@@ -87,6 +88,9 @@ def lib() -> C.CDLL:
         l.ss_tree_verify.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                      C.c_size_t, C.c_void_p]
+        l.ss_tree_verify_static.restype = C.c_int32
+        l.ss_tree_verify_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
+                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         l.ss_kv_compact.restype = C.c_int32
         l.ss_kv_compact.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(CacheLayout), C.c_int32, C.c_void_p,
                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -179,6 +183,19 @@ def ss_tree_verify(logits, draft_tokens, trees, accept_len, accept_path, last_no
                                 _ptr(accept_path), _ptr(last_node), _ptr(bonus_token), _ptr(node_argmax),
                                 _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
            "ss_tree_verify")
+
+
+def ss_tree_verify_static(logits, draft_tokens, trees, accept_len, accept_path, last_node, bonus_token,
+                          node_argmax, stream=None) -> None:
+    """ss_tree_verify for callers that cannot supply scratch memory (no allocator of their own, or
+    allocation forbidden where they call): the scratch is a fixed array inside the library, shared
+    by every call on the device, so overlapping calls race.  Raises SsError(SS_ERR_WORKSPACE) when
+    the sizes need more than SS_VERIFY_STATIC_SCRATCH_BYTES.  Make the first call on a device
+    outside any stream capture."""
+    B, Tmax, V = logits.shape
+    _check(lib().ss_tree_verify_static(_ptr(logits), _ptr(draft_tokens), _ptr(trees), B, Tmax, V,
+                                       _ptr(accept_len), _ptr(accept_path), _ptr(last_node), _ptr(bonus_token),
+                                       _ptr(node_argmax), _stream(stream)), "ss_tree_verify_static")
 
 
 def make_cache_layout(k_all: torch.Tensor) -> CacheLayout:

@@ -158,3 +158,69 @@ extern "C" int32_t ss_tree_verify(const float* logits, const int32_t* draft_toke
         bonus_token, node_argmax, counters, partials);
     return cudaGetLastError() == cudaSuccess ? SS_OK : SS_ERR_CUDA;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Verification without a caller-provided workspace.
+//
+// Some callers cannot hand this library scratch memory: code that runs where allocating device
+// memory is not allowed (inside a region that forbids cudaMalloc, a plug-in that owns no allocator,
+// a real-time loop whose memory was fixed at start-up).  For them the scratch of the verification
+// kernel lives in this fixed device array, which every GPU that loads the library holds until the
+// process exits.  All calls on a device share it, so calls that overlap on that device race.
+namespace ss {
+
+static __device__ __align__(256) unsigned char g_verify_static_scratch[SS_VERIFY_STATIC_SCRATCH_BYTES];
+
+// Device address of the array, looked up once per device.  In host code the array's name is only a
+// host-side handle, never a device address: the address must come from cudaGetSymbolAddress, taken
+// with the device current.
+static void* verify_static_scratch_ptr(int32_t* status) {
+    static void* cached[64] = {nullptr};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        *status = SS_ERR_CUDA;
+        return nullptr;
+    }
+    if (cached[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_verify_static_scratch) != cudaSuccess || p == nullptr) {
+            *status = SS_ERR_CUDA;
+            return nullptr;
+        }
+        cached[dev] = p;
+    }
+    *status = SS_OK;
+    return cached[dev];
+}
+
+}  // namespace ss
+
+extern "C" int32_t ss_tree_verify_static(const float* logits, const int32_t* draft_tokens,
+                                         const ss_tree_desc* trees, int32_t batch, int32_t max_nodes,
+                                         int32_t vocab, int32_t* accept_len, int32_t* accept_path,
+                                         int32_t* last_node, int32_t* bonus_token, int32_t* node_argmax,
+                                         void* stream) {
+    if (!logits || !draft_tokens || !trees || !accept_len || !accept_path || !last_node || !bonus_token)
+        return SS_ERR_INVALID_ARG;
+    if (batch < 1 || max_nodes < 1 || vocab < 1 || batch > 65535) return SS_ERR_INVALID_ARG;
+    if (max_nodes > SS_MAX_NODES) return SS_ERR_UNSUPPORTED;
+    if (!ss::aligned16(logits)) return SS_ERR_INVALID_ARG;
+    const size_t need = ss_tree_verify_workspace_bytes(batch, max_nodes, vocab);
+    if (need == 0 || need > SS_VERIFY_STATIC_SCRATCH_BYTES) return SS_ERR_WORKSPACE;   // beyond the fixed scratch
+    int32_t st = SS_OK;
+    char* ws = static_cast<char*>(ss::verify_static_scratch_ptr(&st));
+    if (ws == nullptr) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // the array keeps the previous call's contents: the status word and the arrival counters must
+    // start at zero (the per-chunk candidates are fully rewritten before they are read)
+    const size_t counter_bytes = (static_cast<size_t>(batch) * sizeof(int32_t) + 255) / 256 * 256;
+    if (cudaMemsetAsync(ws, 0, ss::kWsHeaderBytes + counter_bytes, s) != cudaSuccess) return SS_ERR_CUDA;
+    const int n_chunks = (vocab + ss::kVerifyChunk - 1) / ss::kVerifyChunk;
+    int32_t* counters = reinterpret_cast<int32_t*>(ws + ss::kWsHeaderBytes);
+    ss::Cand* partials = reinterpret_cast<ss::Cand*>(ws + ss::kWsHeaderBytes + counter_bytes);
+    dim3 grid(n_chunks, max_nodes, batch);
+    ss::tree_verify_kernel<<<grid, ss::kVerifyThreads, 0, s>>>(
+        logits, draft_tokens, trees, max_nodes, vocab, n_chunks, accept_len, accept_path, last_node,
+        bonus_token, node_argmax, counters, partials);
+    return cudaGetLastError() == cudaSuccess ? SS_OK : SS_ERR_CUDA;
+}
