@@ -1,515 +1,819 @@
-// Tree-masked multi-stream attention, one layer (Eq. 1, Eq. 2): split-KV flash-decode.
+// Tree-masked multi-stream attention, one layer (Eq. 1, Eq. 2): split-KV flash-decode for sm_100a.
 //
-// Work decomposition.  For sequence b the "extended key sequence" of a head is
-//     [0, L_b)                      cached prefix,
-//     [L_b, L_b + T_b)              this step's tree nodes (already in the cache, masked by ancestry),
-//     [L_b + T_b, L_b + T_b(1+g))   the transient stream keys, node-major: (t,1)..(t,g), (t+1,1)...
-// All (sequence, head) pairs are laid end to end in units of 16 keys and the persistent grid cuts
-// that line into equal spans, so every CTA streams the same number of K/V bytes whatever the
-// batch's length mix.  The cut points are computed on the device from kv_len[], so the host never
-// needs the lengths.  A span crossing a pair boundary yields several segments; each segment of a
-// pair that is split over CTAs leaves an un-normalised partial (m, l, O) in the workspace, and the
-// last CTA to arrive on the pair's counter merges them (no CTA ever waits for another).
+// Work decomposition.  A thread-block cluster of C CTAs owns one (sequence, head) pair.  The pair's
+// keys are the cached slots [0, L+T) (prefix, then this step's tree nodes, masked by ancestry) and
+// the T*gamma transient stream keys (node-major).  They are cut into 16-key units and CTA r of the
+// cluster takes units [U*r/C, U*(r+1)/C), so every CTA of a pair streams the same number of bytes.
 //
-// Inside a CTA: all (node x stream) query rows of the head are processed against each staged K/V
-// tile, 64 rows per pass; warp (rb, kh) owns 16 rows x one 32-key half of the 64-key tile, S = QK^T
-// and O += PV run on bf16 tensor-core MMAs with fp32 accumulators, the online softmax lives in
-// registers, and the tree / stream mask is evaluated from the node's 64-bit ancestor word only for
-// tiles that reach past the prefix.
+// Inside a CTA.  ALL query rows of the head -- T main rows, then the T*gamma stream rows -- sit in
+// shared memory as up to three 128-row blocks, so each K/V tile that TMA brings in is used by every
+// (node x stream) row: the prefix crosses HBM once per head, not once per stream.
+//   warp 0      TMA producer: Q once, then 64-key K/V tiles into a ring of stages (mbarrier
+//               complete_tx); swizzle-128B boxes straight from the caller's strided tensors.
+//   warp 1      tcgen05 issuer: S = Q K^T (128 x 64 x d) into one of two TMEM buffers, later
+//               O += P V (128 x d x 64) into the block's TMEM accumulator; tcgen05.commit arrives
+//               on the mbarriers that hand buffers back.
+//   warps 4..   one warpgroup per 128-row block, one thread per query row: tcgen05.ld of the S row,
+//               tree / stream mask from the node's 64-bit ancestor word, online softmax in fp32
+//               registers (the running maximum is only raised when it would grow by more than 2^8,
+//               which keeps the TMEM accumulator untouched on almost every tile), P as bf16 into a
+//               swizzled shared-memory tile that feeds the second MMA.
+// Split-KV merge.  Each CTA ends with un-normalised (m, l, O) per row.  CTA r of the cluster merges
+// rows [128/C * r, 128/C * (r+1)) of every block: all CTAs push those rows into r's shared memory
+// (st.shared::cluster), one cluster barrier, then r combines the C partials and writes bf16 output.
+// No CTA ever spins on another: the only cross-CTA waits are hardware cluster barriers that every
+// thread reaches unconditionally; every mbarrier wait is bounded and reports SS_ERR_DEVICE_TIMEOUT.
+#include <cuda.h>
 #include <cuda_bf16.h>
 
 #include "ss_common.cuh"
 
 namespace ss {
 
-constexpr int kThreads = 256;
-constexpr int kTileKeys = 64;      // keys per staged tile
-constexpr int kUnit = 16;          // scheduling granularity (keys)
-constexpr int kRowChunk = 64;      // query rows per pass
-constexpr int kStages = 3;
-constexpr int kMinUnitsPerCta = 4; // do not spread less than 64 keys per CTA
+constexpr int kTileKeys = 64;        // keys per staged tile (N of the S MMA, K of the PV MMA)
+constexpr int kUnit = 16;            // split granularity (keys)
+constexpr int kBlockRows = 128;      // query rows per block (M of both MMAs)
+constexpr int kMaxBlocks = 3;        // 64 main rows + 256 stream rows = 320 rows at most
+constexpr int kMaxStages = 6;
+constexpr int kAuxThreads = 128;     // warps 0..3: producer, MMA issuer, two spare
+constexpr int kHalfBytes = 64 * 128; // one TMA box: 64 rows x 128 B (64 bf16 of head_dim)
+constexpr int kPBytes = kBlockRows * 128;   // one P tile: 128 rows x 64 keys bf16
+constexpr int kMaxDynSmem = 232448 - 4096;  // 227 KB per CTA less the static control block
+constexpr float kRescaleStep = 8.f;  // raise the running maximum only when it grows by more than 2^8
+constexpr long long kWaitCycles = 2000000000ll;   // bound of every mbarrier wait (~1 s)
 
-struct AttnArgs {
+struct alignas(64) AttnArgs {
+    CUtensorMap tm_k, tm_v;          // cache slab    dims (d, H, slots)        box (64, 1, 64)
+    CUtensorMap tm_qm;               // q_main        dims (d, H, B*Tmax)       box (64, 1, tmax8)
+    CUtensorMap tm_qs;               // q_spec        dims (d, H, B*Tmax*g)     box (64, 1, spec_rows)
+    CUtensorMap tm_ks, tm_vs;        // k_spec/v_spec dims (d, H, B*Tmax*g)     box (64, 1, 64)
     int batch, n_heads, gamma, max_nodes;
-    float scale_log2;              // sm_scale * log2(e)
-    const __nv_bfloat16* q_main;
+    int tmax8;                       // max_nodes rounded up to 8: first stream row in shared memory
+    int spec_rows;                   // max_nodes * gamma rounded up to 8 (rows of the q_spec box)
+    int n_blocks, n_stages, cluster;
+    int head_coord;                  // 1, or 0 when all heads share one K/V (head stride 0)
+    float scale_log2;                // sm_scale * log2(e)
     __nv_bfloat16* o_main;
-    const __nv_bfloat16* q_spec;
-    const __nv_bfloat16* k_spec;
-    const __nv_bfloat16* v_spec;
     __nv_bfloat16* o_spec;
-    const __nv_bfloat16* k_cache;
-    const __nv_bfloat16* v_cache;
-    long long slot_stride, head_stride;
+    float* lse_main;
+    float* lse_spec;
     const long long* kv_start;
     const int* kv_len;
     const int* kv_capacity;
     const ss_tree_desc* trees;
-    float* lse_main;
-    float* lse_spec;
-    int* status;                   // workspace word 0
-    int* counters;                 // [batch * n_heads]
-    float* partials;               // [2 * grid][m_pad][HD + 2]
-    int m_pad;                     // rows per partial slot
+    int* status;
+};
+
+struct Ctrl {
+    unsigned long long q_full;
+    unsigned long long kv_full[kMaxStages], kv_empty[kMaxStages];
+    unsigned long long s_full[kMaxBlocks][2], s_free[2];   // s_full per (block, buffer): a warpgroup sees every phase of its own
+    unsigned long long p_full[kMaxBlocks], o_done[kMaxBlocks];
+    unsigned long long anc[SS_MAX_NODES];
+    float2 ml[kMaxBlocks][kBlockRows];   // (m, l) received for the rows this CTA merges: [block][src * rpc + lr]
+    uint32_t tmem_base;
+    int abort;
 };
 
 // ---------------------------------------------------------------------------------------------
-// small PTX wrappers
+// PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
-    const int n = valid ? 16 : 0;   // n = 0 zero-fills the 16 bytes
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(n));
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-    asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
 }
-__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
+__device__ __forceinline__ void st_cluster_v4(uint32_t addr, float x, float y, float z, float w) {
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(x), "f"(y), "f"(z), "f"(w) : "memory");
 }
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
+__device__ __forceinline__ void st_cluster_v2(uint32_t addr, float x, float y) {
+    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(x), "f"(y) : "memory");
 }
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
     asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
 }
+// Bounded wait: gives up when another thread of the CTA already gave up, or after kWaitCycles.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort, int* status) {
+    const long long t0 = clock64();
+    for (;;) {
+        for (int i = 0; i < 256; ++i) {
+            if (mbar_try(bar, parity)) return true;
+            if (*abort) return false;
+        }
+        if (clock64() - t0 > kWaitCycles) {
+            *abort = 1;
+            set_status(status, SS_ERR_DEVICE_TIMEOUT);
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort, int* status) {
+    if (mbar_try(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort, status);
+}
+// the same for a whole warp: either every lane saw the phase complete or every lane gives up
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort, int* status) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort, status));
+}
+// after giving up: a short bounded wait that lets a copy already in flight land
+__device__ __noinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
+    const long long t0 = clock64();
+    while (!mbar_try(bar, parity) && clock64() - t0 < kWaitCycles / 16) {}
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem], bf16 inputs, fp32 accumulate
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+#define SS_R16(r, o) "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), \
+                     "=r"(r[o + 6]), "=r"(r[o + 7]), "=r"(r[o + 8]), "=r"(r[o + 9]), "=r"(r[o + 10]), "=r"(r[o + 11]), \
+                     "=r"(r[o + 12]), "=r"(r[o + 13]), "=r"(r[o + 14]), "=r"(r[o + 15])
+#define SS_W16(r, o) "r"(r[o + 0]), "r"(r[o + 1]), "r"(r[o + 2]), "r"(r[o + 3]), "r"(r[o + 4]), "r"(r[o + 5]), \
+                     "r"(r[o + 6]), "r"(r[o + 7]), "r"(r[o + 8]), "r"(r[o + 9]), "r"(r[o + 10]), "r"(r[o + 11]), \
+                     "r"(r[o + 12]), "r"(r[o + 13]), "r"(r[o + 14]), "r"(r[o + 15])
+// 16 consecutive fp32 columns of this thread's TMEM lane <-> registers r[o .. o+15]
+template <int O, int N>
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[N]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : SS_R16(r, O) : "r"(taddr) : "memory");
+}
+template <int O, int N>
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[N]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
+        ::SS_W16(r, O), "r"(taddr) : "memory");
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// Shared-memory matrix descriptors (swizzle-128B canonical layouts, 8-row groups 1024 B apart).
+//   K-major  (Q, K, P): rows of 128 B, the contraction index contiguous; a 16-element step is +32 B.
+//   MN-major (V): rows of 128 B are keys (contraction), the 64 contiguous elements are head_dim;
+//                 the next 64 elements of head_dim start `lbo` bytes further; a 16-key step is +2048 B.
+__device__ __forceinline__ uint64_t desc_k_major(uint32_t addr) {
+    return static_cast<uint64_t>((addr & 0x3FFFFu) >> 4) | (1ull << 16) | (static_cast<uint64_t>(1024 >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ uint64_t desc_mn_major(uint32_t addr, uint32_t lbo) {
+    return static_cast<uint64_t>((addr & 0x3FFFFu) >> 4) | (static_cast<uint64_t>(lbo >> 4) << 16) |
+           (static_cast<uint64_t>(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: fp32 accumulator, bf16 A and B, M = 128
+__host__ __device__ constexpr uint32_t idesc_bf16(int n, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | (static_cast<uint32_t>(n >> 3) << 17) |
+           (static_cast<uint32_t>(kBlockRows >> 4) << 24);
+}
+
 // ---------------------------------------------------------------------------------------------
-// schedule: the line of 16-key units over all (sequence, head) pairs
-struct Schedule {
-    long long total_units;
-    int g_eff;
+// The CTA's share of the pair's keys, as a list of tiles.  Every role derives it from the same
+// four numbers, so no tile list is ever stored.
+struct Span {
+    int L, T, n_stream;            // prefix length, tree nodes, stream keys (T * gamma)
+    int kc0, kc1;                  // cache keys [kc0, kc1) (indices into [0, L+T))
+    int ks0, ks1;                  // stream keys [ks0, ks1) (indices into [0, T*gamma))
+    int n_cache_tiles, n_tiles;
+    int tmax8, gamma, n_blocks;
+    int main_rows, spec_end;       // valid rows: [0, main_rows) and [tmax8, spec_end)
+
+    __device__ __forceinline__ bool is_cache(int j) const { return j < n_cache_tiles; }
+    __device__ __forceinline__ int first_key(int j) const {
+        return j < n_cache_tiles ? kc0 + j * kTileKeys : ks0 + (j - n_cache_tiles) * kTileKeys;
+    }
+    __device__ __forceinline__ int valid_keys(int j) const {
+        return min(kTileKeys, (j < n_cache_tiles ? kc1 : ks1) - first_key(j));
+    }
+    // does row block `blk` hold a row that can see a key of tile j?
+    __device__ __forceinline__ bool active(int j, int blk) const {
+        const int r0 = blk * kBlockRows, r1 = r0 + kBlockRows;
+        if (j < n_cache_tiles) return r0 < main_rows || (r0 < spec_end && r1 > tmax8);
+        // stream key s is seen by the stream rows s .. (end of its node's group)
+        const int s0 = first_key(j), s_last = s0 + valid_keys(j) - 1;
+        const int row_lo = tmax8 + s0, row_hi = tmax8 + (s_last / gamma) * gamma + gamma - 1;
+        return row_lo < r1 && row_hi >= r0;
+    }
+    // next active (tile, block) after (j, blk) in tile-major order; j == n_tiles when exhausted
+    __device__ __forceinline__ void next(int& j, int& blk) const {
+        for (;;) {
+            if (++blk >= n_blocks) { blk = 0; ++j; }
+            if (j >= n_tiles || active(j, blk)) return;
+        }
+    }
+    __device__ __forceinline__ void first(int& j, int& blk) const {
+        j = 0; blk = -1;
+        if (n_tiles == 0) { blk = 0; return; }
+        next(j, blk);
+    }
 };
 
-__device__ __forceinline__ int ext_keys(const AttnArgs& a, int b) {
-    return a.kv_len[b] + a.trees[b].n_nodes * (1 + a.gamma);
+__device__ __forceinline__ Span make_span(const AttnArgs& a, int L, int T, int rank) {
+    Span s;
+    s.L = L; s.T = T; s.gamma = a.gamma; s.tmax8 = a.tmax8; s.n_blocks = a.n_blocks;
+    s.n_stream = T * a.gamma;
+    s.main_rows = T;
+    s.spec_end = a.tmax8 + s.n_stream;
+    const int ec = L + T;
+    const int uc = (ec + kUnit - 1) / kUnit, us = (s.n_stream + kUnit - 1) / kUnit;
+    const int u = uc + us;
+    const int u0 = static_cast<int>(static_cast<long long>(u) * rank / a.cluster);
+    const int u1 = static_cast<int>(static_cast<long long>(u) * (rank + 1) / a.cluster);
+    s.kc0 = min(u0, uc) * kUnit;
+    s.kc1 = min(min(u1, uc) * kUnit, ec);
+    s.ks0 = (max(u0, uc) - uc) * kUnit;
+    s.ks1 = min((max(u1, uc) - uc) * kUnit, s.n_stream);
+    s.n_cache_tiles = s.kc1 > s.kc0 ? (s.kc1 - s.kc0 + kTileKeys - 1) / kTileKeys : 0;
+    const int nst = s.ks1 > s.ks0 ? (s.ks1 - s.ks0 + kTileKeys - 1) / kTileKeys : 0;
+    s.n_tiles = s.n_cache_tiles + nst;
+    return s;
 }
-__device__ __forceinline__ long long span_begin(long long total, int g_eff, int c) { return total * c / g_eff; }
-// the CTA whose span holds unit x
-__device__ __forceinline__ int cta_of(long long total, int g_eff, long long x) {
-    return static_cast<int>(((x + 1) * g_eff - 1) / total);
+
+// Row r of the head's query tile: rows [0, T) are the main-stream rows of nodes 0..T-1, rows
+// [tmax8, tmax8 + T*gamma) the stream rows in (node, stream) order; everything else is padding.
+struct RowInfo {
+    bool valid;
+    int node, stream;              // stream 0 = main row, 1..gamma = speculative stream
+};
+__device__ __forceinline__ RowInfo row_info(const Span& s, int row) {
+    RowInfo r;
+    if (row < s.tmax8) {
+        r.valid = row < s.main_rows; r.node = row; r.stream = 0;
+    } else {
+        const int x = row - s.tmax8;
+        r.valid = x < s.n_stream;
+        r.node = s.gamma > 0 ? x / s.gamma : 0;
+        r.stream = x - r.node * s.gamma + 1;
+    }
+    return r;
+}
+
+// Bit i set <=> key i of tile j is visible to the row (Eq. 1 / Eq. 2 with the tree mask of App. A).
+__device__ __forceinline__ unsigned long long visible_mask(const Span& s, int j, const RowInfo& r, unsigned long long anc) {
+    if (!r.valid) return 0ull;
+    const int x = s.first_key(j), nv = s.valid_keys(j);
+    const unsigned long long in_tile = nv >= 64 ? ~0ull : ((1ull << nv) - 1ull);
+    unsigned long long m;
+    if (s.is_cache(j)) {
+        if (x >= s.L) {                        // tree keys only: key x+i is node (x - L + i)
+            const int sh = x - s.L;
+            m = sh >= 64 ? 0ull : (anc >> sh);
+        } else {                               // prefix keys (all visible), then tree keys
+            const int np = s.L - x;
+            m = np >= 64 ? ~0ull : (((1ull << np) - 1ull) | (anc << np));
+        }
+    } else {                                   // stream keys: (node, 1..stream) of the row's own node
+        if (r.stream == 0) return 0ull;
+        const int lo = r.node * s.gamma - x, hi = lo + r.stream;      // visible tile positions [lo, hi)
+        const unsigned long long below_hi = hi >= 64 ? ~0ull : (hi <= 0 ? 0ull : ((1ull << hi) - 1ull));
+        const unsigned long long below_lo = lo >= 64 ? ~0ull : (lo <= 0 ? 0ull : ((1ull << lo) - 1ull));
+        m = below_hi & ~below_lo;
+    }
+    return m & in_tile;
 }
 
 template <int HD>
-struct Smem {
-    static constexpr int kPitch = HD * 2 + 16;                  // bytes per staged row (bank-conflict padding)
-    static constexpr int kTileBytes = kTileKeys * kPitch;       // one K (or V) tile
-    static constexpr int kStageBytes = 2 * kTileBytes;          // K + V
-    static constexpr int kQBytes = kRowChunk * kPitch;
-    static constexpr int kPipeBytes = kStages * kStageBytes;
-    static constexpr int kMergeBytes = 4 * 16 * (HD + 2) * 4;   // (m, l, O) of the four kh = 1 warps
-    static_assert(kMergeBytes <= kPipeBytes, "merge buffer aliases the pipeline stages");
-    static constexpr int kTotal = kPipeBytes + kQBytes;
+struct Geo {
+    static constexpr int kHalves = HD > 64 ? 2 : 1;               // 64-element boxes along head_dim
+    static constexpr int kStageBytes = 2 * kHalves * kHalfBytes;  // K + V
+    static constexpr int kKSteps = HD / 16;                       // MMA K steps of S = Q K^T
+    static constexpr int kMergePitch = HD + 4;                    // floats per row in the merge buffer
+    static constexpr uint32_t kIdescS = idesc_bf16(kTileKeys, false);
+    static constexpr uint32_t kIdescPV = idesc_bf16(HD, true);
+    static constexpr int kOCols = 128;                            // TMEM columns reserved per block accumulator
 };
 
+// ---------------------------------------------------------------------------------------------
 template <int HD>
-__global__ void __launch_bounds__(kThreads, 1) msa_attention_kernel(const AttnArgs a) {
-    extern __shared__ __align__(128) unsigned char smem[];
-    using S = Smem<HD>;
-    __shared__ unsigned long long s_anc[SS_MAX_NODES];
-    __shared__ int s_flag;
+__global__ void __launch_bounds__(kAuxThreads + kMaxBlocks * kBlockRows, 1)
+msa_attention_kernel(const __grid_constant__ AttnArgs a) {
+    using G = Geo<HD>;
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ Ctrl c;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int g = lane >> 2, q = lane & 3;
-    const int rb = warp & 3, kh = warp >> 2;
-    const int H = a.n_heads, gamma = a.gamma, rows_per_node = 1 + gamma;
+    const int C = a.cluster;
+    const uint32_t rank = C > 1 ? cluster_rank() : 0u;
+    const int pair = blockIdx.x / C;
+    const int b = pair / a.n_heads, h = pair - b * a.n_heads;
+    const int n_blocks = a.n_blocks, n_stages = a.n_stages;
+    volatile int* abort_flag = &c.abort;
 
-    // ---- schedule ------------------------------------------------------------------------------
-    long long total = 0;
-    for (int b = 0; b < a.batch; ++b) total += static_cast<long long>(H) * ((ext_keys(a, b) + kUnit - 1) / kUnit);
-    if (total == 0) return;
-    const int g_eff = static_cast<int>(min(static_cast<long long>(gridDim.x), max(1ll, total / kMinUnitsPerCta)));
-    const int cta = blockIdx.x;
-    if (cta >= g_eff) return;
-    long long u = span_begin(total, g_eff, cta);
-    const long long u_end = span_begin(total, g_eff, cta + 1);
+    // ---- shared-memory carve-up (1024-byte aligned: swizzle atoms) ----------------------------
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t q_rows = n_blocks * kBlockRows;
+    const uint32_t q_base = base;                                       // [half][q_rows][128 B]
+    const uint32_t p_base = q_base + G::kHalves * q_rows * 128u;        // [block][128 rows][128 B]
+    const uint32_t kv_base = p_base + n_blocks * kPBytes;               // [stage][K halves | V halves]
+    const uint32_t merge_base = base;                                   // aliases everything above, after the main loop
 
-    const uint32_t smem_base = smem_u32(smem);
-    const uint32_t q_base = smem_base + S::kPipeBytes;
-
-    int b = 0;
-    long long pair_base = 0;   // first unit of sequence b
-    while (u < u_end) {
-        // locate the pair that holds unit u
-        int units_b = (ext_keys(a, b) + kUnit - 1) / kUnit;
-        while (u >= pair_base + static_cast<long long>(H) * units_b) {
-            pair_base += static_cast<long long>(H) * units_b;
-            ++b;
-            units_b = (ext_keys(a, b) + kUnit - 1) / kUnit;
+    // ---- prologue ---------------------------------------------------------------------------------
+    if (tid == 0) {
+        mbar_init(smem_u32(&c.q_full), 1);
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(smem_u32(&c.kv_full[s]), 1); mbar_init(smem_u32(&c.kv_empty[s]), 1); }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(smem_u32(&c.s_free[s]), 4);
+            for (int k = 0; k < kMaxBlocks; ++k) mbar_init(smem_u32(&c.s_full[k][s]), 1);
         }
-        const int h = static_cast<int>((u - pair_base) / units_b);
-        const long long p0 = pair_base + static_cast<long long>(h) * units_b;   // pair's first unit
-        const long long p1 = p0 + units_b;
-        const long long seg_end_u = min(u_end, p1);
-        const int L = a.kv_len[b];
-        const int T = a.trees[b].n_nodes;
-        const int M = T * rows_per_node;
-        const int E = L + M;                                   // extended keys of the pair
-        const int e0 = static_cast<int>(u - p0) * kUnit;
-        const int e1 = min(E, static_cast<int>(seg_end_u - p0) * kUnit);
-        const bool continuation = (u > p0);
-        const int c_first = cta_of(total, g_eff, p0), c_last = cta_of(total, g_eff, p1 - 1);
-        const int n_splits = c_last - c_first + 1;
-        const bool over_capacity = a.kv_capacity != nullptr && L + T > a.kv_capacity[b];
-        if (over_capacity && tid == 0) set_status(a.status, SS_ERR_CAPACITY);
-        u = seg_end_u;
-        if (over_capacity) continue;
+        for (int s = 0; s < kMaxBlocks; ++s) { mbar_init(smem_u32(&c.p_full[s]), kBlockRows); mbar_init(smem_u32(&c.o_done[s]), 1); }
+        c.abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        tma_prefetch_desc(&a.tm_k); tma_prefetch_desc(&a.tm_v); tma_prefetch_desc(&a.tm_qm);
+        if (a.gamma > 0) { tma_prefetch_desc(&a.tm_qs); tma_prefetch_desc(&a.tm_ks); tma_prefetch_desc(&a.tm_vs); }
+    }
+    const uint32_t tmem_cols = n_blocks == 1 ? 256u : 512u;
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&c.tmem_base)), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    int L = a.kv_len[b];
+    int T = min(max(a.trees[b].n_nodes, 0), a.max_nodes);
+    const long long slot0 = a.kv_start[b];
+    bool skip = false;                                    // sequence over its slot capacity: nothing read or written
+    if (L < 0 || (a.kv_capacity != nullptr && L + T > a.kv_capacity[b])) {
+        skip = true;
+        if (tid == 0) set_status(a.status, SS_ERR_CAPACITY);
+    }
+    if (skip) { L = 0; T = 0; }
+    if (tid >= kAuxThreads && tid < kAuxThreads + SS_MAX_NODES) c.anc[tid - kAuxThreads] = a.trees[b].anc_mask[tid - kAuxThreads];
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = c.tmem_base;
+    const uint32_t tmem_s = tmem + n_blocks * G::kOCols;  // two S buffers of 64 columns
 
-        __syncthreads();   // previous segment is completely done with shared memory
-        if (tid < SS_MAX_NODES) s_anc[tid] = a.trees[b].anc_mask[tid];
+    const Span sp = make_span(a, L, T, static_cast<int>(rank));
+    const long long spec_row0 = static_cast<long long>(b) * a.max_nodes * a.gamma;   // first stream row of the sequence
 
-        const long long seq_slot0 = a.kv_start[b];
-        const __nv_bfloat16* kc = a.k_cache + seq_slot0 * a.slot_stride + static_cast<long long>(h) * a.head_stride;
-        const __nv_bfloat16* vc = a.v_cache + seq_slot0 * a.slot_stride + static_cast<long long>(h) * a.head_stride;
-        const long long spec_row0 = static_cast<long long>(b) * a.max_nodes * gamma;   // [b][0][0]
-        float* part = a.partials + static_cast<size_t>(2 * cta + (continuation ? 0 : 1)) * a.m_pad * (HD + 2);
-
-        const int n_tiles = (e1 - e0 + kTileKeys - 1) / kTileKeys;
-        const int n_chunks = (M + kRowChunk - 1) / kRowChunk;
-
-        for (int rc = 0; rc < n_chunks; ++rc) {
-            const int row_base = rc * kRowChunk;
-            __syncthreads();   // shared memory of the previous pass is free; s_anc is visible
-            // ---- stage the query rows of this pass -------------------------------------------
-            for (int i = tid; i < kRowChunk * (HD / 8); i += kThreads) {
-                const int r = i / (HD / 8), ch = i - r * (HD / 8);
-                const int row = row_base + r;
-                const bool valid = row < M;
-                const __nv_bfloat16* src = a.q_main;
-                if (valid) {
-                    const int t = row / rows_per_node, j = row - t * rows_per_node;
-                    if (j == 0)
-                        src = a.q_main + ((static_cast<long long>(b) * a.max_nodes + t) * H + h) * HD + ch * 8;
-                    else
-                        src = a.q_spec + ((spec_row0 + static_cast<long long>(t) * gamma + (j - 1)) * H + h) * HD + ch * 8;
-                }
-                cp_async16(q_base + r * S::kPitch + ch * 16, src, valid);
+    // ================================= warp 0: TMA producer =====================================
+    if (warp == 0) {
+        if (lane == 0 && sp.n_tiles > 0) {
+            const uint32_t qbytes = G::kHalves * (a.tmax8 + (a.gamma > 0 ? a.spec_rows : 0)) * 128u;
+            mbar_expect_tx(smem_u32(&c.q_full), qbytes);
+            for (int hh = 0; hh < G::kHalves; ++hh) {
+                tma_load_3d(q_base + hh * q_rows * 128u, &a.tm_qm, hh * 64, h, b * a.max_nodes, smem_u32(&c.q_full));
+                if (a.gamma > 0)
+                    tma_load_3d(q_base + hh * q_rows * 128u + a.tmax8 * 128u, &a.tm_qs, hh * 64, h,
+                                static_cast<int>(spec_row0), smem_u32(&c.q_full));
             }
-            // ---- K/V tile loader ---------------------------------------------------------------
-            auto issue_tile = [&](int tile) {
-                const uint32_t kdst = smem_base + (tile % kStages) * S::kStageBytes;
-                const uint32_t vdst = kdst + S::kTileBytes;
-                const int eb = e0 + tile * kTileKeys;
-                for (int i = tid; i < kTileKeys * (HD / 8); i += kThreads) {
-                    const int r = i / (HD / 8), ch = i - r * (HD / 8);
-                    const int e = eb + r;
-                    const bool valid = e < e1;
-                    const __nv_bfloat16 *ks = kc, *vs = vc;
-                    if (valid) {
-                        if (e < L + T) {
-                            ks = kc + static_cast<long long>(e) * a.slot_stride + ch * 8;
-                            vs = vc + static_cast<long long>(e) * a.slot_stride + ch * 8;
-                        } else {
-                            const long long off = ((spec_row0 + (e - L - T)) * H + h) * HD + ch * 8;
-                            ks = a.k_spec + off;
-                            vs = a.v_spec + off;
-                        }
+            int issued = 0;
+            for (int j = 0; j < sp.n_tiles; ++j) {
+                const int st = j % n_stages;
+                if (j >= n_stages && !mbar_wait(smem_u32(&c.kv_empty[st]), ((j / n_stages) - 1) & 1, abort_flag, a.status)) break;
+                const uint32_t bar = smem_u32(&c.kv_full[st]);
+                mbar_expect_tx(bar, G::kStageBytes);
+                const uint32_t kdst = kv_base + st * G::kStageBytes, vdst = kdst + G::kHalves * kHalfBytes;
+                const int x = sp.first_key(j);
+                for (int hh = 0; hh < G::kHalves; ++hh) {
+                    if (sp.is_cache(j)) {
+                        const int slot = static_cast<int>(slot0 + x);
+                        tma_load_3d(kdst + hh * kHalfBytes, &a.tm_k, hh * 64, h * a.head_coord, slot, bar);
+                        tma_load_3d(vdst + hh * kHalfBytes, &a.tm_v, hh * 64, h * a.head_coord, slot, bar);
+                    } else {
+                        const int row = static_cast<int>(spec_row0 + x);
+                        tma_load_3d(kdst + hh * kHalfBytes, &a.tm_ks, hh * 64, h, row, bar);
+                        tma_load_3d(vdst + hh * kHalfBytes, &a.tm_vs, hh * 64, h, row, bar);
                     }
-                    cp_async16(kdst + r * S::kPitch + ch * 16, ks, valid);
-                    cp_async16(vdst + r * S::kPitch + ch * 16, vs, valid);
                 }
+                issued = j + 1;
+            }
+            if (*abort_flag) {
+                // gave up: let the copies already in flight land before shared memory is reused or released
+                mbar_drain(smem_u32(&c.q_full), 0);
+                for (int j = max(0, issued - n_stages); j < issued; ++j)
+                    mbar_drain(smem_u32(&c.kv_full[j % n_stages]), (j / n_stages) & 1);
+            }
+        }
+    }
+    // ================================= warp 1: MMA issuer =======================================
+    else if (warp == 1) {
+        if (lane == 0 && sp.n_tiles > 0) {
+            bool ok = mbar_wait(smem_u32(&c.q_full), 0, abort_flag, a.status);
+            int n_done[kMaxBlocks] = {0, 0, 0};        // PV MMAs issued per block
+            int waited_tile = -1;                      // last tile whose kv_full was observed
+            auto issue_s = [&](int j, int blk, int q) -> bool {
+                const int st = j % n_stages;
+                if (waited_tile != j) {
+                    if (!mbar_wait(smem_u32(&c.kv_full[st]), (j / n_stages) & 1, abort_flag, a.status)) return false;
+                    waited_tile = j;
+                }
+                const int buf = q & 1;
+                if (q >= 2 && !mbar_wait(smem_u32(&c.s_free[buf]), ((q >> 1) - 1) & 1, abort_flag, a.status)) return false;
+                tc_fence_after();
+                const uint32_t qa = q_base + blk * (kBlockRows * 128u);
+                const uint32_t ka = kv_base + st * G::kStageBytes;
+                #pragma unroll
+                for (int ks = 0; ks < G::kKSteps; ++ks) {
+                    const uint32_t hh = ks >> 2, off = (ks & 3) * 32u;
+                    tc_mma(tmem_s + buf * kTileKeys, desc_k_major(qa + hh * q_rows * 128u + off),
+                           desc_k_major(ka + hh * kHalfBytes + off), G::kIdescS, ks > 0);
+                }
+                tc_commit(smem_u32(&c.s_full[blk][buf]));
+                return true;
             };
-            #pragma unroll
-            for (int s = 0; s < kStages - 1; ++s) {
-                if (s < n_tiles) issue_tile(s);
-                cp_async_commit();
+            int j, blk, q = 0;
+            sp.first(j, blk);
+            if (ok && j < sp.n_tiles) ok = issue_s(j, blk, 0);
+            while (ok && j < sp.n_tiles) {
+                int nj = j, nblk = blk;
+                sp.next(nj, nblk);
+                if (nj < sp.n_tiles && !issue_s(nj, nblk, q + 1)) break;
+                // O[blk] (+)= P[blk] V[tile j]
+                if (!mbar_wait(smem_u32(&c.p_full[blk]), n_done[blk] & 1, abort_flag, a.status)) break;
+                tc_fence_after();
+                const int st = j % n_stages;
+                const uint32_t pa = p_base + blk * kPBytes;
+                const uint32_t va = kv_base + st * G::kStageBytes + G::kHalves * kHalfBytes;
+                #pragma unroll
+                for (int ks = 0; ks < kTileKeys / 16; ++ks)
+                    tc_mma(tmem + blk * G::kOCols, desc_k_major(pa + ks * 32u), desc_mn_major(va + ks * 2048u, kHalfBytes),
+                           G::kIdescPV, (n_done[blk] > 0 || ks > 0) ? 1u : 0u);
+                tc_commit(smem_u32(&c.o_done[blk]));
+                if (nj != j) tc_commit(smem_u32(&c.kv_empty[st]));     // last block of tile j: the stage is free
+                ++n_done[blk];
+                j = nj; blk = nblk; ++q;
             }
-
-            // ---- per-thread row info ----------------------------------------------------------
-            // thread rows: r_lo = row_base + rb*16 + g, r_hi = r_lo + 8
-            int row_id[2];
-            unsigned long long anc[2];
-            int s_lo[2], s_hi[2];   // visible stream-key range [s_lo, s_hi) in extended key indices
-            #pragma unroll
-            for (int x = 0; x < 2; ++x) {
-                const int row = row_base + rb * 16 + g + 8 * x;
-                row_id[x] = row;
-                if (row < M) {
-                    const int t = row / rows_per_node, j = row - t * rows_per_node;
-                    anc[x] = s_anc[t];
-                    s_lo[x] = L + T + t * gamma;
-                    s_hi[x] = s_lo[x] + j;
-                } else {
-                    anc[x] = 0ull;
-                    s_lo[x] = s_hi[x] = 0;
+        }
+    }
+    // ============================ warps 4..: softmax warpgroups =================================
+    // per-thread partial of this CTA's key span, kept for the merge
+    float m_run = -INFINITY, l_run = 0.f;
+    int n_own = 0;
+    const int my_blk = (warp - 4) >> 2;
+    const int row_in_blk = ((warp & 3) << 5) | lane;
+    const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    RowInfo ri;
+    ri.valid = false; ri.node = 0; ri.stream = 0;
+    if (warp >= 4) {
+        const int row = my_blk * kBlockRows + row_in_blk;
+        ri = row_info(sp, row);
+        const unsigned long long anc = ri.valid ? c.anc[ri.node] : 0ull;
+        // a warp whose 32 rows are all padding skips the arithmetic but keeps the barrier protocol
+        const bool warp_active = __any_sync(0xffffffffu, ri.valid);
+        const uint32_t o_addr = tmem + lane_base + my_blk * G::kOCols;
+        const uint32_t p_row = p_base + my_blk * kPBytes + row_in_blk * 128u;
+        int j, blk, q = 0;
+        sp.first(j, blk);
+        bool ok = true;
+        int prev_tile = -1;
+        int n_use0 = 0, n_use1 = 0;                    // S buffers of this block consumed so far, per buffer
+        while (ok && j < sp.n_tiles) {
+            const bool first_of_tile = (j != prev_tile);
+            prev_tile = j;
+            if (blk == my_blk) {
+                const int buf = q & 1;
+                if (!mbar_wait_warp(smem_u32(&c.s_full[my_blk][buf]), (buf ? n_use1 : n_use0) & 1, abort_flag, a.status)) break;
+                if (buf) ++n_use1; else ++n_use0;
+                tc_fence_after();
+                uint32_t sr[kTileKeys];
+                if (warp_active) {
+                    const uint32_t s_addr = tmem_s + lane_base + buf * kTileKeys;
+                    tmem_ld16<0>(s_addr, sr); tmem_ld16<16>(s_addr + 16, sr);
+                    tmem_ld16<32>(s_addr + 32, sr); tmem_ld16<48>(s_addr + 48, sr);
+                    tmem_wait_ld();
                 }
-            }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&c.s_free[buf]));
 
-            uint32_t qf[HD / 16][4];
-            float o[HD / 8][4];
-            float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-            #pragma unroll
-            for (int i = 0; i < HD / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
-
-            const bool warp_active = (row_base + rb * 16) < M;
-
-            for (int tile = 0; tile < n_tiles; ++tile) {
-                cp_async_wait<kStages - 2>();
-                __syncthreads();
-                if (tile + kStages - 1 < n_tiles) issue_tile(tile + kStages - 1);
-                cp_async_commit();
-                if (tile == 0) {
-                    #pragma unroll
-                    for (int ks = 0; ks < HD / 16; ++ks)
-                        ldmatrix_x4(qf[ks], q_base + (rb * 16 + (lane & 15)) * S::kPitch + ks * 32 + (lane >> 4) * 16);
-                }
-                if (!warp_active) continue;
-                const uint32_t kbase = smem_base + (tile % kStages) * S::kStageBytes;
-                const uint32_t vbase = kbase + S::kTileBytes;
-                const int eb = e0 + tile * kTileKeys + kh * 32;   // first key of this warp's half tile
-                if (eb >= e1) continue;                            // warp-uniform
-
-                // ---- S = Q K^T over 32 keys ------------------------------------------------------
-                float s[4][4];
-                #pragma unroll
-                for (int i = 0; i < 4; ++i) s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
-                const int mid = lane >> 3;
-                #pragma unroll
-                for (int ks = 0; ks < HD / 16; ++ks) {
-                    #pragma unroll
-                    for (int kp = 0; kp < 2; ++kp) {
-                        uint32_t bf[4];
-                        const int key = kh * 32 + kp * 16 + (mid >> 1) * 8 + (lane & 7);
-                        ldmatrix_x4(bf, kbase + key * S::kPitch + ks * 32 + (mid & 1) * 16);
-                        mma_bf16(s[2 * kp], qf[ks], bf[0], bf[1]);
-                        mma_bf16(s[2 * kp + 1], qf[ks], bf[2], bf[3]);
-                    }
-                }
-                // ---- scale + mask -----------------------------------------------------------------
-                const bool need_mask = (eb + 32 > L) || (eb + 32 > e1);
-                #pragma unroll
-                for (int nt = 0; nt < 4; ++nt) {
-                    #pragma unroll
-                    for (int x = 0; x < 4; ++x) {
-                        float v = s[nt][x] * a.scale_log2;
-                        if (need_mask) {
-                            const int e = eb + nt * 8 + 2 * q + (x & 1);
-                            const int rr = x >> 1;
-                            bool vis;
-                            if (e >= e1) vis = false;
-                            else if (e < L) vis = true;
-                            else if (e < L + T) vis = (anc[rr] >> (e - L)) & 1ull;
-                            else vis = (e >= s_lo[rr]) && (e < s_hi[rr]);
-                            if (!vis) v = -INFINITY;
-                        }
-                        s[nt][x] = v;
-                    }
-                }
-                // ---- online softmax ---------------------------------------------------------------
-                uint32_t pa[2][4];
-                #pragma unroll
-                for (int rr = 0; rr < 2; ++rr) {
+                float corr = 1.f;
+                bool need = false;
+                if (warp_active) {
+                    const int x = sp.first_key(j);
+                    const bool masked = !sp.is_cache(j) || x + kTileKeys > sp.L || sp.valid_keys(j) < kTileKeys;
+                    const unsigned long long vis = masked ? visible_mask(sp, j, ri, anc) : (ri.valid ? ~0ull : 0ull);
+                    const uint32_t vlo = static_cast<uint32_t>(vis), vhi = static_cast<uint32_t>(vis >> 32);
                     float mx = -INFINITY;
                     #pragma unroll
-                    for (int nt = 0; nt < 4; ++nt) mx = fmaxf(mx, fmaxf(s[nt][2 * rr], s[nt][2 * rr + 1]));
-                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                    const float m_new = fmaxf(m_run[rr], mx);
-                    const float m_use = (m_new == -INFINITY) ? 0.f : m_new;   // all-masked row: every p is 0
-                    const float corr = exp2f(m_run[rr] - m_use);
+                    for (int i = 0; i < kTileKeys; ++i) {
+                        const bool v = ((i < 32 ? vlo : vhi) >> (i & 31)) & 1u;
+                        const float s = v ? __uint_as_float(sr[i]) * a.scale_log2 : -INFINITY;
+                        sr[i] = __float_as_uint(s);
+                        mx = fmaxf(mx, s);
+                    }
+                    need = mx > m_run + kRescaleStep;
+                    if (need) {
+                        corr = exp2f(m_run - mx);           // 0 when nothing was visible so far
+                        m_run = mx;
+                        l_run *= corr;
+                    }
+                }
+                // the previous PV of this block must be complete: it read the P tile that is about to
+                // be overwritten, and it wrote the accumulator that a raised maximum rescales
+                if (n_own > 0) {
+                    if (!mbar_wait_warp(smem_u32(&c.o_done[my_blk]), (n_own - 1) & 1, abort_flag, a.status)) break;
+                    tc_fence_after();
+                }
+                if (warp_active) {
+                    if (n_own > 0 && __any_sync(0xffffffffu, need)) {
+                        #pragma unroll
+                        for (int c0 = 0; c0 < HD; c0 += 16) {
+                            uint32_t orr[16];
+                            tmem_ld16<0>(o_addr + c0, orr);
+                            tmem_wait_ld();
+                            #pragma unroll
+                            for (int i = 0; i < 16; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * corr);
+                            tmem_st16<0>(o_addr + c0, orr);
+                        }
+                        tmem_wait_st();
+                    }
+                    const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
                     float sum = 0.f;
                     #pragma unroll
-                    for (int nt = 0; nt < 4; ++nt) {
-                        const float p0 = exp2f(s[nt][2 * rr] - m_use), p1 = exp2f(s[nt][2 * rr + 1] - m_use);
-                        sum += p0 + p1;
-                        s[nt][2 * rr] = p0;
-                        s[nt][2 * rr + 1] = p1;
-                    }
-                    sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-                    sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-                    l_run[rr] = l_run[rr] * corr + sum;
-                    m_run[rr] = m_new;
-                    #pragma unroll
-                    for (int i = 0; i < HD / 8; ++i) {
-                        o[i][2 * rr] *= corr;
-                        o[i][2 * rr + 1] *= corr;
-                    }
-                }
-                #pragma unroll
-                for (int kp = 0; kp < 2; ++kp) {
-                    pa[kp][0] = pack_bf16(s[2 * kp][0], s[2 * kp][1]);
-                    pa[kp][1] = pack_bf16(s[2 * kp][2], s[2 * kp][3]);
-                    pa[kp][2] = pack_bf16(s[2 * kp + 1][0], s[2 * kp + 1][1]);
-                    pa[kp][3] = pack_bf16(s[2 * kp + 1][2], s[2 * kp + 1][3]);
-                }
-                // ---- O += P V ---------------------------------------------------------------------
-                #pragma unroll
-                for (int kp = 0; kp < 2; ++kp) {
-                    #pragma unroll
-                    for (int dn = 0; dn < HD / 16; ++dn) {
-                        uint32_t bf[4];
-                        const int key = kh * 32 + kp * 16 + (mid & 1) * 8 + (lane & 7);
-                        ldmatrix_x4_trans(bf, vbase + key * S::kPitch + dn * 32 + (mid >> 1) * 16);
-                        mma_bf16(o[2 * dn], pa[kp], bf[0], bf[1]);
-                        mma_bf16(o[2 * dn + 1], pa[kp], bf[2], bf[3]);
-                    }
-                }
-            }
-            cp_async_wait<0>();
-            __syncthreads();   // all tiles consumed: the stage buffers may be reused for the merge
-
-            // ---- merge the two key halves (kh = 1 -> kh = 0) through shared memory -------------
-            float* mrg = reinterpret_cast<float*>(smem) + rb * 16 * (HD + 2);
-            if (kh == 1) {
-                #pragma unroll
-                for (int rr = 0; rr < 2; ++rr) {
-                    float* dst = mrg + (g + 8 * rr) * (HD + 2);
-                    if (q == 0) { dst[HD] = m_run[rr]; dst[HD + 1] = l_run[rr]; }
-                    #pragma unroll
-                    for (int i = 0; i < HD / 8; ++i) {
-                        dst[i * 8 + 2 * q] = o[i][2 * rr];
-                        dst[i * 8 + 2 * q + 1] = o[i][2 * rr + 1];
-                    }
-                }
-            }
-            __syncthreads();
-            if (kh == 0 && warp_active) {
-                #pragma unroll
-                for (int rr = 0; rr < 2; ++rr) {
-                    const float* src = mrg + (g + 8 * rr) * (HD + 2);
-                    const float m2 = src[HD], l2 = src[HD + 1];
-                    const float m_new = fmaxf(m_run[rr], m2);
-                    const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-                    const float c1 = exp2f(m_run[rr] - m_use), c2 = exp2f(m2 - m_use);
-                    l_run[rr] = l_run[rr] * c1 + l2 * c2;
-                    m_run[rr] = m_new;
-                    #pragma unroll
-                    for (int i = 0; i < HD / 8; ++i) {
-                        o[i][2 * rr] = o[i][2 * rr] * c1 + src[i * 8 + 2 * q] * c2;
-                        o[i][2 * rr + 1] = o[i][2 * rr + 1] * c1 + src[i * 8 + 2 * q + 1] * c2;
-                    }
-                }
-                // ---- write: final rows when the pair is not split, else the partial -----------
-                #pragma unroll
-                for (int rr = 0; rr < 2; ++rr) {
-                    const int row = row_id[rr];
-                    if (row >= M) continue;
-                    if (n_splits == 1) {
-                        const int t = row / rows_per_node, j = row - t * rows_per_node;
-                        const float inv = 1.f / l_run[rr];
-                        __nv_bfloat16* dst;
-                        float* lse = nullptr;
-                        if (j == 0) {
-                            const long long idx = (static_cast<long long>(b) * a.max_nodes + t) * H + h;
-                            dst = a.o_main + idx * HD;
-                            if (a.lse_main) lse = a.lse_main + idx;
-                        } else {
-                            const long long idx = (spec_row0 + static_cast<long long>(t) * gamma + (j - 1)) * H + h;
-                            dst = a.o_spec + idx * HD;
-                            if (a.lse_spec) lse = a.lse_spec + idx;
+                    for (int ch = 0; ch < 8; ++ch) {           // 8 chunks of 8 keys = 16 B of bf16
+                        float p[8];
+                        #pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            p[i] = exp2f(__uint_as_float(sr[ch * 8 + i]) - m_use);
+                            sum += p[i];
                         }
-                        #pragma unroll
-                        for (int i = 0; i < HD / 8; ++i)
-                            *reinterpret_cast<uint32_t*>(dst + i * 8 + 2 * q) =
-                                pack_bf16(o[i][2 * rr] * inv, o[i][2 * rr + 1] * inv);
-                        if (lse && q == 0) *lse = (m_run[rr] + log2f(l_run[rr])) * 0.6931471805599453f;
-                    } else {
-                        float* dst = part + static_cast<size_t>(row) * (HD + 2);
-                        if (q == 0) { dst[HD] = m_run[rr]; dst[HD + 1] = l_run[rr]; }
-                        #pragma unroll
-                        for (int i = 0; i < HD / 8; ++i)
-                            *reinterpret_cast<float2*>(dst + i * 8 + 2 * q) = make_float2(o[i][2 * rr], o[i][2 * rr + 1]);
+                        const uint32_t dst = p_row + ((ch ^ (row_in_blk & 7)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pack_bf16(p[0], p[1])),
+                                     "r"(pack_bf16(p[2], p[3])), "r"(pack_bf16(p[4], p[5])), "r"(pack_bf16(p[6], p[7])) : "memory");
+                    }
+                    l_run += sum;
+                }
+                // V rows past the tile's last valid key may hold anything (even NaN patterns): P is 0 there,
+                // but 0 * NaN is NaN, so the first block to use the tile clears them
+                const int nv = sp.valid_keys(j);
+                if (first_of_tile && nv < kTileKeys) {
+                    const int st = j % n_stages;
+                    if (!mbar_wait_warp(smem_u32(&c.kv_full[st]), (j / n_stages) & 1, abort_flag, a.status)) break;
+                    const uint32_t vdst = kv_base + st * G::kStageBytes + G::kHalves * kHalfBytes;
+                    const int n16 = (kTileKeys - nv) * 8 * G::kHalves;      // 16-byte pieces to clear
+                    for (int i = row_in_blk; i < n16; i += kBlockRows) {
+                        const int hh = i / ((kTileKeys - nv) * 8), rem = i - hh * ((kTileKeys - nv) * 8);
+                        const uint32_t dst = vdst + hh * kHalfBytes + (nv + (rem >> 3)) * 128u + ((rem & 7) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
                     }
                 }
+                fence_async_smem();
+                tc_fence_before();
+                mbar_arrive(smem_u32(&c.p_full[my_blk]));
+                ++n_own;
             }
-        }   // row chunks
+            sp.next(j, blk);
+            ++q;
+        }
+        // the block's last PV must have landed in TMEM before the accumulator is read
+        if (n_own > 0) {
+            mbar_wait_warp(smem_u32(&c.o_done[my_blk]), (n_own - 1) & 1, abort_flag, a.status);
+            tc_fence_after();
+        }
+    }
 
-        // ---- split pair: arrive; the last CTA merges every partial of the pair ------------------
-        if (n_splits > 1) {
-            __syncthreads();
-            if (tid == 0) {
-                __threadfence();
-                const int prev = atomicAdd(&a.counters[b * H + h], 1);
-                s_flag = (prev == n_splits - 1);
-                if (s_flag) a.counters[b * H + h] = 0;   // ready for the next call
+    __syncwarp();     // the single-lane roles of warps 0 and 1 rejoin their warps
+
+    // ======================================== epilogue ==========================================
+    const bool has_acc = (warp >= 4) && n_own > 0;     // otherwise the partial is (m = -inf, l = 0, O = 0)
+    if (C == 1) {
+        // the pair was not split: normalise and write this thread's row
+        if (warp >= 4 && __any_sync(0xffffffffu, ri.valid) && !skip) {
+            const float inv = 1.f / l_run;
+            __nv_bfloat16* dst;
+            float* lse;
+            if (!ri.valid) {
+                dst = nullptr; lse = nullptr;
+            } else if (ri.stream == 0) {
+                const long long idx = (static_cast<long long>(b) * a.max_nodes + ri.node) * a.n_heads + h;
+                dst = a.o_main + idx * HD;
+                lse = a.lse_main ? a.lse_main + idx : nullptr;
+            } else {
+                const long long idx = (spec_row0 + static_cast<long long>(ri.node) * a.gamma + (ri.stream - 1)) * a.n_heads + h;
+                dst = a.o_spec + idx * HD;
+                lse = a.lse_spec ? a.lse_spec + idx : nullptr;
             }
-            __syncthreads();
-            if (s_flag) {
-                __threadfence();
-                for (int i = tid; i < M * (HD / 4); i += kThreads) {
-                    const int row = i / (HD / 4), c4 = i - row * (HD / 4);
-                    float mx = -INFINITY;
-                    for (int c = c_first; c <= c_last; ++c) {
-                        const float* ps = a.partials + (static_cast<size_t>(2 * c + (c == c_first ? 1 : 0)) * a.m_pad + row) * (HD + 2);
-                        mx = fmaxf(mx, __ldcg(ps + HD));
-                    }
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                    float l = 0.f;
-                    for (int c = c_first; c <= c_last; ++c) {
-                        const float* ps = a.partials + (static_cast<size_t>(2 * c + (c == c_first ? 1 : 0)) * a.m_pad + row) * (HD + 2);
-                        const float w = exp2f(__ldcg(ps + HD) - mx);
-                        l += w * __ldcg(ps + HD + 1);
-                        const float2 lo = __ldcg(reinterpret_cast<const float2*>(ps + c4 * 4));
-                        const float2 hi = __ldcg(reinterpret_cast<const float2*>(ps + c4 * 4 + 2));
-                        acc.x += w * lo.x; acc.y += w * lo.y; acc.z += w * hi.x; acc.w += w * hi.y;
-                    }
-                    const float inv = 1.f / l;
-                    const int t = row / rows_per_node, j = row - t * rows_per_node;
-                    __nv_bfloat16* dst;
-                    float* lse = nullptr;
-                    if (j == 0) {
-                        const long long idx = (static_cast<long long>(b) * a.max_nodes + t) * H + h;
-                        dst = a.o_main + idx * HD;
-                        if (a.lse_main) lse = a.lse_main + idx;
-                    } else {
-                        const long long idx = (spec_row0 + static_cast<long long>(t) * gamma + (j - 1)) * H + h;
-                        dst = a.o_spec + idx * HD;
-                        if (a.lse_spec) lse = a.lse_spec + idx;
-                    }
-                    uint2 packed;
-                    packed.x = pack_bf16(acc.x * inv, acc.y * inv);
-                    packed.y = pack_bf16(acc.z * inv, acc.w * inv);
-                    *reinterpret_cast<uint2*>(dst + c4 * 4) = packed;
-                    if (lse && c4 == 0) *lse = (mx + log2f(l)) * 0.6931471805599453f;
-                }
+            if (lse) *lse = (m_run + log2f(l_run)) * 0.6931471805599453f;
+            const uint32_t o_addr = tmem + lane_base + my_blk * G::kOCols;
+            #pragma unroll
+            for (int c0 = 0; c0 < HD; c0 += 16) {
+                uint32_t orr[16];
+                if (has_acc) { tmem_ld16<0>(o_addr + c0, orr); tmem_wait_ld(); }     // all 32 lanes of the warp
+                else { for (int i = 0; i < 16; ++i) orr[i] = 0u; }
+                if (dst == nullptr) continue;
+                uint4 lo, hi;
+                lo.x = pack_bf16(__uint_as_float(orr[0]) * inv, __uint_as_float(orr[1]) * inv);
+                lo.y = pack_bf16(__uint_as_float(orr[2]) * inv, __uint_as_float(orr[3]) * inv);
+                lo.z = pack_bf16(__uint_as_float(orr[4]) * inv, __uint_as_float(orr[5]) * inv);
+                lo.w = pack_bf16(__uint_as_float(orr[6]) * inv, __uint_as_float(orr[7]) * inv);
+                hi.x = pack_bf16(__uint_as_float(orr[8]) * inv, __uint_as_float(orr[9]) * inv);
+                hi.y = pack_bf16(__uint_as_float(orr[10]) * inv, __uint_as_float(orr[11]) * inv);
+                hi.z = pack_bf16(__uint_as_float(orr[12]) * inv, __uint_as_float(orr[13]) * inv);
+                hi.w = pack_bf16(__uint_as_float(orr[14]) * inv, __uint_as_float(orr[15]) * inv);
+                *reinterpret_cast<uint4*>(dst + c0) = lo;
+                *reinterpret_cast<uint4*>(dst + c0 + 8) = hi;
             }
         }
-    }   // segments
+    } else {
+        // Every thread of the cluster passes both barriers, whatever happened above.
+        // Barrier A: all CTAs are done with their pipelines, so shared memory can be reused.
+        cluster_arrive();
+        cluster_wait();
+        const int rpc = kBlockRows / C;                 // rows of each block merged by one CTA
+        if (warp >= 4) {
+            const uint32_t dst_rank = row_in_blk / rpc;
+            const int lr = row_in_blk - dst_rank * rpc;
+            // receiver layout: [block][source rank][local row][kMergePitch floats]
+            const uint32_t local = merge_base + (((my_blk * C + rank) * rpc + lr) * G::kMergePitch) * 4u;
+            const uint32_t remote = map_to_rank(local, dst_rank);
+            const uint32_t o_addr = tmem + lane_base + my_blk * G::kOCols;
+            #pragma unroll
+            for (int c0 = 0; c0 < HD; c0 += 16) {
+                uint32_t orr[16];
+                if (has_acc) { tmem_ld16<0>(o_addr + c0, orr); tmem_wait_ld(); }
+                else { for (int i = 0; i < 16; ++i) orr[i] = 0u; }
+                #pragma unroll
+                for (int i = 0; i < 16; i += 4)
+                    st_cluster_v4(remote + (c0 + i) * 4u, __uint_as_float(orr[i]), __uint_as_float(orr[i + 1]),
+                                  __uint_as_float(orr[i + 2]), __uint_as_float(orr[i + 3]));
+            }
+            const uint32_t ml_local = smem_u32(&c.ml[my_blk][rank * rpc + lr]);
+            st_cluster_v2(map_to_rank(ml_local, dst_rank), m_run, l_run);
+        }
+        // Barrier B: every partial has been delivered.
+        cluster_arrive();
+        cluster_wait();
+        if (warp >= 4 && row_in_blk < HD && !skip) {
+            const int col = row_in_blk;
+            for (int lr = 0; lr < rpc; ++lr) {
+                const int row = my_blk * kBlockRows + static_cast<int>(rank) * rpc + lr;
+                const RowInfo r = row_info(sp, row);
+                if (!r.valid) continue;
+                float mx = -INFINITY;
+                for (int s = 0; s < C; ++s) mx = fmaxf(mx, c.ml[my_blk][s * rpc + lr].x);
+                float acc = 0.f, l = 0.f;
+                for (int s = 0; s < C; ++s) {
+                    const float2 ml = c.ml[my_blk][s * rpc + lr];
+                    const float w = exp2f(ml.x - mx);         // 0 for a CTA that saw no visible key
+                    l += w * ml.y;
+                    float v;
+                    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v)
+                                 : "r"(merge_base + (((my_blk * C + s) * rpc + lr) * G::kMergePitch + col) * 4u) : "memory");
+                    acc += w * v;
+                }
+                long long idx;
+                __nv_bfloat16* dst;
+                float* lse;
+                if (r.stream == 0) {
+                    idx = (static_cast<long long>(b) * a.max_nodes + r.node) * a.n_heads + h;
+                    dst = a.o_main + idx * HD;
+                    lse = a.lse_main ? a.lse_main + idx : nullptr;
+                } else {
+                    idx = (spec_row0 + static_cast<long long>(r.node) * a.gamma + (r.stream - 1)) * a.n_heads + h;
+                    dst = a.o_spec + idx * HD;
+                    lse = a.lse_spec ? a.lse_spec + idx : nullptr;
+                }
+                dst[col] = __float2bfloat16_rn(acc / l);
+                if (lse && col == 0) *lse = (mx + log2f(l)) * 0.6931471805599453f;
+            }
+        }
+    }
+
+    // ---- release TMEM ---------------------------------------------------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
+// host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// bf16 tensor (d, n1, n2) with element strides (1, s1, s2); box (64, 1, box_rows); swizzle 128 B
+static bool make_map(CUtensorMap* out, const void* basep, int d, long long n1, long long s1, long long n2, long long s2,
+                     int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return false;
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(n1), static_cast<cuuint64_t>(n2)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(s1) * 2u, static_cast<cuuint64_t>(s2) * 2u};
+    cuuint32_t box[3] = {64u, 1u, static_cast<cuuint32_t>(box_rows)};
+    cuuint32_t estr[3] = {1u, 1u, 1u};
+    return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(basep), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 struct AttnPlan {
-    int grid;
-    int m_pad;
-    size_t counter_bytes, partial_bytes;
+    int tmax8, spec_rows, n_blocks, n_stages, cluster, threads;
+    size_t smem;
 };
 
 static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     if (p.batch < 1 || p.n_heads < 1 || p.max_nodes < 1 || p.gamma < 0) return false;
-    plan->grid = sm_count();
-    plan->m_pad = (p.max_nodes * (1 + p.gamma) + 15) / 16 * 16;
-    plan->counter_bytes = (static_cast<size_t>(p.batch) * p.n_heads * sizeof(int32_t) + 255) / 256 * 256;
-    plan->partial_bytes = static_cast<size_t>(2) * plan->grid * plan->m_pad * (p.head_dim + 2) * sizeof(float);
-    return true;
+    if (p.head_dim != 64 && p.head_dim != 80 && p.head_dim != 128) return false;
+    if (p.max_nodes > SS_MAX_NODES || p.gamma > SS_MAX_GAMMA) return false;
+    const int halves = p.head_dim > 64 ? 2 : 1;
+    plan->tmax8 = (p.max_nodes + 7) / 8 * 8;
+    plan->spec_rows = p.gamma > 0 ? (p.max_nodes * p.gamma + 7) / 8 * 8 : 0;
+    plan->n_blocks = (plan->tmax8 + plan->spec_rows + kBlockRows - 1) / kBlockRows;
+    plan->threads = kAuxThreads + plan->n_blocks * kBlockRows;
+    // cluster size: the largest power of two that still fits the grid on the SMs in one wave
+    const long long pairs = static_cast<long long>(p.batch) * p.n_heads;
+    int c = 1;
+    while (c < 8 && pairs * (c * 2) <= sm_count()) c *= 2;
+    plan->cluster = c;
+    const size_t qp = static_cast<size_t>(plan->n_blocks) * (halves * kBlockRows * 128 + kPBytes);
+    const size_t stage = static_cast<size_t>(2) * halves * kHalfBytes;
+    int ns = static_cast<int>((kMaxDynSmem - 1024 - qp) / stage);
+    ns = ns > kMaxStages ? kMaxStages : ns;
+    if (ns < 2) return false;
+    plan->n_stages = ns;
+    size_t bytes = qp + ns * stage;
+    const size_t merge = static_cast<size_t>(plan->n_blocks) * kBlockRows * (p.head_dim + 4) * 4;
+    if (c > 1 && merge > bytes) bytes = merge;
+    plan->smem = bytes + 1024;
+    return plan->smem <= static_cast<size_t>(kMaxDynSmem);
 }
 
 template <int HD>
-static int32_t launch(const AttnArgs& args, int grid, cudaStream_t stream) {
+static int32_t launch(const AttnArgs& args, const AttnPlan& plan, long long pairs, cudaStream_t stream) {
     static bool configured[64] = {false};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return SS_ERR_CUDA;
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        if (cudaFuncSetAttribute(msa_attention_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 Smem<HD>::kTotal) != cudaSuccess)
+        if (cudaFuncSetAttribute(msa_attention_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem) !=
+            cudaSuccess)
             return SS_ERR_CUDA;
         configured[dev] = true;
     }
-    msa_attention_kernel<HD><<<grid, kThreads, Smem<HD>::kTotal, stream>>>(args);
-    return cudaGetLastError() == cudaSuccess ? SS_OK : SS_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(pairs * plan.cluster), 1, 1);
+    cfg.blockDim = dim3(static_cast<unsigned>(plan.threads), 1, 1);
+    // always more than half of an SM's shared memory: one CTA per SM, so a CTA never queues for TMEM
+    cfg.dynamicSmemBytes = plan.smem < 120 * 1024 ? 120 * 1024 : plan.smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(plan.cluster);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, msa_attention_kernel<HD>, args) == cudaSuccess ? SS_OK : SS_ERR_CUDA;
 }
 
 }  // namespace ss
@@ -517,21 +821,25 @@ static int32_t launch(const AttnArgs& args, int grid, cudaStream_t stream) {
 extern "C" size_t ss_msa_attention_workspace_bytes(const ss_attn_params* p) {
     ss::AttnPlan plan;
     if (p == nullptr || !ss::make_plan(*p, &plan)) return 0;
-    return ss::kWsHeaderBytes + plan.counter_bytes + plan.partial_bytes;
+    return ss::kWsHeaderBytes;     // the status word; split-KV partials never leave the chip
 }
 
 extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
     if (p == nullptr) return SS_ERR_INVALID_ARG;
-    ss::AttnPlan plan;
-    if (!ss::make_plan(*p, &plan)) return SS_ERR_INVALID_ARG;
+    if (p->batch < 1 || p->n_heads < 1 || p->max_nodes < 1 || p->gamma < 0) return SS_ERR_INVALID_ARG;
     if (p->head_dim != 64 && p->head_dim != 80 && p->head_dim != 128) return SS_ERR_UNSUPPORTED;
     if (p->max_nodes > SS_MAX_NODES || p->gamma > SS_MAX_GAMMA) return SS_ERR_UNSUPPORTED;
+    ss::AttnPlan plan;
+    if (!ss::make_plan(*p, &plan)) return SS_ERR_UNSUPPORTED;
     if (!p->q_main || !p->o_main || !p->k_cache || !p->v_cache || !p->kv_start || !p->kv_len || !p->trees ||
         !p->workspace)
         return SS_ERR_INVALID_ARG;
     if (p->gamma > 0 && (!p->q_spec || !p->k_spec || !p->v_spec || !p->o_spec)) return SS_ERR_INVALID_ARG;
     if (p->kv_slot_stride < p->head_dim || p->kv_head_stride < 0 || p->kv_total_slots < 1) return SS_ERR_INVALID_ARG;
     if ((p->kv_slot_stride & 7) || (p->kv_head_stride & 7)) return SS_ERR_INVALID_ARG;
+    if (p->kv_total_slots > 0x7fffffffll) return SS_ERR_UNSUPPORTED;
+    const long long rows_main = static_cast<long long>(p->batch) * p->max_nodes;
+    if (rows_main * (p->gamma > 0 ? p->gamma : 1) > 0x7fffffffll) return SS_ERR_UNSUPPORTED;
     const void* ptrs[] = {p->q_main, p->o_main, p->k_cache, p->v_cache, p->workspace,
                           p->gamma ? p->q_spec : nullptr, p->gamma ? p->k_spec : nullptr,
                           p->gamma ? p->v_spec : nullptr, p->gamma ? p->o_spec : nullptr};
@@ -541,29 +849,38 @@ extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
     if (p->workspace_bytes < ss_msa_attention_workspace_bytes(p)) return SS_ERR_WORKSPACE;
 
     ss::AttnArgs a;
-    a.batch = p->batch; a.n_heads = p->n_heads; a.gamma = p->gamma; a.max_nodes = p->max_nodes;
+    const int d = p->head_dim, H = p->n_heads;
+    const bool shared_heads = (p->kv_head_stride == 0);
+    const long long kv_heads = shared_heads ? 1 : H;
+    const long long kv_hstride = shared_heads ? d : p->kv_head_stride;
+    bool ok = ss::make_map(&a.tm_k, p->k_cache, d, kv_heads, kv_hstride, p->kv_total_slots, p->kv_slot_stride, ss::kTileKeys) &&
+              ss::make_map(&a.tm_v, p->v_cache, d, kv_heads, kv_hstride, p->kv_total_slots, p->kv_slot_stride, ss::kTileKeys) &&
+              ss::make_map(&a.tm_qm, p->q_main, d, H, d, rows_main, static_cast<long long>(H) * d, plan.tmax8);
+    if (ok && p->gamma > 0) {
+        const long long rows_spec = rows_main * p->gamma;
+        ok = ss::make_map(&a.tm_qs, p->q_spec, d, H, d, rows_spec, static_cast<long long>(H) * d, plan.spec_rows) &&
+             ss::make_map(&a.tm_ks, p->k_spec, d, H, d, rows_spec, static_cast<long long>(H) * d, ss::kTileKeys) &&
+             ss::make_map(&a.tm_vs, p->v_spec, d, H, d, rows_spec, static_cast<long long>(H) * d, ss::kTileKeys);
+    } else if (ok) {
+        a.tm_qs = a.tm_qm; a.tm_ks = a.tm_k; a.tm_vs = a.tm_v;     // never used when gamma == 0
+    }
+    if (!ok) return SS_ERR_CUDA;
+    a.batch = p->batch; a.n_heads = H; a.gamma = p->gamma; a.max_nodes = p->max_nodes;
+    a.tmax8 = plan.tmax8; a.spec_rows = plan.spec_rows; a.n_blocks = plan.n_blocks; a.n_stages = plan.n_stages;
+    a.cluster = plan.cluster;
+    a.head_coord = shared_heads ? 0 : 1;
     a.scale_log2 = p->sm_scale * 1.4426950408889634f;
-    a.q_main = static_cast<const __nv_bfloat16*>(p->q_main);
     a.o_main = static_cast<__nv_bfloat16*>(p->o_main);
-    a.q_spec = static_cast<const __nv_bfloat16*>(p->q_spec);
-    a.k_spec = static_cast<const __nv_bfloat16*>(p->k_spec);
-    a.v_spec = static_cast<const __nv_bfloat16*>(p->v_spec);
     a.o_spec = static_cast<__nv_bfloat16*>(p->o_spec);
-    a.k_cache = static_cast<const __nv_bfloat16*>(p->k_cache);
-    a.v_cache = static_cast<const __nv_bfloat16*>(p->v_cache);
-    a.slot_stride = p->kv_slot_stride; a.head_stride = p->kv_head_stride;
+    a.lse_main = p->lse_main; a.lse_spec = p->lse_spec;
     a.kv_start = reinterpret_cast<const long long*>(p->kv_start);
     a.kv_len = p->kv_len; a.kv_capacity = p->kv_capacity; a.trees = p->trees;
-    a.lse_main = p->lse_main; a.lse_spec = p->lse_spec;
-    char* ws = static_cast<char*>(p->workspace);
-    a.status = reinterpret_cast<int*>(ws);
-    a.counters = reinterpret_cast<int*>(ws + ss::kWsHeaderBytes);
-    a.partials = reinterpret_cast<float*>(ws + ss::kWsHeaderBytes + plan.counter_bytes);
-    a.m_pad = plan.m_pad;
+    a.status = reinterpret_cast<int*>(p->workspace);
+    const long long pairs = static_cast<long long>(p->batch) * H;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    switch (p->head_dim) {
-        case 64: return ss::launch<64>(a, plan.grid, s);
-        case 80: return ss::launch<80>(a, plan.grid, s);
-        default: return ss::launch<128>(a, plan.grid, s);
+    switch (d) {
+        case 64: return ss::launch<64>(a, plan, pairs, s);
+        case 80: return ss::launch<80>(a, plan, pairs, s);
+        default: return ss::launch<128>(a, plan, pairs, s);
     }
 }
