@@ -8,21 +8,24 @@
 // Inside a CTA.  ALL query rows of the head -- T main rows, then the T*gamma stream rows -- sit in
 // shared memory as up to three 128-row blocks, so each K/V tile that TMA brings in is used by every
 // (node x stream) row: the prefix crosses HBM once per head, not once per stream.
-//   warp 0      TMA producer: Q once, then 64-key K/V tiles into a ring of stages (mbarrier
-//               complete_tx); swizzle-128B boxes straight from the caller's strided tensors.
-//   warp 1      tcgen05 issuer: S = Q K^T (128 x 64 x d) into one of two TMEM buffers, later
-//               O += P V (128 x d x 64) into the block's TMEM accumulator; tcgen05.commit arrives
-//               on the mbarriers that hand buffers back.
+//   thread 0    TMA producer: Q once, then K tiles and V tiles into two independent rings
+//               (mbarrier complete_tx); swizzle-128B boxes straight from the caller's strided tensors.
+//               A K slot is handed back as soon as S has been computed, a V slot after P V.
+//   warp 1      tcgen05 issuer: S = Q K^T (128 x TK x d) into one of two TMEM buffers, later
+//               O += P V (128 x d x TK) into the block's TMEM accumulator; tcgen05.commit arrives
+//               on the mbarriers that hand buffers back.  TK = 128 keys when the head has one row
+//               block (N = 128 MMAs run at the full tensor rate), 64 keys otherwise.
 //   warps 4..   one warpgroup per 128-row block, one thread per query row: tcgen05.ld of the S row,
 //               tree / stream mask from the node's 64-bit ancestor word, online softmax in fp32
 //               registers (the running maximum is only raised when it would grow by more than 2^8,
 //               which keeps the TMEM accumulator untouched on almost every tile), P as bf16 into a
 //               swizzled shared-memory tile that feeds the second MMA.
-// Split-KV merge.  Each CTA ends with un-normalised (m, l, O) per row.  CTA r of the cluster merges
-// rows [128/C * r, 128/C * (r+1)) of every block: all CTAs push those rows into r's shared memory
-// (st.shared::cluster), one cluster barrier, then r combines the C partials and writes bf16 output.
-// No CTA ever spins on another: the only cross-CTA waits are hardware cluster barriers that every
-// thread reaches unconditionally; every mbarrier wait is bounded and reports SS_ERR_DEVICE_TIMEOUT.
+// Split-KV merge.  Each CTA ends with un-normalised (m, l, O) per row.  The valid rows of every
+// block are dealt out to the C CTAs of the cluster: all CTAs push a row's partial into the shared
+// memory of the CTA that merges it (st.shared::cluster), one cluster barrier, then that CTA combines
+// the C partials and writes bf16 output.  No CTA ever spins on another: the only cross-CTA waits are
+// hardware cluster barriers that every thread reaches unconditionally; every mbarrier wait is
+// bounded and reports SS_ERR_DEVICE_TIMEOUT.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -30,27 +33,25 @@
 
 namespace ss {
 
-constexpr int kTileKeys = 64;        // keys per staged tile (N of the S MMA, K of the PV MMA)
 constexpr int kUnit = 16;            // split granularity (keys)
 constexpr int kBlockRows = 128;      // query rows per block (M of both MMAs)
 constexpr int kMaxBlocks = 3;        // 64 main rows + 256 stream rows = 320 rows at most
-constexpr int kMaxStages = 6;
+constexpr int kMaxSlots = 4;         // slots per ring (K ring, V ring)
 constexpr int kAuxThreads = 128;     // warps 0..3: producer, MMA issuer, two spare
-constexpr int kHalfBytes = 64 * 128; // one TMA box: 64 rows x 128 B (64 bf16 of head_dim)
-constexpr int kPBytes = kBlockRows * 128;   // one P tile: 128 rows x 64 keys bf16
 constexpr int kMaxDynSmem = 232448 - 4096;  // 227 KB per CTA less the static control block
 constexpr float kRescaleStep = 8.f;  // raise the running maximum only when it grows by more than 2^8
 constexpr long long kWaitCycles = 2000000000ll;   // bound of every mbarrier wait (~1 s)
 
 struct alignas(64) AttnArgs {
-    CUtensorMap tm_k, tm_v;          // cache slab    dims (d, H, slots)        box (64, 1, 64)
+    CUtensorMap tm_k, tm_v;          // cache slab    dims (d, H, slots)        box (64, 1, TK)
     CUtensorMap tm_qm;               // q_main        dims (d, H, B*Tmax)       box (64, 1, tmax8)
     CUtensorMap tm_qs;               // q_spec        dims (d, H, B*Tmax*g)     box (64, 1, spec_rows)
-    CUtensorMap tm_ks, tm_vs;        // k_spec/v_spec dims (d, H, B*Tmax*g)     box (64, 1, 64)
+    CUtensorMap tm_ks, tm_vs;        // k_spec/v_spec dims (d, H, B*Tmax*g)     box (64, 1, TK)
     int batch, n_heads, gamma, max_nodes;
     int tmax8;                       // max_nodes rounded up to 8: first stream row in shared memory
     int spec_rows;                   // max_nodes * gamma rounded up to 8 (rows of the q_spec box)
-    int n_blocks, n_stages, cluster;
+    int n_blocks, cluster;
+    int n_kslots, n_vslots;          // ring depths
     int head_coord;                  // 1, or 0 when all heads share one K/V (head stride 0)
     float scale_log2;                // sm_scale * log2(e)
     __nv_bfloat16* o_main;
@@ -66,11 +67,12 @@ struct alignas(64) AttnArgs {
 
 struct Ctrl {
     unsigned long long q_full;
-    unsigned long long kv_full[kMaxStages], kv_empty[kMaxStages];
-    unsigned long long s_full[kMaxBlocks][2], s_free[2];   // s_full per (block, buffer): a warpgroup sees every phase of its own
+    unsigned long long k_full[kMaxSlots], k_empty[kMaxSlots], v_full[kMaxSlots], v_empty[kMaxSlots];
+    unsigned long long s_full[kMaxBlocks][2];   // per (block, S buffer): a warpgroup sees every phase of its own
+    unsigned long long s_free[2];
     unsigned long long p_full[kMaxBlocks], o_done[kMaxBlocks];
     unsigned long long anc[SS_MAX_NODES];
-    float2 ml[kMaxBlocks][kBlockRows];   // (m, l) received for the rows this CTA merges: [block][src * rpc + lr]
+    float2 ml[kMaxBlocks][kBlockRows];   // (m, l) received for the rows this CTA merges: [block][src * rpc_max + lr]
     uint32_t tmem_base;
     int abort;
 };
@@ -92,11 +94,16 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
     return r;
 }
-__device__ __forceinline__ void st_cluster_v4(uint32_t addr, float x, float y, float z, float w) {
-    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(x), "f"(y), "f"(z), "f"(w) : "memory");
+__device__ __forceinline__ void st_cluster_v4(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
+    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
 }
 __device__ __forceinline__ void st_cluster_v2(uint32_t addr, float x, float y) {
     asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(x), "f"(y) : "memory");
+}
+__device__ __forceinline__ float4 ld_shared_v4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
 }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -174,7 +181,7 @@ __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.
 #define SS_W16(r, o) "r"(r[o + 0]), "r"(r[o + 1]), "r"(r[o + 2]), "r"(r[o + 3]), "r"(r[o + 4]), "r"(r[o + 5]), \
                      "r"(r[o + 6]), "r"(r[o + 7]), "r"(r[o + 8]), "r"(r[o + 9]), "r"(r[o + 10]), "r"(r[o + 11]), \
                      "r"(r[o + 12]), "r"(r[o + 13]), "r"(r[o + 14]), "r"(r[o + 15])
-// 16 consecutive fp32 columns of this thread's TMEM lane <-> registers r[o .. o+15]
+// N consecutive fp32 columns of this thread's TMEM lane <-> registers r[O .. O+N-1]
 template <int O, int N>
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[N]) {
     asm volatile(
@@ -182,10 +189,22 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[N]) {
         : SS_R16(r, O) : "r"(taddr) : "memory");
 }
 template <int O, int N>
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[N]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : SS_R16(r, O), SS_R16(r, O + 16) : "r"(taddr) : "memory");
+}
+template <int O, int N>
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[N]) {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
         ::SS_W16(r, O), "r"(taddr) : "memory");
+}
+// 64 columns starting at taddr
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t (&r)[64]) {
+    tmem_ld32<0>(taddr, r);
+    tmem_ld32<32>(taddr + 32, r);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -212,51 +231,86 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int n, bool b_mn_major) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// The CTA's share of the pair's keys, as a list of tiles.  Every role derives it from the same
-// four numbers, so no tile list is ever stored.
+// The CTA's share of the pair's keys, as a list of tiles of TK keys.  Every role derives it from
+// the same few numbers, so no tile list is ever stored.
+template <int TK>
 struct Span {
     int L, T, n_stream;            // prefix length, tree nodes, stream keys (T * gamma)
     int kc0, kc1;                  // cache keys [kc0, kc1) (indices into [0, L+T))
     int ks0, ks1;                  // stream keys [ks0, ks1) (indices into [0, T*gamma))
     int n_cache_tiles, n_tiles;
     int tmax8, gamma, n_blocks;
-    int main_rows, spec_end;       // valid rows: [0, main_rows) and [tmax8, spec_end)
+    int spec_end;                  // valid rows: [0, T) and [tmax8, spec_end)
+    unsigned valid_blocks;         // bit b set: row block b holds a valid row
 
     __device__ __forceinline__ bool is_cache(int j) const { return j < n_cache_tiles; }
     __device__ __forceinline__ int first_key(int j) const {
-        return j < n_cache_tiles ? kc0 + j * kTileKeys : ks0 + (j - n_cache_tiles) * kTileKeys;
+        return j < n_cache_tiles ? kc0 + j * TK : ks0 + (j - n_cache_tiles) * TK;
     }
     __device__ __forceinline__ int valid_keys(int j) const {
-        return min(kTileKeys, (j < n_cache_tiles ? kc1 : ks1) - first_key(j));
+        return min(TK, (j < n_cache_tiles ? kc1 : ks1) - first_key(j));
     }
-    // does row block `blk` hold a row that can see a key of tile j?
-    __device__ __forceinline__ bool active(int j, int blk) const {
-        const int r0 = blk * kBlockRows, r1 = r0 + kBlockRows;
-        if (j < n_cache_tiles) return r0 < main_rows || (r0 < spec_end && r1 > tmax8);
+    // bit b set: row block b holds a row that can see a key of tile j
+    __device__ __forceinline__ unsigned active_mask(int j) const {
+        if (j < n_cache_tiles) return valid_blocks;
         // stream key s is seen by the stream rows s .. (end of its node's group)
         const int s0 = first_key(j), s_last = s0 + valid_keys(j) - 1;
         const int row_lo = tmax8 + s0, row_hi = tmax8 + (s_last / gamma) * gamma + gamma - 1;
-        return row_lo < r1 && row_hi >= r0;
+        unsigned m = 0;
+        for (int b = 0; b < n_blocks; ++b)
+            if (row_lo < (b + 1) * kBlockRows && row_hi >= b * kBlockRows) m |= 1u << b;
+        return m;
     }
-    // next active (tile, block) after (j, blk) in tile-major order; j == n_tiles when exhausted
-    __device__ __forceinline__ void next(int& j, int& blk) const {
-        for (;;) {
-            if (++blk >= n_blocks) { blk = 0; ++j; }
-            if (j >= n_tiles || active(j, blk)) return;
-        }
+    // valid rows of a block, numbered 0 .. n_valid-1 (main rows first, then stream rows)
+    __device__ __forceinline__ int main_in_block(int blk) const { return blk == 0 ? T : 0; }
+    __device__ __forceinline__ int n_valid(int blk) const {
+        const int r0 = blk * kBlockRows, r1 = r0 + kBlockRows;
+        return main_in_block(blk) + max(0, min(spec_end, r1) - max(tmax8, r0));
     }
-    __device__ __forceinline__ void first(int& j, int& blk) const {
-        j = 0; blk = -1;
-        if (n_tiles == 0) { blk = 0; return; }
-        next(j, blk);
+    __device__ __forceinline__ int valid_index(int row) const {      // -1 for a padding row
+        const int blk = row / kBlockRows, r0 = blk * kBlockRows;
+        if (row < tmax8) return row < T ? row - r0 : -1;
+        return row < spec_end ? main_in_block(blk) + row - max(tmax8, r0) : -1;
+    }
+    __device__ __forceinline__ int row_of(int blk, int vi) const {
+        const int r0 = blk * kBlockRows, mb = main_in_block(blk);
+        return vi < mb ? r0 + vi : max(tmax8, r0) + (vi - mb);
     }
 };
 
-__device__ __forceinline__ Span make_span(const AttnArgs& a, int L, int T, int rank) {
-    Span s;
+// (tile, block) items in tile-major order, only the active ones
+struct ItemIter {
+    int j;
+    unsigned m;
+    template <class S>
+    __device__ __forceinline__ void begin(const S& sp) {
+        j = 0;
+        m = sp.n_tiles > 0 ? sp.active_mask(0) : 0u;
+        skip_empty(sp);
+    }
+    template <class S>
+    __device__ __forceinline__ void skip_empty(const S& sp) {
+        while (m == 0u && j < sp.n_tiles) {
+            ++j;
+            m = j < sp.n_tiles ? sp.active_mask(j) : 0u;
+        }
+    }
+    template <class S>
+    __device__ __forceinline__ bool done(const S& sp) const { return j >= sp.n_tiles; }
+    __device__ __forceinline__ int blk() const { return __ffs(m) - 1; }
+    __device__ __forceinline__ bool last_of_tile() const { return (m & (m - 1u)) == 0u; }
+    template <class S>
+    __device__ __forceinline__ void next(const S& sp) {
+        m &= m - 1u;
+        skip_empty(sp);
+    }
+};
+
+template <int TK>
+__device__ __forceinline__ Span<TK> make_span(const AttnArgs& a, int L, int T, int rank) {
+    Span<TK> s;
     s.L = L; s.T = T; s.gamma = a.gamma; s.tmax8 = a.tmax8; s.n_blocks = a.n_blocks;
     s.n_stream = T * a.gamma;
-    s.main_rows = T;
     s.spec_end = a.tmax8 + s.n_stream;
     const int ec = L + T;
     const int uc = (ec + kUnit - 1) / kUnit, us = (s.n_stream + kUnit - 1) / kUnit;
@@ -267,9 +321,12 @@ __device__ __forceinline__ Span make_span(const AttnArgs& a, int L, int T, int r
     s.kc1 = min(min(u1, uc) * kUnit, ec);
     s.ks0 = (max(u0, uc) - uc) * kUnit;
     s.ks1 = min((max(u1, uc) - uc) * kUnit, s.n_stream);
-    s.n_cache_tiles = s.kc1 > s.kc0 ? (s.kc1 - s.kc0 + kTileKeys - 1) / kTileKeys : 0;
-    const int nst = s.ks1 > s.ks0 ? (s.ks1 - s.ks0 + kTileKeys - 1) / kTileKeys : 0;
+    s.n_cache_tiles = s.kc1 > s.kc0 ? (s.kc1 - s.kc0 + TK - 1) / TK : 0;
+    const int nst = s.ks1 > s.ks0 ? (s.ks1 - s.ks0 + TK - 1) / TK : 0;
     s.n_tiles = s.n_cache_tiles + nst;
+    s.valid_blocks = 0;
+    for (int b = 0; b < a.n_blocks; ++b)
+        if (s.n_valid(b) > 0) s.valid_blocks |= 1u << b;
     return s;
 }
 
@@ -279,10 +336,11 @@ struct RowInfo {
     bool valid;
     int node, stream;              // stream 0 = main row, 1..gamma = speculative stream
 };
-__device__ __forceinline__ RowInfo row_info(const Span& s, int row) {
+template <int TK>
+__device__ __forceinline__ RowInfo row_info(const Span<TK>& s, int row) {
     RowInfo r;
     if (row < s.tmax8) {
-        r.valid = row < s.main_rows; r.node = row; r.stream = 0;
+        r.valid = row < s.T; r.node = row; r.stream = 0;
     } else {
         const int x = row - s.tmax8;
         r.valid = x < s.n_stream;
@@ -292,23 +350,24 @@ __device__ __forceinline__ RowInfo row_info(const Span& s, int row) {
     return r;
 }
 
-// Bit i set <=> key i of tile j is visible to the row (Eq. 1 / Eq. 2 with the tree mask of App. A).
-__device__ __forceinline__ unsigned long long visible_mask(const Span& s, int j, const RowInfo& r, unsigned long long anc) {
-    if (!r.valid) return 0ull;
-    const int x = s.first_key(j), nv = s.valid_keys(j);
+// Bit i set <=> key x+i (i < 64) is visible to the row (Eq. 1 / Eq. 2 with the tree mask of App. A).
+// `cache`: x indexes the cached slots [0, L+T), else the stream keys; nv = valid keys from x on.
+__device__ __forceinline__ unsigned long long visible_mask(bool cache, int x, int nv, int L, int gamma, const RowInfo& r,
+                                                            unsigned long long anc) {
+    if (!r.valid || nv <= 0) return 0ull;
     const unsigned long long in_tile = nv >= 64 ? ~0ull : ((1ull << nv) - 1ull);
     unsigned long long m;
-    if (s.is_cache(j)) {
-        if (x >= s.L) {                        // tree keys only: key x+i is node (x - L + i)
-            const int sh = x - s.L;
+    if (cache) {
+        if (x >= L) {                          // tree keys only: key x+i is node (x - L + i)
+            const int sh = x - L;
             m = sh >= 64 ? 0ull : (anc >> sh);
         } else {                               // prefix keys (all visible), then tree keys
-            const int np = s.L - x;
+            const int np = L - x;
             m = np >= 64 ? ~0ull : (((1ull << np) - 1ull) | (anc << np));
         }
     } else {                                   // stream keys: (node, 1..stream) of the row's own node
         if (r.stream == 0) return 0ull;
-        const int lo = r.node * s.gamma - x, hi = lo + r.stream;      // visible tile positions [lo, hi)
+        const int lo = r.node * gamma - x, hi = lo + r.stream;        // visible positions [lo, hi)
         const unsigned long long below_hi = hi >= 64 ? ~0ull : (hi <= 0 ? 0ull : ((1ull << hi) - 1ull));
         const unsigned long long below_lo = lo >= 64 ? ~0ull : (lo <= 0 ? 0ull : ((1ull << lo) - 1ull));
         m = below_hi & ~below_lo;
@@ -316,22 +375,81 @@ __device__ __forceinline__ unsigned long long visible_mask(const Span& s, int j,
     return m & in_tile;
 }
 
-template <int HD>
+// max over 64 scores of (visible ? s * scale : -inf), four independent chains
+template <bool MASKED>
+__device__ __forceinline__ float chunk_max(const uint32_t (&v)[64], float scale, unsigned long long vis) {
+    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+    const uint32_t vlo = static_cast<uint32_t>(vis), vhi = static_cast<uint32_t>(vis >> 32);
+    #pragma unroll
+    for (int i = 0; i < 64; ++i) {
+        float s = __uint_as_float(v[i]) * scale;
+        if (MASKED) s = (((i < 32 ? vlo : vhi) >> (i & 31)) & 1u) ? s : -INFINITY;
+        mx[i & 3] = fmaxf(mx[i & 3], s);
+    }
+    return fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+}
+// p = exp2(s * scale - m) for 64 scores -> bf16 into the row's eight 16-byte chunks; returns sum of p
+template <bool MASKED>
+__device__ __forceinline__ float chunk_exp_store(const uint32_t (&v)[64], float scale, float m_use, unsigned long long vis,
+                                                 uint32_t p_row, int row_in_blk) {
+    float sum[4] = {0.f, 0.f, 0.f, 0.f};
+    const uint32_t vlo = static_cast<uint32_t>(vis), vhi = static_cast<uint32_t>(vis >> 32);
+    const float neg_m = -m_use;
+    #pragma unroll
+    for (int ch = 0; ch < 8; ++ch) {
+        float p[8];
+        #pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int k = ch * 8 + i;
+            float e = exp2f(fmaf(__uint_as_float(v[k]), scale, neg_m));
+            if (MASKED) e = (((k < 32 ? vlo : vhi) >> (k & 31)) & 1u) ? e : 0.f;
+            p[i] = e;
+            sum[i & 3] += e;
+        }
+        const uint32_t dst = p_row + ((ch ^ (row_in_blk & 7)) << 4);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pack_bf16(p[0], p[1])),
+                     "r"(pack_bf16(p[2], p[3])), "r"(pack_bf16(p[4], p[5])), "r"(pack_bf16(p[6], p[7])) : "memory");
+    }
+    return (sum[0] + sum[1]) + (sum[2] + sum[3]);
+}
+
+template <int HD, int TK>
 struct Geo {
     static constexpr int kHalves = HD > 64 ? 2 : 1;               // 64-element boxes along head_dim
-    static constexpr int kStageBytes = 2 * kHalves * kHalfBytes;  // K + V
+    static constexpr int kBoxBytes = TK * 128;                    // one TMA box: TK rows x 128 B
+    static constexpr int kSlotBytes = kHalves * kBoxBytes;        // one K tile (or one V tile)
     static constexpr int kKSteps = HD / 16;                       // MMA K steps of S = Q K^T
     static constexpr int kMergePitch = HD + 4;                    // floats per row in the merge buffer
-    static constexpr uint32_t kIdescS = idesc_bf16(kTileKeys, false);
+    static constexpr uint32_t kIdescS = idesc_bf16(TK, false);
     static constexpr uint32_t kIdescPV = idesc_bf16(HD, true);
     static constexpr int kOCols = 128;                            // TMEM columns reserved per block accumulator
+    static constexpr int kThreads = kAuxThreads + (TK == 128 ? 1 : kMaxBlocks) * kBlockRows;
 };
 
-// ---------------------------------------------------------------------------------------------
+// destination of a row's output and log-sum-exp
+struct OutPtr {
+    __nv_bfloat16* o;
+    float* lse;
+};
 template <int HD>
-__global__ void __launch_bounds__(kAuxThreads + kMaxBlocks * kBlockRows, 1)
-msa_attention_kernel(const __grid_constant__ AttnArgs a) {
-    using G = Geo<HD>;
+__device__ __forceinline__ OutPtr out_ptr(const AttnArgs& a, int b, int h, long long spec_row0, const RowInfo& r) {
+    OutPtr p;
+    if (r.stream == 0) {
+        const long long idx = (static_cast<long long>(b) * a.max_nodes + r.node) * a.n_heads + h;
+        p.o = a.o_main + idx * HD;
+        p.lse = a.lse_main ? a.lse_main + idx : nullptr;
+    } else {
+        const long long idx = (spec_row0 + static_cast<long long>(r.node) * a.gamma + (r.stream - 1)) * a.n_heads + h;
+        p.o = a.o_spec + idx * HD;
+        p.lse = a.lse_spec ? a.lse_spec + idx : nullptr;
+    }
+    return p;
+}
+
+// ---------------------------------------------------------------------------------------------
+template <int HD, int TK>
+__global__ void __launch_bounds__(Geo<HD, TK>::kThreads, 1) msa_attention_kernel(const __grid_constant__ AttnArgs a) {
+    using G = Geo<HD, TK>;
     extern __shared__ unsigned char smem_raw[];
     __shared__ Ctrl c;
 
@@ -340,21 +458,35 @@ msa_attention_kernel(const __grid_constant__ AttnArgs a) {
     const uint32_t rank = C > 1 ? cluster_rank() : 0u;
     const int pair = blockIdx.x / C;
     const int b = pair / a.n_heads, h = pair - b * a.n_heads;
-    const int n_blocks = a.n_blocks, n_stages = a.n_stages;
+    const int n_blocks = a.n_blocks, nk = a.n_kslots, nv_slots = a.n_vslots;
     volatile int* abort_flag = &c.abort;
 
+    // per-sequence scalars (every thread reads them; the loads overlap the set-up below)
+    int L = a.kv_len[b];
+    int T = min(max(a.trees[b].n_nodes, 0), a.max_nodes);
+    const long long slot0 = a.kv_start[b];
+    const int cap = a.kv_capacity != nullptr ? a.kv_capacity[b] : 0x7fffffff;
+
     // ---- shared-memory carve-up (1024-byte aligned: swizzle atoms) ----------------------------
+    // Q and P keep only the rows that exist; an MMA that reads the rows of a 128-row block past them
+    // picks up whatever follows in shared memory, which only ever reaches padding rows of S and O.
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t q_rows = n_blocks * kBlockRows;
+    const uint32_t q_rows = a.tmax8 + a.spec_rows;                      // rows TMA brings in
+    const uint32_t p_rows = n_blocks == 1 ? q_rows : kBlockRows;
+    const uint32_t p_bytes = (TK / 64) * p_rows * 128u;                 // one block's P tile
     const uint32_t q_base = base;                                       // [half][q_rows][128 B]
-    const uint32_t p_base = q_base + G::kHalves * q_rows * 128u;        // [block][128 rows][128 B]
-    const uint32_t kv_base = p_base + n_blocks * kPBytes;               // [stage][K halves | V halves]
+    const uint32_t p_base = q_base + G::kHalves * q_rows * 128u;        // [block][key half][p_rows][128 B]
+    const uint32_t k_base = p_base + n_blocks * p_bytes;                // [slot][half][TK][128 B]
+    const uint32_t v_base = k_base + nk * G::kSlotBytes;                // [slot][half][TK][128 B]
     const uint32_t merge_base = base;                                   // aliases everything above, after the main loop
 
     // ---- prologue ---------------------------------------------------------------------------------
     if (tid == 0) {
         mbar_init(smem_u32(&c.q_full), 1);
-        for (int s = 0; s < kMaxStages; ++s) { mbar_init(smem_u32(&c.kv_full[s]), 1); mbar_init(smem_u32(&c.kv_empty[s]), 1); }
+        for (int s = 0; s < kMaxSlots; ++s) {
+            mbar_init(smem_u32(&c.k_full[s]), 1); mbar_init(smem_u32(&c.k_empty[s]), 1);
+            mbar_init(smem_u32(&c.v_full[s]), 1); mbar_init(smem_u32(&c.v_empty[s]), 1);
+        }
         for (int s = 0; s < 2; ++s) {
             mbar_init(smem_u32(&c.s_free[s]), 4);
             for (int k = 0; k < kMaxBlocks; ++k) mbar_init(smem_u32(&c.s_full[k][s]), 1);
@@ -365,67 +497,87 @@ msa_attention_kernel(const __grid_constant__ AttnArgs a) {
         tma_prefetch_desc(&a.tm_k); tma_prefetch_desc(&a.tm_v); tma_prefetch_desc(&a.tm_qm);
         if (a.gamma > 0) { tma_prefetch_desc(&a.tm_qs); tma_prefetch_desc(&a.tm_ks); tma_prefetch_desc(&a.tm_vs); }
     }
-    const uint32_t tmem_cols = n_blocks == 1 ? 256u : 512u;
+    constexpr uint32_t kTmemCols = 512;
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&c.tmem_base)), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&c.tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    int L = a.kv_len[b];
-    int T = min(max(a.trees[b].n_nodes, 0), a.max_nodes);
-    const long long slot0 = a.kv_start[b];
     bool skip = false;                                    // sequence over its slot capacity: nothing read or written
-    if (L < 0 || (a.kv_capacity != nullptr && L + T > a.kv_capacity[b])) {
+    if (L < 0 || L + T > cap) {
         skip = true;
         if (tid == 0) set_status(a.status, SS_ERR_CAPACITY);
+        L = 0; T = 0;
     }
-    if (skip) { L = 0; T = 0; }
     if (tid >= kAuxThreads && tid < kAuxThreads + SS_MAX_NODES) c.anc[tid - kAuxThreads] = a.trees[b].anc_mask[tid - kAuxThreads];
+
+    const Span<TK> sp = make_span<TK>(a, L, T, static_cast<int>(rank));
+    const long long spec_row0 = static_cast<long long>(b) * a.max_nodes * a.gamma;   // first stream row of the sequence
+
+    // K tile j / V tile j of the span -> ring slot (thread 0 only)
+    auto load_k = [&](int j) {
+        const int st = j % nk;
+        const uint32_t bar = smem_u32(&c.k_full[st]);
+        mbar_expect_tx(bar, G::kSlotBytes);
+        const uint32_t dst = k_base + st * G::kSlotBytes;
+        const int x = sp.first_key(j);
+        #pragma unroll
+        for (int hh = 0; hh < G::kHalves; ++hh) {
+            if (sp.is_cache(j)) tma_load_3d(dst + hh * G::kBoxBytes, &a.tm_k, hh * 64, h * a.head_coord, static_cast<int>(slot0 + x), bar);
+            else tma_load_3d(dst + hh * G::kBoxBytes, &a.tm_ks, hh * 64, h, static_cast<int>(spec_row0 + x), bar);
+        }
+    };
+    auto load_v = [&](int j) {
+        const int st = j % nv_slots;
+        const uint32_t bar = smem_u32(&c.v_full[st]);
+        mbar_expect_tx(bar, G::kSlotBytes);
+        const uint32_t dst = v_base + st * G::kSlotBytes;
+        const int x = sp.first_key(j);
+        #pragma unroll
+        for (int hh = 0; hh < G::kHalves; ++hh) {
+            if (sp.is_cache(j)) tma_load_3d(dst + hh * G::kBoxBytes, &a.tm_v, hh * 64, h * a.head_coord, static_cast<int>(slot0 + x), bar);
+            else tma_load_3d(dst + hh * G::kBoxBytes, &a.tm_vs, hh * 64, h, static_cast<int>(spec_row0 + x), bar);
+        }
+    };
+    // the producer starts before the CTA-wide synchronisation: Q and the first tiles need no hand-back
+    const int n_early = min(sp.n_tiles, min(nk, nv_slots));
+    if (tid == 0 && sp.n_tiles > 0) {
+        const uint32_t qbytes = G::kHalves * q_rows * 128u;
+        mbar_expect_tx(smem_u32(&c.q_full), qbytes);
+        #pragma unroll
+        for (int hh = 0; hh < G::kHalves; ++hh) {
+            tma_load_3d(q_base + hh * q_rows * 128u, &a.tm_qm, hh * 64, h, b * a.max_nodes, smem_u32(&c.q_full));
+            if (a.gamma > 0)
+                tma_load_3d(q_base + hh * q_rows * 128u + a.tmax8 * 128u, &a.tm_qs, hh * 64, h,
+                            static_cast<int>(spec_row0), smem_u32(&c.q_full));
+        }
+        for (int j = 0; j < n_early; ++j) { load_k(j); load_v(j); }
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = c.tmem_base;
-    const uint32_t tmem_s = tmem + n_blocks * G::kOCols;  // two S buffers of 64 columns
-
-    const Span sp = make_span(a, L, T, static_cast<int>(rank));
-    const long long spec_row0 = static_cast<long long>(b) * a.max_nodes * a.gamma;   // first stream row of the sequence
+    const uint32_t tmem_s = tmem + n_blocks * G::kOCols;  // two S buffers of TK columns
 
     // ================================= warp 0: TMA producer =====================================
     if (warp == 0) {
-        if (lane == 0 && sp.n_tiles > 0) {
-            const uint32_t qbytes = G::kHalves * (a.tmax8 + (a.gamma > 0 ? a.spec_rows : 0)) * 128u;
-            mbar_expect_tx(smem_u32(&c.q_full), qbytes);
-            for (int hh = 0; hh < G::kHalves; ++hh) {
-                tma_load_3d(q_base + hh * q_rows * 128u, &a.tm_qm, hh * 64, h, b * a.max_nodes, smem_u32(&c.q_full));
-                if (a.gamma > 0)
-                    tma_load_3d(q_base + hh * q_rows * 128u + a.tmax8 * 128u, &a.tm_qs, hh * 64, h,
-                                static_cast<int>(spec_row0), smem_u32(&c.q_full));
-            }
-            int issued = 0;
-            for (int j = 0; j < sp.n_tiles; ++j) {
-                const int st = j % n_stages;
-                if (j >= n_stages && !mbar_wait(smem_u32(&c.kv_empty[st]), ((j / n_stages) - 1) & 1, abort_flag, a.status)) break;
-                const uint32_t bar = smem_u32(&c.kv_full[st]);
-                mbar_expect_tx(bar, G::kStageBytes);
-                const uint32_t kdst = kv_base + st * G::kStageBytes, vdst = kdst + G::kHalves * kHalfBytes;
-                const int x = sp.first_key(j);
-                for (int hh = 0; hh < G::kHalves; ++hh) {
-                    if (sp.is_cache(j)) {
-                        const int slot = static_cast<int>(slot0 + x);
-                        tma_load_3d(kdst + hh * kHalfBytes, &a.tm_k, hh * 64, h * a.head_coord, slot, bar);
-                        tma_load_3d(vdst + hh * kHalfBytes, &a.tm_v, hh * 64, h * a.head_coord, slot, bar);
-                    } else {
-                        const int row = static_cast<int>(spec_row0 + x);
-                        tma_load_3d(kdst + hh * kHalfBytes, &a.tm_ks, hh * 64, h, row, bar);
-                        tma_load_3d(vdst + hh * kHalfBytes, &a.tm_vs, hh * 64, h, row, bar);
-                    }
+        if (lane == 0 && sp.n_tiles > n_early) {
+            int jk = n_early, jv = n_early;               // next K tile / V tile to request
+            bool ok = true;
+            while (ok && (jk < sp.n_tiles || jv < sp.n_tiles)) {
+                // K slots come back early (after S), so K runs ahead of V by at most one ring
+                if (jk < sp.n_tiles && (jk <= jv || jv >= sp.n_tiles)) {
+                    ok = jk < nk || mbar_wait(smem_u32(&c.k_empty[jk % nk]), ((jk / nk) - 1) & 1, abort_flag, a.status);
+                    if (ok) load_k(jk++);
+                } else {
+                    ok = jv < nv_slots || mbar_wait(smem_u32(&c.v_empty[jv % nv_slots]), ((jv / nv_slots) - 1) & 1, abort_flag, a.status);
+                    if (ok) load_v(jv++);
                 }
-                issued = j + 1;
             }
-            if (*abort_flag) {
+            if (!ok) {
                 // gave up: let the copies already in flight land before shared memory is reused or released
                 mbar_drain(smem_u32(&c.q_full), 0);
-                for (int j = max(0, issued - n_stages); j < issued; ++j)
-                    mbar_drain(smem_u32(&c.kv_full[j % n_stages]), (j / n_stages) & 1);
+                for (int j = max(0, jk - nk); j < jk; ++j) mbar_drain(smem_u32(&c.k_full[j % nk]), (j / nk) & 1);
+                for (int j = max(0, jv - nv_slots); j < jv; ++j) mbar_drain(smem_u32(&c.v_full[j % nv_slots]), (j / nv_slots) & 1);
             }
         }
     }
@@ -433,49 +585,58 @@ msa_attention_kernel(const __grid_constant__ AttnArgs a) {
     else if (warp == 1) {
         if (lane == 0 && sp.n_tiles > 0) {
             bool ok = mbar_wait(smem_u32(&c.q_full), 0, abort_flag, a.status);
-            int n_done[kMaxBlocks] = {0, 0, 0};        // PV MMAs issued per block
-            int waited_tile = -1;                      // last tile whose kv_full was observed
-            auto issue_s = [&](int j, int blk, int q) -> bool {
-                const int st = j % n_stages;
-                if (waited_tile != j) {
-                    if (!mbar_wait(smem_u32(&c.kv_full[st]), (j / n_stages) & 1, abort_flag, a.status)) return false;
-                    waited_tile = j;
+            int n_done0 = 0, n_done1 = 0, n_done2 = 0;   // PV MMAs issued per block
+            int k_tile = -1, v_tile = -1;                // last tiles whose K / V arrival was observed
+            // S[q & 1] = Q[blk] K[tile j]^T
+            auto issue_s = [&](const ItemIter& it, int q) -> bool {
+                const int j = it.j, blk = it.blk(), st = j % nk;
+                if (k_tile != j) {
+                    if (!mbar_wait(smem_u32(&c.k_full[st]), (j / nk) & 1, abort_flag, a.status)) return false;
+                    k_tile = j;
                 }
                 const int buf = q & 1;
                 if (q >= 2 && !mbar_wait(smem_u32(&c.s_free[buf]), ((q >> 1) - 1) & 1, abort_flag, a.status)) return false;
                 tc_fence_after();
                 const uint32_t qa = q_base + blk * (kBlockRows * 128u);
-                const uint32_t ka = kv_base + st * G::kStageBytes;
+                const uint32_t ka = k_base + st * G::kSlotBytes;
                 #pragma unroll
                 for (int ks = 0; ks < G::kKSteps; ++ks) {
                     const uint32_t hh = ks >> 2, off = (ks & 3) * 32u;
-                    tc_mma(tmem_s + buf * kTileKeys, desc_k_major(qa + hh * q_rows * 128u + off),
-                           desc_k_major(ka + hh * kHalfBytes + off), G::kIdescS, ks > 0);
+                    tc_mma(tmem_s + buf * TK, desc_k_major(qa + hh * q_rows * 128u + off),
+                           desc_k_major(ka + hh * G::kBoxBytes + off), G::kIdescS, ks > 0);
                 }
                 tc_commit(smem_u32(&c.s_full[blk][buf]));
+                if (it.last_of_tile()) tc_commit(smem_u32(&c.k_empty[st]));     // every S of tile j is queued: K may go
                 return true;
             };
-            int j, blk, q = 0;
-            sp.first(j, blk);
-            if (ok && j < sp.n_tiles) ok = issue_s(j, blk, 0);
-            while (ok && j < sp.n_tiles) {
-                int nj = j, nblk = blk;
-                sp.next(nj, nblk);
-                if (nj < sp.n_tiles && !issue_s(nj, nblk, q + 1)) break;
+            ItemIter cur;
+            cur.begin(sp);
+            int q = 0;
+            if (ok && !cur.done(sp)) ok = issue_s(cur, 0);
+            while (ok && !cur.done(sp)) {
+                ItemIter nxt = cur;
+                nxt.next(sp);
+                if (!nxt.done(sp) && !issue_s(nxt, q + 1)) break;
                 // O[blk] (+)= P[blk] V[tile j]
-                if (!mbar_wait(smem_u32(&c.p_full[blk]), n_done[blk] & 1, abort_flag, a.status)) break;
+                const int j = cur.j, blk = cur.blk(), st = j % nv_slots;
+                const int nd = blk == 0 ? n_done0 : (blk == 1 ? n_done1 : n_done2);
+                if (v_tile != j) {
+                    if (!mbar_wait(smem_u32(&c.v_full[st]), (j / nv_slots) & 1, abort_flag, a.status)) break;
+                    v_tile = j;
+                }
+                if (!mbar_wait(smem_u32(&c.p_full[blk]), nd & 1, abort_flag, a.status)) break;
                 tc_fence_after();
-                const int st = j % n_stages;
-                const uint32_t pa = p_base + blk * kPBytes;
-                const uint32_t va = kv_base + st * G::kStageBytes + G::kHalves * kHalfBytes;
+                const uint32_t pa = p_base + blk * p_bytes;
+                const uint32_t va = v_base + st * G::kSlotBytes;
                 #pragma unroll
-                for (int ks = 0; ks < kTileKeys / 16; ++ks)
-                    tc_mma(tmem + blk * G::kOCols, desc_k_major(pa + ks * 32u), desc_mn_major(va + ks * 2048u, kHalfBytes),
-                           G::kIdescPV, (n_done[blk] > 0 || ks > 0) ? 1u : 0u);
+                for (int ks = 0; ks < TK / 16; ++ks)
+                    tc_mma(tmem + blk * G::kOCols, desc_k_major(pa + (ks >> 2) * (p_rows * 128u) + (ks & 3) * 32u),
+                           desc_mn_major(va + ks * 2048u, G::kBoxBytes), G::kIdescPV, (nd > 0 || ks > 0) ? 1u : 0u);
                 tc_commit(smem_u32(&c.o_done[blk]));
-                if (nj != j) tc_commit(smem_u32(&c.kv_empty[st]));     // last block of tile j: the stage is free
-                ++n_done[blk];
-                j = nj; blk = nblk; ++q;
+                if (cur.last_of_tile()) tc_commit(smem_u32(&c.v_empty[st]));    // last block of tile j: V may go
+                if (blk == 0) ++n_done0; else if (blk == 1) ++n_done1; else ++n_done2;
+                cur = nxt;
+                ++q;
             }
         }
     }
@@ -495,45 +656,42 @@ msa_attention_kernel(const __grid_constant__ AttnArgs a) {
         // a warp whose 32 rows are all padding skips the arithmetic but keeps the barrier protocol
         const bool warp_active = __any_sync(0xffffffffu, ri.valid);
         const uint32_t o_addr = tmem + lane_base + my_blk * G::kOCols;
-        const uint32_t p_row = p_base + my_blk * kPBytes + row_in_blk * 128u;
-        int j, blk, q = 0;
-        sp.first(j, blk);
-        bool ok = true;
+        const uint32_t p_row = p_base + my_blk * p_bytes + row_in_blk * 128u;
+        const bool p_row_ok = static_cast<uint32_t>(row_in_blk) < p_rows;      // rows past p_rows are padding: never stored
+        ItemIter it;
+        it.begin(sp);
+        int q = 0;
         int prev_tile = -1;
         int n_use0 = 0, n_use1 = 0;                    // S buffers of this block consumed so far, per buffer
-        while (ok && j < sp.n_tiles) {
+        while (!it.done(sp)) {
+            const int j = it.j;
             const bool first_of_tile = (j != prev_tile);
             prev_tile = j;
-            if (blk == my_blk) {
+            if (it.blk() == my_blk) {
                 const int buf = q & 1;
                 if (!mbar_wait_warp(smem_u32(&c.s_full[my_blk][buf]), (buf ? n_use1 : n_use0) & 1, abort_flag, a.status)) break;
                 if (buf) ++n_use1; else ++n_use0;
                 tc_fence_after();
-                uint32_t sr[kTileKeys];
-                if (warp_active) {
-                    const uint32_t s_addr = tmem_s + lane_base + buf * kTileKeys;
-                    tmem_ld16<0>(s_addr, sr); tmem_ld16<16>(s_addr + 16, sr);
-                    tmem_ld16<32>(s_addr + 32, sr); tmem_ld16<48>(s_addr + 48, sr);
-                    tmem_wait_ld();
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&c.s_free[buf]));
+                const uint32_t s_addr = tmem_s + lane_base + buf * TK;
+                const int x = sp.first_key(j), nvk = sp.valid_keys(j);
+                const bool cache = sp.is_cache(j);
+                const bool masked = !cache || x + TK > sp.L || nvk < TK;
+                unsigned long long vis[TK / 64];
+                #pragma unroll
+                for (int hf = 0; hf < TK / 64; ++hf)
+                    vis[hf] = masked ? visible_mask(cache, x + hf * 64, nvk - hf * 64, sp.L, sp.gamma, ri, anc) : ~0ull;
 
+                uint32_t sr[64];
                 float corr = 1.f;
                 bool need = false;
+                // ---- pass 1: the tile's maximum ------------------------------------------------------
                 if (warp_active) {
-                    const int x = sp.first_key(j);
-                    const bool masked = !sp.is_cache(j) || x + kTileKeys > sp.L || sp.valid_keys(j) < kTileKeys;
-                    const unsigned long long vis = masked ? visible_mask(sp, j, ri, anc) : (ri.valid ? ~0ull : 0ull);
-                    const uint32_t vlo = static_cast<uint32_t>(vis), vhi = static_cast<uint32_t>(vis >> 32);
                     float mx = -INFINITY;
                     #pragma unroll
-                    for (int i = 0; i < kTileKeys; ++i) {
-                        const bool v = ((i < 32 ? vlo : vhi) >> (i & 31)) & 1u;
-                        const float s = v ? __uint_as_float(sr[i]) * a.scale_log2 : -INFINITY;
-                        sr[i] = __float_as_uint(s);
-                        mx = fmaxf(mx, s);
+                    for (int hf = 0; hf < TK / 64; ++hf) {
+                        tmem_ld64(s_addr + hf * 64, sr);
+                        tmem_wait_ld();
+                        mx = fmaxf(mx, masked ? chunk_max<true>(sr, a.scale_log2, vis[hf]) : chunk_max<false>(sr, a.scale_log2, 0ull));
                     }
                     need = mx > m_run + kRescaleStep;
                     if (need) {
@@ -541,6 +699,11 @@ msa_attention_kernel(const __grid_constant__ AttnArgs a) {
                         m_run = mx;
                         l_run *= corr;
                     }
+                }
+                if (TK == 64) {                             // the scores stay in registers: S can be overwritten
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&c.s_free[buf]));
                 }
                 // the previous PV of this block must be complete: it read the P tile that is about to
                 // be overwritten, and it wrote the accumulator that a raised maximum rescales
@@ -561,33 +724,38 @@ msa_attention_kernel(const __grid_constant__ AttnArgs a) {
                         }
                         tmem_wait_st();
                     }
+                    // ---- pass 2: P = exp2(S - m) as bf16, row sum ---------------------------------------
                     const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
                     float sum = 0.f;
                     #pragma unroll
-                    for (int ch = 0; ch < 8; ++ch) {           // 8 chunks of 8 keys = 16 B of bf16
-                        float p[8];
-                        #pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            p[i] = exp2f(__uint_as_float(sr[ch * 8 + i]) - m_use);
-                            sum += p[i];
+                    for (int hf = 0; hf < TK / 64; ++hf) {
+                        if (TK > 64) {
+                            tmem_ld64(s_addr + hf * 64, sr);
+                            tmem_wait_ld();
                         }
-                        const uint32_t dst = p_row + ((ch ^ (row_in_blk & 7)) << 4);
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pack_bf16(p[0], p[1])),
-                                     "r"(pack_bf16(p[2], p[3])), "r"(pack_bf16(p[4], p[5])), "r"(pack_bf16(p[6], p[7])) : "memory");
+                        if (p_row_ok) {
+                            const uint32_t dst = p_row + hf * (p_rows * 128u);
+                            sum += masked ? chunk_exp_store<true>(sr, a.scale_log2, m_use, vis[hf], dst, row_in_blk)
+                                          : chunk_exp_store<false>(sr, a.scale_log2, m_use, 0ull, dst, row_in_blk);
+                        }
                     }
                     l_run += sum;
                 }
+                if (TK > 64) {                              // both passes have read S
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&c.s_free[buf]));
+                }
                 // V rows past the tile's last valid key may hold anything (even NaN patterns): P is 0 there,
                 // but 0 * NaN is NaN, so the first block to use the tile clears them
-                const int nv = sp.valid_keys(j);
-                if (first_of_tile && nv < kTileKeys) {
-                    const int st = j % n_stages;
-                    if (!mbar_wait_warp(smem_u32(&c.kv_full[st]), (j / n_stages) & 1, abort_flag, a.status)) break;
-                    const uint32_t vdst = kv_base + st * G::kStageBytes + G::kHalves * kHalfBytes;
-                    const int n16 = (kTileKeys - nv) * 8 * G::kHalves;      // 16-byte pieces to clear
-                    for (int i = row_in_blk; i < n16; i += kBlockRows) {
-                        const int hh = i / ((kTileKeys - nv) * 8), rem = i - hh * ((kTileKeys - nv) * 8);
-                        const uint32_t dst = vdst + hh * kHalfBytes + (nv + (rem >> 3)) * 128u + ((rem & 7) << 4);
+                if (first_of_tile && nvk < TK) {
+                    const int st = j % nv_slots;
+                    if (!mbar_wait_warp(smem_u32(&c.v_full[st]), (j / nv_slots) & 1, abort_flag, a.status)) break;
+                    const uint32_t vdst = v_base + st * G::kSlotBytes;
+                    const int per_half = (TK - nvk) * 8;                     // 16-byte pieces to clear per half
+                    for (int i = row_in_blk; i < per_half * G::kHalves; i += kBlockRows) {
+                        const int hh = i / per_half, rem = i - hh * per_half;
+                        const uint32_t dst = vdst + hh * G::kBoxBytes + (nvk + (rem >> 3)) * 128u + ((rem & 7) << 4);
                         asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
                     }
                 }
@@ -596,7 +764,7 @@ msa_attention_kernel(const __grid_constant__ AttnArgs a) {
                 mbar_arrive(smem_u32(&c.p_full[my_blk]));
                 ++n_own;
             }
-            sp.next(j, blk);
+            it.next(sp);
             ++q;
         }
         // the block's last PV must have landed in TMEM before the accumulator is read
@@ -605,36 +773,25 @@ msa_attention_kernel(const __grid_constant__ AttnArgs a) {
             tc_fence_after();
         }
     }
-
     __syncwarp();     // the single-lane roles of warps 0 and 1 rejoin their warps
 
     // ======================================== epilogue ==========================================
     const bool has_acc = (warp >= 4) && n_own > 0;     // otherwise the partial is (m = -inf, l = 0, O = 0)
+    const uint32_t o_addr = tmem + lane_base + (warp >= 4 ? my_blk : 0) * G::kOCols;
     if (C == 1) {
         // the pair was not split: normalise and write this thread's row
         if (warp >= 4 && __any_sync(0xffffffffu, ri.valid) && !skip) {
             const float inv = 1.f / l_run;
-            __nv_bfloat16* dst;
-            float* lse;
-            if (!ri.valid) {
-                dst = nullptr; lse = nullptr;
-            } else if (ri.stream == 0) {
-                const long long idx = (static_cast<long long>(b) * a.max_nodes + ri.node) * a.n_heads + h;
-                dst = a.o_main + idx * HD;
-                lse = a.lse_main ? a.lse_main + idx : nullptr;
-            } else {
-                const long long idx = (spec_row0 + static_cast<long long>(ri.node) * a.gamma + (ri.stream - 1)) * a.n_heads + h;
-                dst = a.o_spec + idx * HD;
-                lse = a.lse_spec ? a.lse_spec + idx : nullptr;
-            }
-            if (lse) *lse = (m_run + log2f(l_run)) * 0.6931471805599453f;
-            const uint32_t o_addr = tmem + lane_base + my_blk * G::kOCols;
+            OutPtr dst;
+            dst.o = nullptr; dst.lse = nullptr;
+            if (ri.valid) dst = out_ptr<HD>(a, b, h, spec_row0, ri);
+            if (dst.lse) *dst.lse = (m_run + log2f(l_run)) * 0.6931471805599453f;
             #pragma unroll
             for (int c0 = 0; c0 < HD; c0 += 16) {
                 uint32_t orr[16];
                 if (has_acc) { tmem_ld16<0>(o_addr + c0, orr); tmem_wait_ld(); }     // all 32 lanes of the warp
                 else { for (int i = 0; i < 16; ++i) orr[i] = 0u; }
-                if (dst == nullptr) continue;
+                if (dst.o == nullptr) continue;
                 uint4 lo, hi;
                 lo.x = pack_bf16(__uint_as_float(orr[0]) * inv, __uint_as_float(orr[1]) * inv);
                 lo.y = pack_bf16(__uint_as_float(orr[2]) * inv, __uint_as_float(orr[3]) * inv);
@@ -644,8 +801,8 @@ msa_attention_kernel(const __grid_constant__ AttnArgs a) {
                 hi.y = pack_bf16(__uint_as_float(orr[10]) * inv, __uint_as_float(orr[11]) * inv);
                 hi.z = pack_bf16(__uint_as_float(orr[12]) * inv, __uint_as_float(orr[13]) * inv);
                 hi.w = pack_bf16(__uint_as_float(orr[14]) * inv, __uint_as_float(orr[15]) * inv);
-                *reinterpret_cast<uint4*>(dst + c0) = lo;
-                *reinterpret_cast<uint4*>(dst + c0 + 8) = hi;
+                *reinterpret_cast<uint4*>(dst.o + c0) = lo;
+                *reinterpret_cast<uint4*>(dst.o + c0 + 8) = hi;
             }
         }
     } else {
@@ -653,62 +810,69 @@ msa_attention_kernel(const __grid_constant__ AttnArgs a) {
         // Barrier A: all CTAs are done with their pipelines, so shared memory can be reused.
         cluster_arrive();
         cluster_wait();
-        const int rpc = kBlockRows / C;                 // rows of each block merged by one CTA
+        const int rpc_max = kBlockRows / C;             // row stride of the receive buffers
         if (warp >= 4) {
-            const uint32_t dst_rank = row_in_blk / rpc;
-            const int lr = row_in_blk - dst_rank * rpc;
-            // receiver layout: [block][source rank][local row][kMergePitch floats]
-            const uint32_t local = merge_base + (((my_blk * C + rank) * rpc + lr) * G::kMergePitch) * 4u;
-            const uint32_t remote = map_to_rank(local, dst_rank);
-            const uint32_t o_addr = tmem + lane_base + my_blk * G::kOCols;
-            #pragma unroll
-            for (int c0 = 0; c0 < HD; c0 += 16) {
-                uint32_t orr[16];
-                if (has_acc) { tmem_ld16<0>(o_addr + c0, orr); tmem_wait_ld(); }
-                else { for (int i = 0; i < 16; ++i) orr[i] = 0u; }
+            // valid row number vi of the block goes to CTA vi / rpc, local row vi % rpc
+            const int nvr = sp.n_valid(my_blk);
+            const int rpc = (nvr + C - 1) / C;
+            const int vi = ri.valid ? sp.valid_index(my_blk * kBlockRows + row_in_blk) : -1;
+            if (__any_sync(0xffffffffu, vi >= 0)) {
+                uint32_t remote = 0, ml_remote = 0;
+                if (vi >= 0) {
+                    const uint32_t dst_rank = vi / rpc;
+                    const int lr = vi - dst_rank * rpc;
+                    // receiver layout: [block][source rank][local row][kMergePitch floats]
+                    remote = map_to_rank(merge_base + (((my_blk * C + rank) * rpc_max + lr) * G::kMergePitch) * 4u, dst_rank);
+                    ml_remote = map_to_rank(smem_u32(&c.ml[my_blk][rank * rpc_max + lr]), dst_rank);
+                }
                 #pragma unroll
-                for (int i = 0; i < 16; i += 4)
-                    st_cluster_v4(remote + (c0 + i) * 4u, __uint_as_float(orr[i]), __uint_as_float(orr[i + 1]),
-                                  __uint_as_float(orr[i + 2]), __uint_as_float(orr[i + 3]));
+                for (int c0 = 0; c0 < HD; c0 += 16) {
+                    uint32_t orr[16];
+                    if (has_acc) { tmem_ld16<0>(o_addr + c0, orr); tmem_wait_ld(); }
+                    else { for (int i = 0; i < 16; ++i) orr[i] = 0u; }
+                    if (vi >= 0) {
+                        #pragma unroll
+                        for (int i = 0; i < 16; i += 4)
+                            st_cluster_v4(remote + (c0 + i) * 4u, orr[i], orr[i + 1], orr[i + 2], orr[i + 3]);
+                    }
+                }
+                if (vi >= 0) st_cluster_v2(ml_remote, m_run, l_run);
             }
-            const uint32_t ml_local = smem_u32(&c.ml[my_blk][rank * rpc + lr]);
-            st_cluster_v2(map_to_rank(ml_local, dst_rank), m_run, l_run);
         }
         // Barrier B: every partial has been delivered.
         cluster_arrive();
         cluster_wait();
-        if (warp >= 4 && row_in_blk < HD && !skip) {
-            const int col = row_in_blk;
-            for (int lr = 0; lr < rpc; ++lr) {
-                const int row = my_blk * kBlockRows + static_cast<int>(rank) * rpc + lr;
-                const RowInfo r = row_info(sp, row);
-                if (!r.valid) continue;
+        if (warp >= 4 && !skip) {
+            const int nvr = sp.n_valid(my_blk);
+            const int rpc = (nvr + C - 1) / C;
+            const int wq = warp & 3;
+            // one warp per row, one lane per four columns
+            for (int lr = wq; lr < rpc; lr += 4) {
+                const int vi = static_cast<int>(rank) * rpc + lr;
+                if (vi >= nvr) break;
+                const RowInfo r = row_info(sp, sp.row_of(my_blk, vi));
                 float mx = -INFINITY;
-                for (int s = 0; s < C; ++s) mx = fmaxf(mx, c.ml[my_blk][s * rpc + lr].x);
-                float acc = 0.f, l = 0.f;
+                for (int s = 0; s < C; ++s) mx = fmaxf(mx, c.ml[my_blk][s * rpc_max + lr].x);
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                float l = 0.f;
                 for (int s = 0; s < C; ++s) {
-                    const float2 ml = c.ml[my_blk][s * rpc + lr];
+                    const float2 ml = c.ml[my_blk][s * rpc_max + lr];
                     const float w = exp2f(ml.x - mx);         // 0 for a CTA that saw no visible key
                     l += w * ml.y;
-                    float v;
-                    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v)
-                                 : "r"(merge_base + (((my_blk * C + s) * rpc + lr) * G::kMergePitch + col) * 4u) : "memory");
-                    acc += w * v;
+                    if (lane * 4 < HD) {
+                        const float4 v = ld_shared_v4(merge_base + (((my_blk * C + s) * rpc_max + lr) * G::kMergePitch + lane * 4) * 4u);
+                        acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+                    }
                 }
-                long long idx;
-                __nv_bfloat16* dst;
-                float* lse;
-                if (r.stream == 0) {
-                    idx = (static_cast<long long>(b) * a.max_nodes + r.node) * a.n_heads + h;
-                    dst = a.o_main + idx * HD;
-                    lse = a.lse_main ? a.lse_main + idx : nullptr;
-                } else {
-                    idx = (spec_row0 + static_cast<long long>(r.node) * a.gamma + (r.stream - 1)) * a.n_heads + h;
-                    dst = a.o_spec + idx * HD;
-                    lse = a.lse_spec ? a.lse_spec + idx : nullptr;
+                const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, r);
+                const float inv = 1.f / l;
+                if (lane * 4 < HD) {
+                    uint2 o;
+                    o.x = pack_bf16(acc.x * inv, acc.y * inv);
+                    o.y = pack_bf16(acc.z * inv, acc.w * inv);
+                    *reinterpret_cast<uint2*>(dst.o + lane * 4) = o;
                 }
-                dst[col] = __float2bfloat16_rn(acc / l);
-                if (lse && col == 0) *lse = (mx + log2f(l)) * 0.6931471805599453f;
+                if (dst.lse && lane == 0) *dst.lse = (mx + log2f(l)) * 0.6931471805599453f;
             }
         }
     }
@@ -719,7 +883,7 @@ msa_attention_kernel(const __grid_constant__ AttnArgs a) {
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
 }
 
@@ -758,7 +922,7 @@ static bool make_map(CUtensorMap* out, const void* basep, int d, long long n1, l
 }
 
 struct AttnPlan {
-    int tmax8, spec_rows, n_blocks, n_stages, cluster, threads;
+    int tmax8, spec_rows, n_blocks, tile_keys, n_kslots, n_vslots, cluster, threads;
     size_t smem;
 };
 
@@ -769,33 +933,41 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     const int halves = p.head_dim > 64 ? 2 : 1;
     plan->tmax8 = (p.max_nodes + 7) / 8 * 8;
     plan->spec_rows = p.gamma > 0 ? (p.max_nodes * p.gamma + 7) / 8 * 8 : 0;
-    plan->n_blocks = (plan->tmax8 + plan->spec_rows + kBlockRows - 1) / kBlockRows;
-    plan->threads = kAuxThreads + plan->n_blocks * kBlockRows;
+    const int q_rows = plan->tmax8 + plan->spec_rows;
+    plan->n_blocks = (q_rows + kBlockRows - 1) / kBlockRows;
+    plan->tile_keys = plan->n_blocks == 1 ? 128 : 64;
+    plan->threads = kAuxThreads + (plan->n_blocks == 1 ? 1 : kMaxBlocks) * kBlockRows;
     // cluster size: the largest power of two that still fits the grid on the SMs in one wave
     const long long pairs = static_cast<long long>(p.batch) * p.n_heads;
     int c = 1;
     while (c < 8 && pairs * (c * 2) <= sm_count()) c *= 2;
     plan->cluster = c;
-    const size_t qp = static_cast<size_t>(plan->n_blocks) * (halves * kBlockRows * 128 + kPBytes);
-    const size_t stage = static_cast<size_t>(2) * halves * kHalfBytes;
-    int ns = static_cast<int>((kMaxDynSmem - 1024 - qp) / stage);
-    ns = ns > kMaxStages ? kMaxStages : ns;
-    if (ns < 2) return false;
-    plan->n_stages = ns;
-    size_t bytes = qp + ns * stage;
+    const int p_rows = plan->n_blocks == 1 ? q_rows : kBlockRows;
+    const size_t qp = static_cast<size_t>(halves) * q_rows * 128 +
+                      static_cast<size_t>(plan->n_blocks) * (plan->tile_keys / 64) * p_rows * 128;
+    const size_t slot = static_cast<size_t>(halves) * plan->tile_keys * 128;
+    // the MMAs of the last block read up to 128 rows past the start of their block: keep that inside the allocation
+    const size_t overhang = static_cast<size_t>(kBlockRows) * 128;
+    int slots = static_cast<int>((kMaxDynSmem - 1024 - qp) / slot);
+    if (slots > 2 * kMaxSlots) slots = 2 * kMaxSlots;
+    if (slots < 4) return false;
+    plan->n_kslots = slots / 2 > 2 ? 2 : slots / 2;          // K comes back right after S: two slots suffice
+    plan->n_vslots = slots - plan->n_kslots > kMaxSlots ? kMaxSlots : slots - plan->n_kslots;
+    size_t bytes = qp + static_cast<size_t>(plan->n_kslots + plan->n_vslots) * slot;
+    if (bytes < qp + overhang) bytes = qp + overhang;
     const size_t merge = static_cast<size_t>(plan->n_blocks) * kBlockRows * (p.head_dim + 4) * 4;
     if (c > 1 && merge > bytes) bytes = merge;
     plan->smem = bytes + 1024;
     return plan->smem <= static_cast<size_t>(kMaxDynSmem);
 }
 
-template <int HD>
+template <int HD, int TK>
 static int32_t launch(const AttnArgs& args, const AttnPlan& plan, long long pairs, cudaStream_t stream) {
     static bool configured[64] = {false};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return SS_ERR_CUDA;
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        if (cudaFuncSetAttribute(msa_attention_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem) !=
+        if (cudaFuncSetAttribute(msa_attention_kernel<HD, TK>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem) !=
             cudaSuccess)
             return SS_ERR_CUDA;
         configured[dev] = true;
@@ -813,7 +985,7 @@ static int32_t launch(const AttnArgs& args, const AttnPlan& plan, long long pair
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, msa_attention_kernel<HD>, args) == cudaSuccess ? SS_OK : SS_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, msa_attention_kernel<HD, TK>, args) == cudaSuccess ? SS_OK : SS_ERR_CUDA;
 }
 
 }  // namespace ss
@@ -849,24 +1021,25 @@ extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
     if (p->workspace_bytes < ss_msa_attention_workspace_bytes(p)) return SS_ERR_WORKSPACE;
 
     ss::AttnArgs a;
-    const int d = p->head_dim, H = p->n_heads;
+    const int d = p->head_dim, H = p->n_heads, tk = plan.tile_keys;
     const bool shared_heads = (p->kv_head_stride == 0);
     const long long kv_heads = shared_heads ? 1 : H;
     const long long kv_hstride = shared_heads ? d : p->kv_head_stride;
-    bool ok = ss::make_map(&a.tm_k, p->k_cache, d, kv_heads, kv_hstride, p->kv_total_slots, p->kv_slot_stride, ss::kTileKeys) &&
-              ss::make_map(&a.tm_v, p->v_cache, d, kv_heads, kv_hstride, p->kv_total_slots, p->kv_slot_stride, ss::kTileKeys) &&
+    bool ok = ss::make_map(&a.tm_k, p->k_cache, d, kv_heads, kv_hstride, p->kv_total_slots, p->kv_slot_stride, tk) &&
+              ss::make_map(&a.tm_v, p->v_cache, d, kv_heads, kv_hstride, p->kv_total_slots, p->kv_slot_stride, tk) &&
               ss::make_map(&a.tm_qm, p->q_main, d, H, d, rows_main, static_cast<long long>(H) * d, plan.tmax8);
     if (ok && p->gamma > 0) {
         const long long rows_spec = rows_main * p->gamma;
         ok = ss::make_map(&a.tm_qs, p->q_spec, d, H, d, rows_spec, static_cast<long long>(H) * d, plan.spec_rows) &&
-             ss::make_map(&a.tm_ks, p->k_spec, d, H, d, rows_spec, static_cast<long long>(H) * d, ss::kTileKeys) &&
-             ss::make_map(&a.tm_vs, p->v_spec, d, H, d, rows_spec, static_cast<long long>(H) * d, ss::kTileKeys);
+             ss::make_map(&a.tm_ks, p->k_spec, d, H, d, rows_spec, static_cast<long long>(H) * d, tk) &&
+             ss::make_map(&a.tm_vs, p->v_spec, d, H, d, rows_spec, static_cast<long long>(H) * d, tk);
     } else if (ok) {
         a.tm_qs = a.tm_qm; a.tm_ks = a.tm_k; a.tm_vs = a.tm_v;     // never used when gamma == 0
     }
     if (!ok) return SS_ERR_CUDA;
     a.batch = p->batch; a.n_heads = H; a.gamma = p->gamma; a.max_nodes = p->max_nodes;
-    a.tmax8 = plan.tmax8; a.spec_rows = plan.spec_rows; a.n_blocks = plan.n_blocks; a.n_stages = plan.n_stages;
+    a.tmax8 = plan.tmax8; a.spec_rows = plan.spec_rows; a.n_blocks = plan.n_blocks;
+    a.n_kslots = plan.n_kslots; a.n_vslots = plan.n_vslots;
     a.cluster = plan.cluster;
     a.head_coord = shared_heads ? 0 : 1;
     a.scale_log2 = p->sm_scale * 1.4426950408889634f;
@@ -878,9 +1051,16 @@ extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
     a.status = reinterpret_cast<int*>(p->workspace);
     const long long pairs = static_cast<long long>(p->batch) * H;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (tk == 128) {
+        switch (d) {
+            case 64: return ss::launch<64, 128>(a, plan, pairs, s);
+            case 80: return ss::launch<80, 128>(a, plan, pairs, s);
+            default: return ss::launch<128, 128>(a, plan, pairs, s);
+        }
+    }
     switch (d) {
-        case 64: return ss::launch<64>(a, plan, pairs, s);
-        case 80: return ss::launch<80>(a, plan, pairs, s);
-        default: return ss::launch<128>(a, plan, pairs, s);
+        case 64: return ss::launch<64, 64>(a, plan, pairs, s);
+        case 80: return ss::launch<80, 64>(a, plan, pairs, s);
+        default: return ss::launch<128, 64>(a, plan, pairs, s);
     }
 }
