@@ -11,10 +11,10 @@
 //   thread 0    TMA producer: Q once, then K tiles and V tiles into two independent rings
 //               (mbarrier complete_tx); swizzle-128B boxes straight from the caller's strided tensors.
 //               A K slot is handed back as soon as S has been computed, a V slot after P V.
-//   warp 1      tcgen05 issuer: S = Q K^T (128 x TK x d) into one of two TMEM buffers, later
-//               O += P V (128 x d x TK) into the block's TMEM accumulator; tcgen05.commit arrives
-//               on the mbarriers that hand buffers back.  TK = 128 keys when the head has one row
-//               block (N = 128 MMAs run at the full tensor rate), 64 keys otherwise.
+//   warp 1      tcgen05 issuer of S = Q K^T (128 x TK x d) into one of two TMEM buffers;
+//   warp 2      tcgen05 issuer of O += P V (128 x d x TK) into the block's TMEM accumulator;
+//               tcgen05.commit arrives on the mbarriers that hand buffers back.  TK = 128 keys when
+//               the head has one row block (N = 128 MMAs run at the full tensor rate), 64 otherwise.
 //   warps 4..   one warpgroup per 128-row block, one thread per query row: tcgen05.ld of the S row,
 //               tree / stream mask from the node's 64-bit ancestor word, online softmax in fp32
 //               registers (the running maximum is only raised when it would grow by more than 2^8,
@@ -413,8 +413,15 @@ __device__ __forceinline__ float chunk_exp_store(const uint32_t (&v)[64], float 
     return (sum[0] + sum[1]) + (sum[2] + sum[3]);
 }
 
-template <int HD, int TK>
+// Kernel variants.  kMulti: up to three 128-row blocks, 64-key tiles.  kSingle: one block of 65..128
+// rows, 128-key tiles.  kDual: at most 64 rows: the block holds the rows twice, copy 0 takes keys
+// 0..63 of every 128-key tile and copy 1 keys 64..127 (P is zero in the other half), so all four
+// sub-partitions share the exponentials; the two copies are merged like two more split-KV partials.
+enum Mode { kMulti = 0, kSingle = 1, kDual = 2 };
+
+template <int HD, int MODE>
 struct Geo {
+    static constexpr int TK = MODE == kMulti ? 64 : 128;          // keys per tile
     static constexpr int kHalves = HD > 64 ? 2 : 1;               // 64-element boxes along head_dim
     static constexpr int kBoxBytes = TK * 128;                    // one TMA box: TK rows x 128 B
     static constexpr int kSlotBytes = kHalves * kBoxBytes;        // one K tile (or one V tile)
@@ -423,7 +430,9 @@ struct Geo {
     static constexpr uint32_t kIdescS = idesc_bf16(TK, false);
     static constexpr uint32_t kIdescPV = idesc_bf16(HD, true);
     static constexpr int kOCols = 128;                            // TMEM columns reserved per block accumulator
-    static constexpr int kThreads = kAuxThreads + (TK == 128 ? 1 : kMaxBlocks) * kBlockRows;
+    static constexpr int kThreads = kAuxThreads + (MODE == kMulti ? kMaxBlocks : 1) * kBlockRows;
+    static constexpr int kCopies = MODE == kDual ? 2 : 1;
+    static constexpr int kChunks = MODE == kSingle ? 2 : 1;       // 64-key chunks of a tile one thread handles
 };
 
 // destination of a row's output and log-sum-exp
@@ -447,9 +456,10 @@ __device__ __forceinline__ OutPtr out_ptr(const AttnArgs& a, int b, int h, long 
 }
 
 // ---------------------------------------------------------------------------------------------
-template <int HD, int TK>
-__global__ void __launch_bounds__(Geo<HD, TK>::kThreads, 1) msa_attention_kernel(const __grid_constant__ AttnArgs a) {
-    using G = Geo<HD, TK>;
+template <int HD, int MODE>
+__global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kernel(const __grid_constant__ AttnArgs a) {
+    using G = Geo<HD, MODE>;
+    constexpr int TK = G::TK;
     extern __shared__ unsigned char smem_raw[];
     __shared__ Ctrl c;
 
@@ -466,16 +476,18 @@ __global__ void __launch_bounds__(Geo<HD, TK>::kThreads, 1) msa_attention_kernel
     int T = min(max(a.trees[b].n_nodes, 0), a.max_nodes);
     const long long slot0 = a.kv_start[b];
     const int cap = a.kv_capacity != nullptr ? a.kv_capacity[b] : 0x7fffffff;
+    const long long spec_row0 = static_cast<long long>(b) * a.max_nodes * a.gamma;   // first stream row of the sequence
 
     // ---- shared-memory carve-up (1024-byte aligned: swizzle atoms) ----------------------------
     // Q and P keep only the rows that exist; an MMA that reads the rows of a 128-row block past them
     // picks up whatever follows in shared memory, which only ever reaches padding rows of S and O.
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t q_rows = a.tmax8 + a.spec_rows;                      // rows TMA brings in
-    const uint32_t p_rows = n_blocks == 1 ? q_rows : kBlockRows;
+    const uint32_t q_rows = a.tmax8 + a.spec_rows;                      // rows of the head's query tile
+    const uint32_t q_smem_rows = MODE == kDual ? kBlockRows : q_rows;   // kDual: second copy at row 64
+    const uint32_t p_rows = MODE == kMulti || MODE == kDual ? kBlockRows : q_rows;
     const uint32_t p_bytes = (TK / 64) * p_rows * 128u;                 // one block's P tile
-    const uint32_t q_base = base;                                       // [half][q_rows][128 B]
-    const uint32_t p_base = q_base + G::kHalves * q_rows * 128u;        // [block][key half][p_rows][128 B]
+    const uint32_t q_base = base;                                       // [half][q_smem_rows][128 B]
+    const uint32_t p_base = q_base + G::kHalves * q_smem_rows * 128u;   // [block][key half][p_rows][128 B]
     const uint32_t k_base = p_base + n_blocks * p_bytes;                // [slot][half][TK][128 B]
     const uint32_t v_base = k_base + nk * G::kSlotBytes;                // [slot][half][TK][128 B]
     const uint32_t merge_base = base;                                   // aliases everything above, after the main loop
@@ -494,8 +506,18 @@ __global__ void __launch_bounds__(Geo<HD, TK>::kThreads, 1) msa_attention_kernel
         for (int s = 0; s < kMaxBlocks; ++s) { mbar_init(smem_u32(&c.p_full[s]), kBlockRows); mbar_init(smem_u32(&c.o_done[s]), 1); }
         c.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        tma_prefetch_desc(&a.tm_k); tma_prefetch_desc(&a.tm_v); tma_prefetch_desc(&a.tm_qm);
-        if (a.gamma > 0) { tma_prefetch_desc(&a.tm_qs); tma_prefetch_desc(&a.tm_ks); tma_prefetch_desc(&a.tm_vs); }
+        // the queries depend on nothing but (sequence, head): request them before the lengths are known
+        const uint32_t qbar = smem_u32(&c.q_full);
+        mbar_expect_tx(qbar, G::kCopies * G::kHalves * q_rows * 128u);
+        #pragma unroll
+        for (int cp = 0; cp < G::kCopies; ++cp) {
+            #pragma unroll
+            for (int hh = 0; hh < G::kHalves; ++hh) {
+                const uint32_t dst = q_base + hh * q_smem_rows * 128u + cp * 64u * 128u;
+                tma_load_3d(dst, &a.tm_qm, hh * 64, h, b * a.max_nodes, qbar);
+                if (a.gamma > 0) tma_load_3d(dst + a.tmax8 * 128u, &a.tm_qs, hh * 64, h, static_cast<int>(spec_row0), qbar);
+            }
+        }
     }
     constexpr uint32_t kTmemCols = 512;
     if (warp == 1) {
@@ -511,7 +533,6 @@ __global__ void __launch_bounds__(Geo<HD, TK>::kThreads, 1) msa_attention_kernel
     if (tid >= kAuxThreads && tid < kAuxThreads + SS_MAX_NODES) c.anc[tid - kAuxThreads] = a.trees[b].anc_mask[tid - kAuxThreads];
 
     const Span<TK> sp = make_span<TK>(a, L, T, static_cast<int>(rank));
-    const long long spec_row0 = static_cast<long long>(b) * a.max_nodes * a.gamma;   // first stream row of the sequence
 
     // K tile j / V tile j of the span -> ring slot (thread 0 only)
     auto load_k = [&](int j) {
@@ -538,19 +559,18 @@ __global__ void __launch_bounds__(Geo<HD, TK>::kThreads, 1) msa_attention_kernel
             else tma_load_3d(dst + hh * G::kBoxBytes, &a.tm_vs, hh * 64, h, static_cast<int>(spec_row0 + x), bar);
         }
     };
-    // the producer starts before the CTA-wide synchronisation: Q and the first tiles need no hand-back
+    // the producer starts before the CTA-wide synchronisation: the first tiles need no hand-back
     const int n_early = min(sp.n_tiles, min(nk, nv_slots));
-    if (tid == 0 && sp.n_tiles > 0) {
-        const uint32_t qbytes = G::kHalves * q_rows * 128u;
-        mbar_expect_tx(smem_u32(&c.q_full), qbytes);
-        #pragma unroll
-        for (int hh = 0; hh < G::kHalves; ++hh) {
-            tma_load_3d(q_base + hh * q_rows * 128u, &a.tm_qm, hh * 64, h, b * a.max_nodes, smem_u32(&c.q_full));
-            if (a.gamma > 0)
-                tma_load_3d(q_base + hh * q_rows * 128u + a.tmax8 * 128u, &a.tm_qs, hh * 64, h,
-                            static_cast<int>(spec_row0), smem_u32(&c.q_full));
-        }
+    if (tid == 0) {
         for (int j = 0; j < n_early; ++j) { load_k(j); load_v(j); }
+    }
+    // kDual: each thread's "other" key half of P stays zero for the whole kernel
+    if (MODE == kDual && tid >= kAuxThreads) {
+        const int r = tid - kAuxThreads;
+        const uint32_t dst = p_base + (1 - (r >> 6)) * (p_rows * 128u) + r * 128u;
+        #pragma unroll
+        for (int i = 0; i < 8; ++i) asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst + i * 16), "r"(0u) : "memory");
+        fence_async_smem();
     }
     tc_fence_before();
     __syncthreads();
@@ -575,50 +595,50 @@ __global__ void __launch_bounds__(Geo<HD, TK>::kThreads, 1) msa_attention_kernel
             }
             if (!ok) {
                 // gave up: let the copies already in flight land before shared memory is reused or released
-                mbar_drain(smem_u32(&c.q_full), 0);
                 for (int j = max(0, jk - nk); j < jk; ++j) mbar_drain(smem_u32(&c.k_full[j % nk]), (j / nk) & 1);
                 for (int j = max(0, jv - nv_slots); j < jv; ++j) mbar_drain(smem_u32(&c.v_full[j % nv_slots]), (j / nv_slots) & 1);
             }
         }
     }
-    // ================================= warp 1: MMA issuer =======================================
+    // ============================ warp 1: issues S = Q K^T =========================================
     else if (warp == 1) {
-        if (lane == 0 && sp.n_tiles > 0) {
+        if (lane == 0) {
+            // the query tile is always requested, so it is always awaited (shared memory is reused later)
             bool ok = mbar_wait(smem_u32(&c.q_full), 0, abort_flag, a.status);
-            int n_done0 = 0, n_done1 = 0, n_done2 = 0;   // PV MMAs issued per block
-            int k_tile = -1, v_tile = -1;                // last tiles whose K / V arrival was observed
-            // S[q & 1] = Q[blk] K[tile j]^T
-            auto issue_s = [&](const ItemIter& it, int q) -> bool {
-                const int j = it.j, blk = it.blk(), st = j % nk;
+            if (!ok) mbar_drain(smem_u32(&c.q_full), 0);
+            ItemIter it;
+            it.begin(sp);
+            int k_tile = -1;
+            for (int q = 0; ok && !it.done(sp); ++q, it.next(sp)) {
+                const int j = it.j, blk = it.blk(), st = j % nk, buf = q & 1;
                 if (k_tile != j) {
-                    if (!mbar_wait(smem_u32(&c.k_full[st]), (j / nk) & 1, abort_flag, a.status)) return false;
+                    if (!mbar_wait(smem_u32(&c.k_full[st]), (j / nk) & 1, abort_flag, a.status)) break;
                     k_tile = j;
                 }
-                const int buf = q & 1;
-                if (q >= 2 && !mbar_wait(smem_u32(&c.s_free[buf]), ((q >> 1) - 1) & 1, abort_flag, a.status)) return false;
+                if (q >= 2 && !mbar_wait(smem_u32(&c.s_free[buf]), ((q >> 1) - 1) & 1, abort_flag, a.status)) break;
                 tc_fence_after();
                 const uint32_t qa = q_base + blk * (kBlockRows * 128u);
                 const uint32_t ka = k_base + st * G::kSlotBytes;
                 #pragma unroll
                 for (int ks = 0; ks < G::kKSteps; ++ks) {
                     const uint32_t hh = ks >> 2, off = (ks & 3) * 32u;
-                    tc_mma(tmem_s + buf * TK, desc_k_major(qa + hh * q_rows * 128u + off),
+                    tc_mma(tmem_s + buf * TK, desc_k_major(qa + hh * q_smem_rows * 128u + off),
                            desc_k_major(ka + hh * G::kBoxBytes + off), G::kIdescS, ks > 0);
                 }
                 tc_commit(smem_u32(&c.s_full[blk][buf]));
                 if (it.last_of_tile()) tc_commit(smem_u32(&c.k_empty[st]));     // every S of tile j is queued: K may go
-                return true;
-            };
-            ItemIter cur;
-            cur.begin(sp);
-            int q = 0;
-            if (ok && !cur.done(sp)) ok = issue_s(cur, 0);
-            while (ok && !cur.done(sp)) {
-                ItemIter nxt = cur;
-                nxt.next(sp);
-                if (!nxt.done(sp) && !issue_s(nxt, q + 1)) break;
-                // O[blk] (+)= P[blk] V[tile j]
-                const int j = cur.j, blk = cur.blk(), st = j % nv_slots;
+            }
+        }
+    }
+    // ============================ warp 2: issues O += P V ==========================================
+    else if (warp == 2) {
+        if (lane == 0) {
+            ItemIter it;
+            it.begin(sp);
+            int n_done0 = 0, n_done1 = 0, n_done2 = 0;   // PV batches issued per block
+            int v_tile = -1;
+            for (; !it.done(sp); it.next(sp)) {
+                const int j = it.j, blk = it.blk(), st = j % nv_slots;
                 const int nd = blk == 0 ? n_done0 : (blk == 1 ? n_done1 : n_done2);
                 if (v_tile != j) {
                     if (!mbar_wait(smem_u32(&c.v_full[st]), (j / nv_slots) & 1, abort_flag, a.status)) break;
@@ -633,10 +653,8 @@ __global__ void __launch_bounds__(Geo<HD, TK>::kThreads, 1) msa_attention_kernel
                     tc_mma(tmem + blk * G::kOCols, desc_k_major(pa + (ks >> 2) * (p_rows * 128u) + (ks & 3) * 32u),
                            desc_mn_major(va + ks * 2048u, G::kBoxBytes), G::kIdescPV, (nd > 0 || ks > 0) ? 1u : 0u);
                 tc_commit(smem_u32(&c.o_done[blk]));
-                if (cur.last_of_tile()) tc_commit(smem_u32(&c.v_empty[st]));    // last block of tile j: V may go
+                if (it.last_of_tile()) tc_commit(smem_u32(&c.v_empty[st]));     // last block of tile j: V may go
                 if (blk == 0) ++n_done0; else if (blk == 1) ++n_done1; else ++n_done2;
-                cur = nxt;
-                ++q;
             }
         }
     }
@@ -645,13 +663,14 @@ __global__ void __launch_bounds__(Geo<HD, TK>::kThreads, 1) msa_attention_kernel
     float m_run = -INFINITY, l_run = 0.f;
     int n_own = 0;
     const int my_blk = (warp - 4) >> 2;
-    const int row_in_blk = ((warp & 3) << 5) | lane;
+    const int row_in_blk = ((warp & 3) << 5) | lane;                          // TMEM lane of this thread
+    const int copy = MODE == kDual ? (row_in_blk >> 6) : 0;
+    const int lrow = MODE == kDual ? (row_in_blk & 63) : row_in_blk;          // row of the block this thread works for
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     RowInfo ri;
     ri.valid = false; ri.node = 0; ri.stream = 0;
     if (warp >= 4) {
-        const int row = my_blk * kBlockRows + row_in_blk;
-        ri = row_info(sp, row);
+        ri = row_info(sp, my_blk * kBlockRows + lrow);
         const unsigned long long anc = ri.valid ? c.anc[ri.node] : 0ull;
         // a warp whose 32 rows are all padding skips the arithmetic but keeps the barrier protocol
         const bool warp_active = __any_sync(0xffffffffu, ri.valid);
@@ -660,112 +679,109 @@ __global__ void __launch_bounds__(Geo<HD, TK>::kThreads, 1) msa_attention_kernel
         const bool p_row_ok = static_cast<uint32_t>(row_in_blk) < p_rows;      // rows past p_rows are padding: never stored
         ItemIter it;
         it.begin(sp);
-        int q = 0;
         int prev_tile = -1;
         int n_use0 = 0, n_use1 = 0;                    // S buffers of this block consumed so far, per buffer
-        while (!it.done(sp)) {
+        for (int q = 0; !it.done(sp); ++q, it.next(sp)) {
             const int j = it.j;
             const bool first_of_tile = (j != prev_tile);
             prev_tile = j;
-            if (it.blk() == my_blk) {
-                const int buf = q & 1;
-                if (!mbar_wait_warp(smem_u32(&c.s_full[my_blk][buf]), (buf ? n_use1 : n_use0) & 1, abort_flag, a.status)) break;
-                if (buf) ++n_use1; else ++n_use0;
-                tc_fence_after();
-                const uint32_t s_addr = tmem_s + lane_base + buf * TK;
-                const int x = sp.first_key(j), nvk = sp.valid_keys(j);
-                const bool cache = sp.is_cache(j);
-                const bool masked = !cache || x + TK > sp.L || nvk < TK;
-                unsigned long long vis[TK / 64];
-                #pragma unroll
-                for (int hf = 0; hf < TK / 64; ++hf)
-                    vis[hf] = masked ? visible_mask(cache, x + hf * 64, nvk - hf * 64, sp.L, sp.gamma, ri, anc) : ~0ull;
+            if (it.blk() != my_blk) continue;
+            const int buf = q & 1;
+            if (!mbar_wait_warp(smem_u32(&c.s_full[my_blk][buf]), (buf ? n_use1 : n_use0) & 1, abort_flag, a.status)) break;
+            if (buf) ++n_use1; else ++n_use0;
+            tc_fence_after();
+            const uint32_t s_addr = tmem_s + lane_base + buf * TK;
+            const int x = sp.first_key(j), nvk = sp.valid_keys(j);
+            const bool cache = sp.is_cache(j);
+            const bool masked = !cache || x + TK > sp.L || nvk < TK;
+            // chunk ch of this thread covers keys x + 64 * (copy + ch) ...
+            unsigned long long vis[G::kChunks];
+            #pragma unroll
+            for (int ch = 0; ch < G::kChunks; ++ch)
+                vis[ch] = masked ? visible_mask(cache, x + (copy + ch) * 64, nvk - (copy + ch) * 64, sp.L, sp.gamma, ri, anc) : ~0ull;
 
-                uint32_t sr[64];
-                float corr = 1.f;
-                bool need = false;
-                // ---- pass 1: the tile's maximum ------------------------------------------------------
-                if (warp_active) {
-                    float mx = -INFINITY;
-                    #pragma unroll
-                    for (int hf = 0; hf < TK / 64; ++hf) {
-                        tmem_ld64(s_addr + hf * 64, sr);
-                        tmem_wait_ld();
-                        mx = fmaxf(mx, masked ? chunk_max<true>(sr, a.scale_log2, vis[hf]) : chunk_max<false>(sr, a.scale_log2, 0ull));
-                    }
-                    need = mx > m_run + kRescaleStep;
-                    if (need) {
-                        corr = exp2f(m_run - mx);           // 0 when nothing was visible so far
-                        m_run = mx;
-                        l_run *= corr;
-                    }
+            uint32_t sr[64];
+            float corr = 1.f;
+            bool need = false;
+            // ---- pass 1: the tile's maximum ----------------------------------------------------------
+            if (warp_active) {
+                float mx = -INFINITY;
+                #pragma unroll
+                for (int ch = 0; ch < G::kChunks; ++ch) {
+                    tmem_ld64(s_addr + (copy + ch) * 64, sr);
+                    tmem_wait_ld();
+                    mx = fmaxf(mx, masked ? chunk_max<true>(sr, a.scale_log2, vis[ch]) : chunk_max<false>(sr, a.scale_log2, 0ull));
                 }
-                if (TK == 64) {                             // the scores stay in registers: S can be overwritten
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&c.s_free[buf]));
+                need = mx > m_run + kRescaleStep;
+                if (need) {
+                    corr = exp2f(m_run - mx);           // 0 when nothing was visible so far
+                    m_run = mx;
+                    l_run *= corr;
                 }
-                // the previous PV of this block must be complete: it read the P tile that is about to
-                // be overwritten, and it wrote the accumulator that a raised maximum rescales
-                if (n_own > 0) {
-                    if (!mbar_wait_warp(smem_u32(&c.o_done[my_blk]), (n_own - 1) & 1, abort_flag, a.status)) break;
-                    tc_fence_after();
-                }
-                if (warp_active) {
-                    if (n_own > 0 && __any_sync(0xffffffffu, need)) {
-                        #pragma unroll
-                        for (int c0 = 0; c0 < HD; c0 += 16) {
-                            uint32_t orr[16];
-                            tmem_ld16<0>(o_addr + c0, orr);
-                            tmem_wait_ld();
-                            #pragma unroll
-                            for (int i = 0; i < 16; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * corr);
-                            tmem_st16<0>(o_addr + c0, orr);
-                        }
-                        tmem_wait_st();
-                    }
-                    // ---- pass 2: P = exp2(S - m) as bf16, row sum ---------------------------------------
-                    const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
-                    float sum = 0.f;
-                    #pragma unroll
-                    for (int hf = 0; hf < TK / 64; ++hf) {
-                        if (TK > 64) {
-                            tmem_ld64(s_addr + hf * 64, sr);
-                            tmem_wait_ld();
-                        }
-                        if (p_row_ok) {
-                            const uint32_t dst = p_row + hf * (p_rows * 128u);
-                            sum += masked ? chunk_exp_store<true>(sr, a.scale_log2, m_use, vis[hf], dst, row_in_blk)
-                                          : chunk_exp_store<false>(sr, a.scale_log2, m_use, 0ull, dst, row_in_blk);
-                        }
-                    }
-                    l_run += sum;
-                }
-                if (TK > 64) {                              // both passes have read S
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&c.s_free[buf]));
-                }
-                // V rows past the tile's last valid key may hold anything (even NaN patterns): P is 0 there,
-                // but 0 * NaN is NaN, so the first block to use the tile clears them
-                if (first_of_tile && nvk < TK) {
-                    const int st = j % nv_slots;
-                    if (!mbar_wait_warp(smem_u32(&c.v_full[st]), (j / nv_slots) & 1, abort_flag, a.status)) break;
-                    const uint32_t vdst = v_base + st * G::kSlotBytes;
-                    const int per_half = (TK - nvk) * 8;                     // 16-byte pieces to clear per half
-                    for (int i = row_in_blk; i < per_half * G::kHalves; i += kBlockRows) {
-                        const int hh = i / per_half, rem = i - hh * per_half;
-                        const uint32_t dst = vdst + hh * G::kBoxBytes + (nvk + (rem >> 3)) * 128u + ((rem & 7) << 4);
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
-                    }
-                }
-                fence_async_smem();
-                tc_fence_before();
-                mbar_arrive(smem_u32(&c.p_full[my_blk]));
-                ++n_own;
             }
-            it.next(sp);
-            ++q;
+            if (G::kChunks == 1) {                      // the scores stay in registers: S can be overwritten
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&c.s_free[buf]));
+            }
+            // the previous PV of this block must be complete: it read the P tile that is about to
+            // be overwritten, and it wrote the accumulator that a raised maximum rescales
+            if (n_own > 0) {
+                if (!mbar_wait_warp(smem_u32(&c.o_done[my_blk]), (n_own - 1) & 1, abort_flag, a.status)) break;
+                tc_fence_after();
+            }
+            if (warp_active) {
+                if (n_own > 0 && __any_sync(0xffffffffu, need)) {
+                    #pragma unroll
+                    for (int c0 = 0; c0 < HD; c0 += 16) {
+                        uint32_t orr[16];
+                        tmem_ld16<0>(o_addr + c0, orr);
+                        tmem_wait_ld();
+                        #pragma unroll
+                        for (int i = 0; i < 16; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * corr);
+                        tmem_st16<0>(o_addr + c0, orr);
+                    }
+                    tmem_wait_st();
+                }
+                // ---- pass 2: P = exp2(S - m) as bf16, row sum -------------------------------------------
+                const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
+                float sum = 0.f;
+                #pragma unroll
+                for (int ch = 0; ch < G::kChunks; ++ch) {
+                    if (G::kChunks > 1) {
+                        tmem_ld64(s_addr + ch * 64, sr);
+                        tmem_wait_ld();
+                    }
+                    if (p_row_ok) {
+                        const uint32_t dst = p_row + (copy + ch) * (p_rows * 128u);
+                        sum += masked ? chunk_exp_store<true>(sr, a.scale_log2, m_use, vis[ch], dst, row_in_blk)
+                                      : chunk_exp_store<false>(sr, a.scale_log2, m_use, 0ull, dst, row_in_blk);
+                    }
+                }
+                l_run += sum;
+            }
+            if (G::kChunks > 1) {                       // both passes have read S
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&c.s_free[buf]));
+            }
+            // V rows past the tile's last valid key may hold anything (even NaN patterns): P is 0 there,
+            // but 0 * NaN is NaN, so the first block to use the tile clears them
+            if (first_of_tile && nvk < TK) {
+                const int st = j % nv_slots;
+                if (!mbar_wait_warp(smem_u32(&c.v_full[st]), (j / nv_slots) & 1, abort_flag, a.status)) break;
+                const uint32_t vdst = v_base + st * G::kSlotBytes;
+                const int per_half = (TK - nvk) * 8;                     // 16-byte pieces to clear per half
+                for (int i = row_in_blk; i < per_half * G::kHalves; i += kBlockRows) {
+                    const int hh = i / per_half, rem = i - hh * per_half;
+                    const uint32_t dst = vdst + hh * G::kBoxBytes + (nvk + (rem >> 3)) * 128u + ((rem & 7) << 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
+                }
+            }
+            fence_async_smem();
+            tc_fence_before();
+            mbar_arrive(smem_u32(&c.p_full[my_blk]));
+            ++n_own;
         }
         // the block's last PV must have landed in TMEM before the accumulator is read
         if (n_own > 0) {
@@ -773,12 +789,12 @@ __global__ void __launch_bounds__(Geo<HD, TK>::kThreads, 1) msa_attention_kernel
             tc_fence_after();
         }
     }
-    __syncwarp();     // the single-lane roles of warps 0 and 1 rejoin their warps
+    __syncwarp();     // the single-lane roles of warps 0..2 rejoin their warps
 
     // ======================================== epilogue ==========================================
     const bool has_acc = (warp >= 4) && n_own > 0;     // otherwise the partial is (m = -inf, l = 0, O = 0)
     const uint32_t o_addr = tmem + lane_base + (warp >= 4 ? my_blk : 0) * G::kOCols;
-    if (C == 1) {
+    if (C == 1 && MODE != kDual) {
         // the pair was not split: normalise and write this thread's row
         if (warp >= 4 && __any_sync(0xffffffffu, ri.valid) && !skip) {
             const float inv = 1.f / l_run;
@@ -809,22 +825,48 @@ __global__ void __launch_bounds__(Geo<HD, TK>::kThreads, 1) msa_attention_kernel
         // Every thread of the cluster passes both barriers, whatever happened above.
         // Barrier A: all CTAs are done with their pipelines, so shared memory can be reused.
         cluster_arrive();
-        cluster_wait();
-        const int rpc_max = kBlockRows / C;             // row stride of the receive buffers
+        const int n_src = C * G::kCopies;                       // partials per row
+        const int rpc_max = kBlockRows / n_src;                 // row stride of the receive buffers
+        // valid row number vi of the block goes to CTA vi / rpc, local row vi % rpc
+        int vi = -1;
+        uint32_t remote = 0, ml_remote = 0;
+        bool sender = false;
         if (warp >= 4) {
-            // valid row number vi of the block goes to CTA vi / rpc, local row vi % rpc
             const int nvr = sp.n_valid(my_blk);
             const int rpc = (nvr + C - 1) / C;
-            const int vi = ri.valid ? sp.valid_index(my_blk * kBlockRows + row_in_blk) : -1;
-            if (__any_sync(0xffffffffu, vi >= 0)) {
-                uint32_t remote = 0, ml_remote = 0;
-                if (vi >= 0) {
-                    const uint32_t dst_rank = vi / rpc;
-                    const int lr = vi - dst_rank * rpc;
-                    // receiver layout: [block][source rank][local row][kMergePitch floats]
-                    remote = map_to_rank(merge_base + (((my_blk * C + rank) * rpc_max + lr) * G::kMergePitch) * 4u, dst_rank);
-                    ml_remote = map_to_rank(smem_u32(&c.ml[my_blk][rank * rpc_max + lr]), dst_rank);
+            vi = ri.valid ? sp.valid_index(my_blk * kBlockRows + lrow) : -1;
+            sender = __any_sync(0xffffffffu, vi >= 0);
+            if (vi >= 0) {
+                const uint32_t dst_rank = vi / rpc;
+                const int lr = vi - dst_rank * rpc;
+                const int src = static_cast<int>(rank) * G::kCopies + copy;
+                // receiver layout: [block][source][local row][kMergePitch floats]
+                remote = map_to_rank(merge_base + (((my_blk * n_src + src) * rpc_max + lr) * G::kMergePitch) * 4u, dst_rank);
+                ml_remote = map_to_rank(smem_u32(&c.ml[my_blk][src * rpc_max + lr]), dst_rank);
+            }
+        }
+        if (MODE != kMulti) {
+            // 256-thread variants have the registers to fetch the whole accumulator row while the barrier completes
+            uint32_t orr[HD];
+            if (sender) {
+                if (has_acc) {
+                    #pragma unroll
+                    for (int c0 = 0; c0 < HD; c0 += 16) tmem_ld16<0>(o_addr + c0, *reinterpret_cast<uint32_t(*)[16]>(&orr[c0]));
+                    tmem_wait_ld();
+                } else {
+                    #pragma unroll
+                    for (int i = 0; i < HD; ++i) orr[i] = 0u;
                 }
+            }
+            cluster_wait();
+            if (vi >= 0) {
+                #pragma unroll
+                for (int i = 0; i < HD; i += 4) st_cluster_v4(remote + i * 4u, orr[i], orr[i + 1], orr[i + 2], orr[i + 3]);
+                st_cluster_v2(ml_remote, m_run, l_run);
+            }
+        } else {
+            cluster_wait();
+            if (sender) {
                 #pragma unroll
                 for (int c0 = 0; c0 < HD; c0 += 16) {
                     uint32_t orr[16];
@@ -848,20 +890,20 @@ __global__ void __launch_bounds__(Geo<HD, TK>::kThreads, 1) msa_attention_kernel
             const int wq = warp & 3;
             // one warp per row, one lane per four columns
             for (int lr = wq; lr < rpc; lr += 4) {
-                const int vi = static_cast<int>(rank) * rpc + lr;
-                if (vi >= nvr) break;
-                const RowInfo r = row_info(sp, sp.row_of(my_blk, vi));
+                const int v = static_cast<int>(rank) * rpc + lr;
+                if (v >= nvr) break;
+                const RowInfo r = row_info(sp, sp.row_of(my_blk, v));
                 float mx = -INFINITY;
-                for (int s = 0; s < C; ++s) mx = fmaxf(mx, c.ml[my_blk][s * rpc_max + lr].x);
+                for (int s = 0; s < n_src; ++s) mx = fmaxf(mx, c.ml[my_blk][s * rpc_max + lr].x);
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
                 float l = 0.f;
-                for (int s = 0; s < C; ++s) {
+                for (int s = 0; s < n_src; ++s) {
                     const float2 ml = c.ml[my_blk][s * rpc_max + lr];
-                    const float w = exp2f(ml.x - mx);         // 0 for a CTA that saw no visible key
+                    const float w = exp2f(ml.x - mx);         // 0 for a partial that saw no visible key
                     l += w * ml.y;
                     if (lane * 4 < HD) {
-                        const float4 v = ld_shared_v4(merge_base + (((my_blk * C + s) * rpc_max + lr) * G::kMergePitch + lane * 4) * 4u);
-                        acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+                        const float4 x4 = ld_shared_v4(merge_base + (((my_blk * n_src + s) * rpc_max + lr) * G::kMergePitch + lane * 4) * 4u);
+                        acc.x += w * x4.x; acc.y += w * x4.y; acc.z += w * x4.z; acc.w += w * x4.w;
                     }
                 }
                 const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, r);
@@ -922,7 +964,7 @@ static bool make_map(CUtensorMap* out, const void* basep, int d, long long n1, l
 }
 
 struct AttnPlan {
-    int tmax8, spec_rows, n_blocks, tile_keys, n_kslots, n_vslots, cluster, threads;
+    int tmax8, spec_rows, n_blocks, mode, tile_keys, n_kslots, n_vslots, cluster, threads;
     size_t smem;
 };
 
@@ -935,15 +977,17 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     plan->spec_rows = p.gamma > 0 ? (p.max_nodes * p.gamma + 7) / 8 * 8 : 0;
     const int q_rows = plan->tmax8 + plan->spec_rows;
     plan->n_blocks = (q_rows + kBlockRows - 1) / kBlockRows;
-    plan->tile_keys = plan->n_blocks == 1 ? 128 : 64;
-    plan->threads = kAuxThreads + (plan->n_blocks == 1 ? 1 : kMaxBlocks) * kBlockRows;
+    plan->mode = plan->n_blocks > 1 ? kMulti : (q_rows <= 64 ? kDual : kSingle);
+    plan->tile_keys = plan->mode == kMulti ? 64 : 128;
+    plan->threads = kAuxThreads + (plan->mode == kMulti ? kMaxBlocks : 1) * kBlockRows;
     // cluster size: the largest power of two that still fits the grid on the SMs in one wave
     const long long pairs = static_cast<long long>(p.batch) * p.n_heads;
     int c = 1;
     while (c < 8 && pairs * (c * 2) <= sm_count()) c *= 2;
     plan->cluster = c;
-    const int p_rows = plan->n_blocks == 1 ? q_rows : kBlockRows;
-    const size_t qp = static_cast<size_t>(halves) * q_rows * 128 +
+    const int p_rows = plan->mode == kSingle ? q_rows : kBlockRows;
+    const int q_smem_rows = plan->mode == kDual ? kBlockRows : q_rows;
+    const size_t qp = static_cast<size_t>(halves) * q_smem_rows * 128 +
                       static_cast<size_t>(plan->n_blocks) * (plan->tile_keys / 64) * p_rows * 128;
     const size_t slot = static_cast<size_t>(halves) * plan->tile_keys * 128;
     // the MMAs of the last block read up to 128 rows past the start of their block: keep that inside the allocation
@@ -961,13 +1005,13 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     return plan->smem <= static_cast<size_t>(kMaxDynSmem);
 }
 
-template <int HD, int TK>
+template <int HD, int MODE>
 static int32_t launch(const AttnArgs& args, const AttnPlan& plan, long long pairs, cudaStream_t stream) {
     static bool configured[64] = {false};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return SS_ERR_CUDA;
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        if (cudaFuncSetAttribute(msa_attention_kernel<HD, TK>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem) !=
+        if (cudaFuncSetAttribute(msa_attention_kernel<HD, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem) !=
             cudaSuccess)
             return SS_ERR_CUDA;
         configured[dev] = true;
@@ -985,7 +1029,7 @@ static int32_t launch(const AttnArgs& args, const AttnPlan& plan, long long pair
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, msa_attention_kernel<HD, TK>, args) == cudaSuccess ? SS_OK : SS_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, msa_attention_kernel<HD, MODE>, args) == cudaSuccess ? SS_OK : SS_ERR_CUDA;
 }
 
 }  // namespace ss
@@ -1051,16 +1095,23 @@ extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
     a.status = reinterpret_cast<int*>(p->workspace);
     const long long pairs = static_cast<long long>(p->batch) * H;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (tk == 128) {
+    if (plan.mode == ss::kDual) {
         switch (d) {
-            case 64: return ss::launch<64, 128>(a, plan, pairs, s);
-            case 80: return ss::launch<80, 128>(a, plan, pairs, s);
-            default: return ss::launch<128, 128>(a, plan, pairs, s);
+            case 64: return ss::launch<64, ss::kDual>(a, plan, pairs, s);
+            case 80: return ss::launch<80, ss::kDual>(a, plan, pairs, s);
+            default: return ss::launch<128, ss::kDual>(a, plan, pairs, s);
+        }
+    }
+    if (plan.mode == ss::kSingle) {
+        switch (d) {
+            case 64: return ss::launch<64, ss::kSingle>(a, plan, pairs, s);
+            case 80: return ss::launch<80, ss::kSingle>(a, plan, pairs, s);
+            default: return ss::launch<128, ss::kSingle>(a, plan, pairs, s);
         }
     }
     switch (d) {
-        case 64: return ss::launch<64, 64>(a, plan, pairs, s);
-        case 80: return ss::launch<80, 64>(a, plan, pairs, s);
-        default: return ss::launch<128, 64>(a, plan, pairs, s);
+        case 64: return ss::launch<64, ss::kMulti>(a, plan, pairs, s);
+        case 80: return ss::launch<80, ss::kMulti>(a, plan, pairs, s);
+        default: return ss::launch<128, ss::kMulti>(a, plan, pairs, s);
     }
 }
