@@ -50,7 +50,7 @@ struct alignas(64) AttnArgs {
     int batch, n_heads, gamma, max_nodes;
     int tmax8;                       // max_nodes rounded up to 8: first stream row in shared memory
     int spec_rows;                   // max_nodes * gamma rounded up to 8 (rows of the q_spec box)
-    int n_blocks, cluster;
+    int n_blocks, cluster, cluster_shift;   // cluster = 1 << cluster_shift
     int n_kslots, n_vslots;          // ring depths
     int head_coord;                  // 1, or 0 when all heads share one K/V (head stride 0)
     float scale_log2;                // sm_scale * log2(e)
@@ -278,6 +278,15 @@ struct Span {
     }
 };
 
+// position in a ring of n slots: slot index and the number of completed rounds
+struct Ring {
+    int slot, round;
+    __device__ __forceinline__ void start() { slot = 0; round = 0; }
+    __device__ __forceinline__ void advance(int n) {
+        if (++slot == n) { slot = 0; ++round; }
+    }
+};
+
 // (tile, block) items in tile-major order, only the active ones
 struct ItemIter {
     int j;
@@ -315,8 +324,9 @@ __device__ __forceinline__ Span<TK> make_span(const AttnArgs& a, int L, int T, i
     const int ec = L + T;
     const int uc = (ec + kUnit - 1) / kUnit, us = (s.n_stream + kUnit - 1) / kUnit;
     const int u = uc + us;
-    const int u0 = static_cast<int>(static_cast<long long>(u) * rank / a.cluster);
-    const int u1 = static_cast<int>(static_cast<long long>(u) * (rank + 1) / a.cluster);
+    // u < 2^28 and rank < 8: the products fit 32 bits; the cluster size is a power of two
+    const int u0 = static_cast<int>((static_cast<unsigned>(u) * static_cast<unsigned>(rank)) >> a.cluster_shift);
+    const int u1 = static_cast<int>((static_cast<unsigned>(u) * static_cast<unsigned>(rank + 1)) >> a.cluster_shift);
     s.kc0 = min(u0, uc) * kUnit;
     s.kc1 = min(min(u1, uc) * kUnit, ec);
     s.ks0 = (max(u0, uc) - uc) * kUnit;
@@ -471,13 +481,6 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     const int n_blocks = a.n_blocks, nk = a.n_kslots, nv_slots = a.n_vslots;
     volatile int* abort_flag = &c.abort;
 
-    // per-sequence scalars (every thread reads them; the loads overlap the set-up below)
-    int L = a.kv_len[b];
-    int T = min(max(a.trees[b].n_nodes, 0), a.max_nodes);
-    const long long slot0 = a.kv_start[b];
-    const int cap = a.kv_capacity != nullptr ? a.kv_capacity[b] : 0x7fffffff;
-    const long long spec_row0 = static_cast<long long>(b) * a.max_nodes * a.gamma;   // first stream row of the sequence
-
     // ---- shared-memory carve-up (1024-byte aligned: swizzle atoms) ----------------------------
     // Q and P keep only the rows that exist; an MMA that reads the rows of a 128-row block past them
     // picks up whatever follows in shared memory, which only ever reaches padding rows of S and O.
@@ -491,21 +494,31 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     const uint32_t k_base = p_base + n_blocks * p_bytes;                // [slot][half][TK][128 B]
     const uint32_t v_base = k_base + nk * G::kSlotBytes;                // [slot][half][TK][128 B]
     const uint32_t merge_base = base;                                   // aliases everything above, after the main loop
+    const long long spec_row0 = static_cast<long long>(b) * a.max_nodes * a.gamma;   // first stream row of the sequence
 
     // ---- prologue ---------------------------------------------------------------------------------
-    if (tid == 0) {
+    // Everything up to the dependency wait touches no global memory, so under programmatic dependent
+    // launch it overlaps the tail of the previous kernel in the stream.
+    if (tid == 0) {                                       // the barriers TMA completes on
         mbar_init(smem_u32(&c.q_full), 1);
-        for (int s = 0; s < kMaxSlots; ++s) {
-            mbar_init(smem_u32(&c.k_full[s]), 1); mbar_init(smem_u32(&c.k_empty[s]), 1);
-            mbar_init(smem_u32(&c.v_full[s]), 1); mbar_init(smem_u32(&c.v_empty[s]), 1);
-        }
+        for (int s = 0; s < kMaxSlots; ++s) { mbar_init(smem_u32(&c.k_full[s]), 1); mbar_init(smem_u32(&c.v_full[s]), 1); }
+        c.abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        tma_prefetch_desc(&a.tm_qm); tma_prefetch_desc(&a.tm_k); tma_prefetch_desc(&a.tm_v);
+        if (a.gamma > 0) { tma_prefetch_desc(&a.tm_qs); tma_prefetch_desc(&a.tm_ks); tma_prefetch_desc(&a.tm_vs); }
+    } else if (tid == 64) {                               // every other barrier (first used after the CTA-wide sync)
+        for (int s = 0; s < kMaxSlots; ++s) { mbar_init(smem_u32(&c.k_empty[s]), 1); mbar_init(smem_u32(&c.v_empty[s]), 1); }
         for (int s = 0; s < 2; ++s) {
             mbar_init(smem_u32(&c.s_free[s]), 4);
             for (int k = 0; k < kMaxBlocks; ++k) mbar_init(smem_u32(&c.s_full[k][s]), 1);
         }
         for (int s = 0; s < kMaxBlocks; ++s) { mbar_init(smem_u32(&c.p_full[s]), kBlockRows); mbar_init(smem_u32(&c.o_done[s]), 1); }
-        c.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    if (tid == 0) {
         // the queries depend on nothing but (sequence, head): request them before the lengths are known
         const uint32_t qbar = smem_u32(&c.q_full);
         mbar_expect_tx(qbar, G::kCopies * G::kHalves * q_rows * 128u);
@@ -519,6 +532,11 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             }
         }
     }
+    // per-sequence scalars (every thread reads them)
+    int L = a.kv_len[b];
+    int T = min(max(a.trees[b].n_nodes, 0), a.max_nodes);
+    const long long slot0 = a.kv_start[b];
+    const int cap = a.kv_capacity != nullptr ? a.kv_capacity[b] : 0x7fffffff;
     constexpr uint32_t kTmemCols = 512;
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&c.tmem_base)), "r"(kTmemCols) : "memory");
@@ -534,9 +552,8 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
 
     const Span<TK> sp = make_span<TK>(a, L, T, static_cast<int>(rank));
 
-    // K tile j / V tile j of the span -> ring slot (thread 0 only)
-    auto load_k = [&](int j) {
-        const int st = j % nk;
+    // K tile j / V tile j of the span -> ring slot st (thread 0 only)
+    auto load_k = [&](int j, int st) {
         const uint32_t bar = smem_u32(&c.k_full[st]);
         mbar_expect_tx(bar, G::kSlotBytes);
         const uint32_t dst = k_base + st * G::kSlotBytes;
@@ -547,8 +564,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             else tma_load_3d(dst + hh * G::kBoxBytes, &a.tm_ks, hh * 64, h, static_cast<int>(spec_row0 + x), bar);
         }
     };
-    auto load_v = [&](int j) {
-        const int st = j % nv_slots;
+    auto load_v = [&](int j, int st) {
         const uint32_t bar = smem_u32(&c.v_full[st]);
         mbar_expect_tx(bar, G::kSlotBytes);
         const uint32_t dst = v_base + st * G::kSlotBytes;
@@ -562,7 +578,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     // the producer starts before the CTA-wide synchronisation: the first tiles need no hand-back
     const int n_early = min(sp.n_tiles, min(nk, nv_slots));
     if (tid == 0) {
-        for (int j = 0; j < n_early; ++j) { load_k(j); load_v(j); }
+        for (int j = 0; j < n_early; ++j) { load_k(j, j); load_v(j, j); }
     }
     // kDual: each thread's "other" key half of P stays zero for the whole kernel
     if (MODE == kDual && tid >= kAuxThreads) {
@@ -582,21 +598,24 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     if (warp == 0) {
         if (lane == 0 && sp.n_tiles > n_early) {
             int jk = n_early, jv = n_early;               // next K tile / V tile to request
+            Ring rk, rv;                                  // their ring positions
+            rk.start(); rv.start();
+            for (int i = 0; i < n_early; ++i) { rk.advance(nk); rv.advance(nv_slots); }
             bool ok = true;
             while (ok && (jk < sp.n_tiles || jv < sp.n_tiles)) {
                 // K slots come back early (after S), so K runs ahead of V by at most one ring
                 if (jk < sp.n_tiles && (jk <= jv || jv >= sp.n_tiles)) {
-                    ok = jk < nk || mbar_wait(smem_u32(&c.k_empty[jk % nk]), ((jk / nk) - 1) & 1, abort_flag, a.status);
-                    if (ok) load_k(jk++);
+                    ok = rk.round == 0 || mbar_wait(smem_u32(&c.k_empty[rk.slot]), (rk.round - 1) & 1, abort_flag, a.status);
+                    if (ok) { load_k(jk++, rk.slot); rk.advance(nk); }
                 } else {
-                    ok = jv < nv_slots || mbar_wait(smem_u32(&c.v_empty[jv % nv_slots]), ((jv / nv_slots) - 1) & 1, abort_flag, a.status);
-                    if (ok) load_v(jv++);
+                    ok = rv.round == 0 || mbar_wait(smem_u32(&c.v_empty[rv.slot]), (rv.round - 1) & 1, abort_flag, a.status);
+                    if (ok) { load_v(jv++, rv.slot); rv.advance(nv_slots); }
                 }
             }
             if (!ok) {
                 // gave up: let the copies already in flight land before shared memory is reused or released
-                for (int j = max(0, jk - nk); j < jk; ++j) mbar_drain(smem_u32(&c.k_full[j % nk]), (j / nk) & 1);
-                for (int j = max(0, jv - nv_slots); j < jv; ++j) mbar_drain(smem_u32(&c.v_full[j % nv_slots]), (j / nv_slots) & 1);
+                for (int s = 0; s < nk; ++s) mbar_drain(smem_u32(&c.k_full[s]), (s < rk.slot ? rk.round : rk.round - 1) & 1);
+                for (int s = 0; s < nv_slots; ++s) mbar_drain(smem_u32(&c.v_full[s]), (s < rv.slot ? rv.round : rv.round - 1) & 1);
             }
         }
     }
@@ -606,19 +625,24 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             // the query tile is always requested, so it is always awaited (shared memory is reused later)
             bool ok = mbar_wait(smem_u32(&c.q_full), 0, abort_flag, a.status);
             if (!ok) mbar_drain(smem_u32(&c.q_full), 0);
-            ItemIter it;
+            ItemIter it = {0, 0u};
             it.begin(sp);
-            int k_tile = -1;
+            Ring rk;
+            rk.start();
+            int k_tile = it.j;                            // tile the ring position belongs to
+            for (int i = 0; i < k_tile; ++i) rk.advance(nk);
+            bool k_seen = false;
             for (int q = 0; ok && !it.done(sp); ++q, it.next(sp)) {
-                const int j = it.j, blk = it.blk(), st = j % nk, buf = q & 1;
-                if (k_tile != j) {
-                    if (!mbar_wait(smem_u32(&c.k_full[st]), (j / nk) & 1, abort_flag, a.status)) break;
-                    k_tile = j;
+                const int j = it.j, blk = it.blk(), buf = q & 1;
+                while (k_tile < j) { rk.advance(nk); ++k_tile; k_seen = false; }
+                if (!k_seen) {
+                    if (!mbar_wait(smem_u32(&c.k_full[rk.slot]), rk.round & 1, abort_flag, a.status)) break;
+                    k_seen = true;
                 }
                 if (q >= 2 && !mbar_wait(smem_u32(&c.s_free[buf]), ((q >> 1) - 1) & 1, abort_flag, a.status)) break;
                 tc_fence_after();
                 const uint32_t qa = q_base + blk * (kBlockRows * 128u);
-                const uint32_t ka = k_base + st * G::kSlotBytes;
+                const uint32_t ka = k_base + rk.slot * G::kSlotBytes;
                 #pragma unroll
                 for (int ks = 0; ks < G::kKSteps; ++ks) {
                     const uint32_t hh = ks >> 2, off = (ks & 3) * 32u;
@@ -626,34 +650,39 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                            desc_k_major(ka + hh * G::kBoxBytes + off), G::kIdescS, ks > 0);
                 }
                 tc_commit(smem_u32(&c.s_full[blk][buf]));
-                if (it.last_of_tile()) tc_commit(smem_u32(&c.k_empty[st]));     // every S of tile j is queued: K may go
+                if (it.last_of_tile()) tc_commit(smem_u32(&c.k_empty[rk.slot]));     // every S of tile j is queued: K may go
             }
         }
     }
     // ============================ warp 2: issues O += P V ==========================================
     else if (warp == 2) {
         if (lane == 0) {
-            ItemIter it;
+            ItemIter it = {0, 0u};
             it.begin(sp);
             int n_done0 = 0, n_done1 = 0, n_done2 = 0;   // PV batches issued per block
-            int v_tile = -1;
+            Ring rv;
+            rv.start();
+            int v_tile = it.j;
+            for (int i = 0; i < v_tile; ++i) rv.advance(nv_slots);
+            bool v_seen = false;
             for (; !it.done(sp); it.next(sp)) {
-                const int j = it.j, blk = it.blk(), st = j % nv_slots;
+                const int j = it.j, blk = it.blk();
                 const int nd = blk == 0 ? n_done0 : (blk == 1 ? n_done1 : n_done2);
-                if (v_tile != j) {
-                    if (!mbar_wait(smem_u32(&c.v_full[st]), (j / nv_slots) & 1, abort_flag, a.status)) break;
-                    v_tile = j;
+                while (v_tile < j) { rv.advance(nv_slots); ++v_tile; v_seen = false; }
+                if (!v_seen) {
+                    if (!mbar_wait(smem_u32(&c.v_full[rv.slot]), rv.round & 1, abort_flag, a.status)) break;
+                    v_seen = true;
                 }
                 if (!mbar_wait(smem_u32(&c.p_full[blk]), nd & 1, abort_flag, a.status)) break;
                 tc_fence_after();
                 const uint32_t pa = p_base + blk * p_bytes;
-                const uint32_t va = v_base + st * G::kSlotBytes;
+                const uint32_t va = v_base + rv.slot * G::kSlotBytes;
                 #pragma unroll
                 for (int ks = 0; ks < TK / 16; ++ks)
                     tc_mma(tmem + blk * G::kOCols, desc_k_major(pa + (ks >> 2) * (p_rows * 128u) + (ks & 3) * 32u),
                            desc_mn_major(va + ks * 2048u, G::kBoxBytes), G::kIdescPV, (nd > 0 || ks > 0) ? 1u : 0u);
                 tc_commit(smem_u32(&c.o_done[blk]));
-                if (it.last_of_tile()) tc_commit(smem_u32(&c.v_empty[st]));     // last block of tile j: V may go
+                if (it.last_of_tile()) tc_commit(smem_u32(&c.v_empty[rv.slot]));     // last block of tile j: V may go
                 if (blk == 0) ++n_done0; else if (blk == 1) ++n_done1; else ++n_done2;
             }
         }
@@ -677,14 +706,19 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
         const uint32_t o_addr = tmem + lane_base + my_blk * G::kOCols;
         const uint32_t p_row = p_base + my_blk * p_bytes + row_in_blk * 128u;
         const bool p_row_ok = static_cast<uint32_t>(row_in_blk) < p_rows;      // rows past p_rows are padding: never stored
-        ItemIter it;
+        ItemIter it = {0, 0u};
         it.begin(sp);
         int prev_tile = -1;
         int n_use0 = 0, n_use1 = 0;                    // S buffers of this block consumed so far, per buffer
+        Ring rv;                                       // V ring position of tile v_tile
+        rv.start();
+        int v_tile = it.j;
+        for (int i = 0; i < v_tile; ++i) rv.advance(nv_slots);
         for (int q = 0; !it.done(sp); ++q, it.next(sp)) {
             const int j = it.j;
             const bool first_of_tile = (j != prev_tile);
             prev_tile = j;
+            while (v_tile < j) { rv.advance(nv_slots); ++v_tile; }
             if (it.blk() != my_blk) continue;
             const int buf = q & 1;
             if (!mbar_wait_warp(smem_u32(&c.s_full[my_blk][buf]), (buf ? n_use1 : n_use0) & 1, abort_flag, a.status)) break;
@@ -765,16 +799,18 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&c.s_free[buf]));
             }
-            // V rows past the tile's last valid key may hold anything (even NaN patterns): P is 0 there,
-            // but 0 * NaN is NaN, so the first block to use the tile clears them
-            if (first_of_tile && nvk < TK) {
-                const int st = j % nv_slots;
-                if (!mbar_wait_warp(smem_u32(&c.v_full[st]), (j / nv_slots) & 1, abort_flag, a.status)) break;
-                const uint32_t vdst = v_base + st * G::kSlotBytes;
-                const int per_half = (TK - nvk) * 8;                     // 16-byte pieces to clear per half
-                for (int i = row_in_blk; i < per_half * G::kHalves; i += kBlockRows) {
-                    const int hh = i / per_half, rem = i - hh * per_half;
-                    const uint32_t dst = vdst + hh * G::kBoxBytes + (nvk + (rem >> 3)) * 128u + ((rem & 7) << 4);
+            // V rows past the end of the sequence's keys may hold anything (even NaN patterns): P is 0
+            // there, but 0 * NaN is NaN, so the first block to use such a tile clears them.  Rows that
+            // only lie past this CTA's share of the keys are real data and need nothing.
+            const int region_left = (cache ? sp.L + sp.T : sp.n_stream) - x;      // real rows in the tile
+            if (first_of_tile && region_left < TK) {
+                if (!mbar_wait_warp(smem_u32(&c.v_full[rv.slot]), rv.round & 1, abort_flag, a.status)) break;
+                const uint32_t vdst = v_base + rv.slot * G::kSlotBytes;
+                constexpr int kPieceShift = G::kHalves == 2 ? 4 : 3;              // 16-byte pieces per row: 8 per half
+                const int n_pieces = (TK - region_left) << kPieceShift;
+                for (int i = row_in_blk; i < n_pieces; i += kBlockRows) {
+                    const int r = region_left + (i >> kPieceShift), pc = i & ((1 << kPieceShift) - 1);
+                    const uint32_t dst = vdst + (pc >> 3) * G::kBoxBytes + r * 128u + ((pc & 7) << 4);
                     asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
                 }
             }
@@ -1022,13 +1058,17 @@ static int32_t launch(const AttnArgs& args, const AttnPlan& plan, long long pair
     // always more than half of an SM's shared memory: one CTA per SM, so a CTA never queues for TMEM
     cfg.dynamicSmemBytes = plan.smem < 120 * 1024 ? 120 * 1024 : plan.smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = static_cast<unsigned>(plan.cluster);
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    // programmatic dependent launch: the CTAs may be scheduled while the previous kernel of the stream
+    // drains; the kernel touches global memory only after its griddepcontrol.wait, so stream order holds
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, msa_attention_kernel<HD, MODE>, args) == cudaSuccess ? SS_OK : SS_ERR_CUDA;
 }
 
@@ -1085,6 +1125,8 @@ extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
     a.tmax8 = plan.tmax8; a.spec_rows = plan.spec_rows; a.n_blocks = plan.n_blocks;
     a.n_kslots = plan.n_kslots; a.n_vslots = plan.n_vslots;
     a.cluster = plan.cluster;
+    a.cluster_shift = 0;
+    while ((1 << a.cluster_shift) < plan.cluster) ++a.cluster_shift;
     a.head_coord = shared_heads ? 0 : 1;
     a.scale_log2 = p->sm_scale * 1.4426950408889634f;
     a.o_main = static_cast<__nv_bfloat16*>(p->o_main);
