@@ -71,6 +71,7 @@ struct Ctrl {
     unsigned long long s_full[kMaxBlocks][2];   // per (block, S buffer): a warpgroup sees every phase of its own
     unsigned long long s_free[2];
     unsigned long long p_full[kMaxBlocks], o_done[kMaxBlocks];
+    unsigned long long recv_full;               // merge rows from every CTA of the cluster have landed (complete_tx)
     unsigned long long anc[SS_MAX_NODES];
     float2 ml[kMaxBlocks][kBlockRows];   // (m, l) received for the rows this CTA merges: [block][src * rpc_max + lr]
     uint32_t tmem_base;
@@ -155,6 +156,22 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
+}
+// local shared memory -> shared memory of a CTA of the cluster, completing on that CTA's mbarrier
+__device__ __forceinline__ void dsmem_bulk_copy(uint32_t dst_cluster, uint32_t src_cta, uint32_t bytes, uint32_t bar_cluster) {
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_cluster), "r"(src_cta), "r"(bytes), "r"(bar_cluster) : "memory");
+}
+__device__ __forceinline__ void named_barrier(int id, int threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+__device__ __forceinline__ float2 ld_shared_v2(uint32_t addr) {
+    float2 v;
+    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+    return v;
 }
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -242,6 +259,7 @@ struct Span {
     int tmax8, gamma, n_blocks;
     int spec_end;                  // valid rows: [0, T) and [tmax8, spec_end)
     unsigned valid_blocks;         // bit b set: row block b holds a valid row
+    bool pingpong;                 // one row block served by two warpgroups that take alternate tiles
 
     __device__ __forceinline__ bool is_cache(int j) const { return j < n_cache_tiles; }
     __device__ __forceinline__ int first_key(int j) const {
@@ -252,6 +270,7 @@ struct Span {
     }
     // bit b set: row block b holds a row that can see a key of tile j
     __device__ __forceinline__ unsigned active_mask(int j) const {
+        if (pingpong) return 1u << (j & 1);
         if (j < n_cache_tiles) return valid_blocks;
         // stream key s is seen by the stream rows s .. (end of its node's group)
         const int s0 = first_key(j), s_last = s0 + valid_keys(j) - 1;
@@ -316,8 +335,9 @@ struct ItemIter {
 };
 
 template <int TK>
-__device__ __forceinline__ Span<TK> make_span(const AttnArgs& a, int L, int T, int rank) {
+__device__ __forceinline__ Span<TK> make_span(const AttnArgs& a, int L, int T, int rank, bool pingpong) {
     Span<TK> s;
+    s.pingpong = pingpong;
     s.L = L; s.T = T; s.gamma = a.gamma; s.tmax8 = a.tmax8; s.n_blocks = a.n_blocks;
     s.n_stream = T * a.gamma;
     s.spec_end = a.tmax8 + s.n_stream;
@@ -426,7 +446,9 @@ __device__ __forceinline__ float chunk_exp_store(const uint32_t (&v)[64], float 
 // Kernel variants.  kMulti: up to three 128-row blocks, 64-key tiles.  kSingle: one block of 65..128
 // rows, 128-key tiles.  kDual: at most 64 rows: the block holds the rows twice, copy 0 takes keys
 // 0..63 of every 128-key tile and copy 1 keys 64..127 (P is zero in the other half), so all four
-// sub-partitions share the exponentials; the two copies are merged like two more split-KV partials.
+// sub-partitions share the exponentials; and two warpgroups, each with its own accumulator, take
+// alternate tiles, so one tile's softmax overlaps the other's MMAs.  The four partials a row then has
+// inside the CTA are combined before the cluster-wide merge.
 enum Mode { kMulti = 0, kSingle = 1, kDual = 2 };
 
 template <int HD, int MODE>
@@ -440,8 +462,10 @@ struct Geo {
     static constexpr uint32_t kIdescS = idesc_bf16(TK, false);
     static constexpr uint32_t kIdescPV = idesc_bf16(HD, true);
     static constexpr int kOCols = 128;                            // TMEM columns reserved per block accumulator
-    static constexpr int kThreads = kAuxThreads + (MODE == kMulti ? kMaxBlocks : 1) * kBlockRows;
+    static constexpr int kWGs = MODE == kMulti ? kMaxBlocks : (MODE == kDual ? 2 : 1);   // softmax warpgroups
+    static constexpr int kThreads = kAuxThreads + kWGs * kBlockRows;
     static constexpr int kCopies = MODE == kDual ? 2 : 1;
+    static constexpr int kRowBytes = kMergePitch * 4;             // one merge row: O, then (m, l)
     static constexpr int kChunks = MODE == kSingle ? 2 : 1;       // 64-key chunks of a tile one thread handles
 };
 
@@ -487,11 +511,16 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t q_rows = a.tmax8 + a.spec_rows;                      // rows of the head's query tile
     const uint32_t q_smem_rows = MODE == kDual ? kBlockRows : q_rows;   // kDual: second copy at row 64
-    const uint32_t p_rows = MODE == kMulti || MODE == kDual ? kBlockRows : q_rows;
-    const uint32_t p_bytes = (TK / 64) * p_rows * 128u;                 // one block's P tile
+    // P of one warpgroup, 128 B rows of 64 keys (swizzled).  kMulti / kSingle: [key half][p_rows].
+    // kDual: [copy-0 rows 0..63 | 64 zero rows | copy-1 rows 0..63]; the MMA reads keys 0..63 from the
+    // first 128 rows and keys 64..127 from the last 128 rows, so each copy's other half is zero.
+    const uint32_t p_rows = MODE == kMulti ? kBlockRows : q_rows;
+    const uint32_t p_half = MODE == kDual ? 64u * 128u : p_rows * 128u;    // byte offset of the second key half
+    const uint32_t p_bytes = MODE == kDual ? 3u * 64u * 128u : (TK / 64) * p_rows * 128u;
+    const int n_acc = MODE == kDual ? 2 : n_blocks;                        // accumulators = warpgroups in use
     const uint32_t q_base = base;                                       // [half][q_smem_rows][128 B]
-    const uint32_t p_base = q_base + G::kHalves * q_smem_rows * 128u;   // [block][key half][p_rows][128 B]
-    const uint32_t k_base = p_base + n_blocks * p_bytes;                // [slot][half][TK][128 B]
+    const uint32_t p_base = q_base + G::kHalves * q_smem_rows * 128u;   // [warpgroup][p_bytes]
+    const uint32_t k_base = p_base + n_acc * p_bytes;                   // [slot][half][TK][128 B]
     const uint32_t v_base = k_base + nk * G::kSlotBytes;                // [slot][half][TK][128 B]
     const uint32_t merge_base = base;                                   // aliases everything above, after the main loop
     const long long spec_row0 = static_cast<long long>(b) * a.max_nodes * a.gamma;   // first stream row of the sequence
@@ -513,6 +542,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             for (int k = 0; k < kMaxBlocks; ++k) mbar_init(smem_u32(&c.s_full[k][s]), 1);
         }
         for (int s = 0; s < kMaxBlocks; ++s) { mbar_init(smem_u32(&c.p_full[s]), kBlockRows); mbar_init(smem_u32(&c.o_done[s]), 1); }
+        mbar_init(smem_u32(&c.recv_full), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -550,7 +580,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     }
     if (tid >= kAuxThreads && tid < kAuxThreads + SS_MAX_NODES) c.anc[tid - kAuxThreads] = a.trees[b].anc_mask[tid - kAuxThreads];
 
-    const Span<TK> sp = make_span<TK>(a, L, T, static_cast<int>(rank));
+    const Span<TK> sp = make_span<TK>(a, L, T, static_cast<int>(rank), MODE == kDual);
 
     // K tile j / V tile j of the span -> ring slot st (thread 0 only)
     auto load_k = [&](int j, int st) {
@@ -580,19 +610,19 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     if (tid == 0) {
         for (int j = 0; j < n_early; ++j) { load_k(j, j); load_v(j, j); }
     }
-    // kDual: each thread's "other" key half of P stays zero for the whole kernel
+    // kDual: the 64 zero rows in the middle of each warpgroup's P stay zero for the whole kernel
     if (MODE == kDual && tid >= kAuxThreads) {
-        const int r = tid - kAuxThreads;
-        const uint32_t dst = p_base + (1 - (r >> 6)) * (p_rows * 128u) + r * 128u;
+        const int r = tid - kAuxThreads;                                  // 256 threads, 64 B each per warpgroup
+        const uint32_t dst = p_base + (r >> 7) * p_bytes + 64u * 128u + (r & 127) * 64u;
         #pragma unroll
-        for (int i = 0; i < 8; ++i) asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst + i * 16), "r"(0u) : "memory");
+        for (int i = 0; i < 4; ++i) st_shared_v4(dst + i * 16, 0u, 0u, 0u, 0u);
         fence_async_smem();
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = c.tmem_base;
-    const uint32_t tmem_s = tmem + n_blocks * G::kOCols;  // two S buffers of TK columns
+    const uint32_t tmem_s = tmem + n_acc * G::kOCols;     // two S buffers of TK columns
 
     // ================================= warp 0: TMA producer =====================================
     if (warp == 0) {
@@ -641,7 +671,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 }
                 if (q >= 2 && !mbar_wait(smem_u32(&c.s_free[buf]), ((q >> 1) - 1) & 1, abort_flag, a.status)) break;
                 tc_fence_after();
-                const uint32_t qa = q_base + blk * (kBlockRows * 128u);
+                const uint32_t qa = q_base + (MODE == kDual ? 0 : blk) * (kBlockRows * 128u);
                 const uint32_t ka = k_base + rk.slot * G::kSlotBytes;
                 #pragma unroll
                 for (int ks = 0; ks < G::kKSteps; ++ks) {
@@ -679,7 +709,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 const uint32_t va = v_base + rv.slot * G::kSlotBytes;
                 #pragma unroll
                 for (int ks = 0; ks < TK / 16; ++ks)
-                    tc_mma(tmem + blk * G::kOCols, desc_k_major(pa + (ks >> 2) * (p_rows * 128u) + (ks & 3) * 32u),
+                    tc_mma(tmem + blk * G::kOCols, desc_k_major(pa + (ks >> 2) * p_half + (ks & 3) * 32u),
                            desc_mn_major(va + ks * 2048u, G::kBoxBytes), G::kIdescPV, (nd > 0 || ks > 0) ? 1u : 0u);
                 tc_commit(smem_u32(&c.o_done[blk]));
                 if (it.last_of_tile()) tc_commit(smem_u32(&c.v_empty[rv.slot]));     // last block of tile j: V may go
@@ -698,14 +728,16 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     RowInfo ri;
     ri.valid = false; ri.node = 0; ri.stream = 0;
+    const int rblk = MODE == kDual ? 0 : my_blk;                              // row block (kDual: both warpgroups serve block 0)
     if (warp >= 4) {
-        ri = row_info(sp, my_blk * kBlockRows + lrow);
+        ri = row_info(sp, rblk * kBlockRows + lrow);
         const unsigned long long anc = ri.valid ? c.anc[ri.node] : 0ull;
         // a warp whose 32 rows are all padding skips the arithmetic but keeps the barrier protocol
         const bool warp_active = __any_sync(0xffffffffu, ri.valid);
         const uint32_t o_addr = tmem + lane_base + my_blk * G::kOCols;
-        const uint32_t p_row = p_base + my_blk * p_bytes + row_in_blk * 128u;
-        const bool p_row_ok = static_cast<uint32_t>(row_in_blk) < p_rows;      // rows past p_rows are padding: never stored
+        const uint32_t p_row = MODE == kDual ? p_base + my_blk * p_bytes + copy * (128u * 128u) + lrow * 128u
+                                             : p_base + my_blk * p_bytes + row_in_blk * 128u;
+        const bool p_row_ok = MODE == kDual || static_cast<uint32_t>(row_in_blk) < p_rows;   // rows past p_rows are padding: never stored
         ItemIter it = {0, 0u};
         it.begin(sp);
         int prev_tile = -1;
@@ -787,7 +819,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                         tmem_wait_ld();
                     }
                     if (p_row_ok) {
-                        const uint32_t dst = p_row + (copy + ch) * (p_rows * 128u);
+                        const uint32_t dst = p_row + ch * p_half;
                         sum += masked ? chunk_exp_store<true>(sr, a.scale_log2, m_use, vis[ch], dst, row_in_blk)
                                       : chunk_exp_store<false>(sr, a.scale_log2, m_use, 0ull, dst, row_in_blk);
                     }
@@ -857,7 +889,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 *reinterpret_cast<uint4*>(dst.o + c0 + 8) = hi;
             }
         }
-    } else {
+    } else if (MODE == kMulti) {
         // Every thread of the cluster passes both barriers, whatever happened above.
         // Barrier A: all CTAs are done with their pipelines, so shared memory can be reused.
         cluster_arrive();
@@ -868,9 +900,9 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
         uint32_t remote = 0, ml_remote = 0;
         bool sender = false;
         if (warp >= 4) {
-            const int nvr = sp.n_valid(my_blk);
+            const int nvr = sp.n_valid(rblk);
             const int rpc = (nvr + C - 1) / C;
-            vi = ri.valid ? sp.valid_index(my_blk * kBlockRows + lrow) : -1;
+            vi = ri.valid ? sp.valid_index(rblk * kBlockRows + lrow) : -1;
             sender = __any_sync(0xffffffffu, vi >= 0);
             if (vi >= 0) {
                 const uint32_t dst_rank = vi / rpc;
@@ -881,26 +913,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 ml_remote = map_to_rank(smem_u32(&c.ml[my_blk][src * rpc_max + lr]), dst_rank);
             }
         }
-        if (MODE != kMulti) {
-            // 256-thread variants have the registers to fetch the whole accumulator row while the barrier completes
-            uint32_t orr[HD];
-            if (sender) {
-                if (has_acc) {
-                    #pragma unroll
-                    for (int c0 = 0; c0 < HD; c0 += 16) tmem_ld16<0>(o_addr + c0, *reinterpret_cast<uint32_t(*)[16]>(&orr[c0]));
-                    tmem_wait_ld();
-                } else {
-                    #pragma unroll
-                    for (int i = 0; i < HD; ++i) orr[i] = 0u;
-                }
-            }
-            cluster_wait();
-            if (vi >= 0) {
-                #pragma unroll
-                for (int i = 0; i < HD; i += 4) st_cluster_v4(remote + i * 4u, orr[i], orr[i + 1], orr[i + 2], orr[i + 3]);
-                st_cluster_v2(ml_remote, m_run, l_run);
-            }
-        } else {
+        {
             cluster_wait();
             if (sender) {
                 #pragma unroll
@@ -921,14 +934,14 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
         cluster_arrive();
         cluster_wait();
         if (warp >= 4 && !skip) {
-            const int nvr = sp.n_valid(my_blk);
+            const int nvr = sp.n_valid(rblk);
             const int rpc = (nvr + C - 1) / C;
             const int wq = warp & 3;
             // one warp per row, one lane per four columns
             for (int lr = wq; lr < rpc; lr += 4) {
                 const int v = static_cast<int>(rank) * rpc + lr;
                 if (v >= nvr) break;
-                const RowInfo r = row_info(sp, sp.row_of(my_blk, v));
+                const RowInfo r = row_info(sp, sp.row_of(rblk, v));
                 float mx = -INFINITY;
                 for (int s = 0; s < n_src; ++s) mx = fmaxf(mx, c.ml[my_blk][s * rpc_max + lr].x);
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -953,6 +966,147 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 if (dst.lse && lane == 0) *dst.lse = (mx + log2f(l)) * 0.6931471805599453f;
             }
         }
+    } else {
+        // ---- kSingle / kDual: one row block.  Rows travel as (O[HD], m, l) records of kRowBytes. ----
+        constexpr uint32_t RB = G::kRowBytes;
+        const int nvr = sp.n_valid(0);
+        const int rpc = (nvr + C - 1) / C;                                     // rows merged per CTA
+        const int my_rows = max(0, min(rpc, nvr - static_cast<int>(rank) * rpc));
+        // staging in the shared memory the pipeline no longer needs (this CTA's MMAs are complete)
+        const uint32_t x_base = merge_base;                                    // kDual: [3 partials][64 rows]
+        const uint32_t y_base = merge_base + (MODE == kDual ? 192u : 0u) * RB; // rows to ship, in valid-row order
+        const uint32_t r_base = merge_base + (MODE == kDual ? 256u : 128u) * RB;   // received: [source CTA][rpc rows]
+        const uint32_t recv_bar = smem_u32(&c.recv_full);
+        if (tid == kAuxThreads) mbar_expect_tx(recv_bar, static_cast<uint32_t>(C * my_rows) * RB);
+        if (warp >= 4) {
+            // the staging areas overlap the query tile and the other warpgroup's P and K/V slots: the query
+            // copy must have landed and every MMA of the CTA must be complete before they are written
+            mbar_wait_warp(smem_u32(&c.q_full), 0, abort_flag, a.status);
+            if (MODE == kDual) named_barrier(2, G::kWGs * kBlockRows);
+            const int vi = ri.valid ? sp.valid_index(lrow) : -1;
+            const bool any_valid = __any_sync(0xffffffffu, vi >= 0);
+            const int pidx = my_blk * 2 + copy;                                // partial of the row inside this CTA
+            if (MODE == kDual && pidx != 0) {
+                // partials 1..3 go to X; partial 0's thread owns the row
+                const uint32_t xrow = x_base + static_cast<uint32_t>((pidx - 1) * 64 + lrow) * RB;
+                if (any_valid) {
+                    #pragma unroll
+                    for (int c0 = 0; c0 < HD; c0 += 16) {
+                        uint32_t orr[16];
+                        if (has_acc) { tmem_ld16<0>(o_addr + c0, orr); tmem_wait_ld(); }
+                        else { for (int i = 0; i < 16; ++i) orr[i] = 0u; }
+                        if (vi >= 0) {
+                            #pragma unroll
+                            for (int i = 0; i < 16; i += 4) st_shared_v4(xrow + (c0 + i) * 4u, orr[i], orr[i + 1], orr[i + 2], orr[i + 3]);
+                        }
+                    }
+                    if (vi >= 0) st_shared_v4(xrow + HD * 4u, __float_as_uint(m_run), __float_as_uint(l_run), 0u, 0u);
+                }
+            }
+            if (MODE == kDual) named_barrier(1, G::kWGs * kBlockRows);
+            if ((MODE != kDual || pidx == 0) && any_valid) {
+                // weights of the partials this thread combines
+                float w[4] = {1.f, 0.f, 0.f, 0.f};
+                float m_out = m_run, l_out = l_run;
+                if (MODE == kDual && vi >= 0) {
+                    float mp[4], lp[4];
+                    mp[0] = m_run; lp[0] = l_run;
+                    #pragma unroll
+                    for (int k = 1; k < 4; ++k) {
+                        const float2 t = ld_shared_v2(x_base + static_cast<uint32_t>((k - 1) * 64 + lrow) * RB + HD * 4u);
+                        mp[k] = t.x; lp[k] = t.y;
+                    }
+                    m_out = fmaxf(fmaxf(mp[0], mp[1]), fmaxf(mp[2], mp[3]));
+                    l_out = 0.f;
+                    #pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        w[k] = mp[k] == -INFINITY ? 0.f : exp2f(mp[k] - m_out);
+                        l_out += w[k] * lp[k];
+                    }
+                }
+                const uint32_t yrow = y_base + static_cast<uint32_t>(vi >= 0 ? vi : 0) * RB;
+                #pragma unroll
+                for (int c0 = 0; c0 < HD; c0 += 16) {
+                    uint32_t orr[16];
+                    if (has_acc) { tmem_ld16<0>(o_addr + c0, orr); tmem_wait_ld(); }
+                    else { for (int i = 0; i < 16; ++i) orr[i] = 0u; }
+                    if (vi >= 0) {
+                        #pragma unroll
+                        for (int i = 0; i < 16; i += 4) {
+                            float4 acc = make_float4(__uint_as_float(orr[i]) * w[0], __uint_as_float(orr[i + 1]) * w[0],
+                                                     __uint_as_float(orr[i + 2]) * w[0], __uint_as_float(orr[i + 3]) * w[0]);
+                            if (MODE == kDual) {
+                                #pragma unroll
+                                for (int k = 1; k < 4; ++k) {
+                                    const float4 t = ld_shared_v4(x_base + static_cast<uint32_t>((k - 1) * 64 + lrow) * RB + (c0 + i) * 4u);
+                                    acc.x += w[k] * t.x; acc.y += w[k] * t.y; acc.z += w[k] * t.z; acc.w += w[k] * t.w;
+                                }
+                            }
+                            st_shared_v4(yrow + (c0 + i) * 4u, __float_as_uint(acc.x), __float_as_uint(acc.y),
+                                         __float_as_uint(acc.z), __float_as_uint(acc.w));
+                        }
+                    }
+                }
+                if (vi >= 0) st_shared_v4(yrow + HD * 4u, __float_as_uint(m_out), __float_as_uint(l_out), 0u, 0u);
+            }
+            fence_async_smem();                          // the rows are read by the bulk-copy engine
+        }
+        // Barrier A (every thread of the cluster, whatever happened above): all CTAs are done with their
+        // pipelines and have staged their rows, so the receive areas can be written.
+        cluster_arrive();
+        cluster_wait();
+        if (tid == kAuxThreads) {
+            for (int d = 0; d < C; ++d) {
+                const int rows_d = max(0, min(rpc, nvr - d * rpc));
+                if (rows_d > 0)
+                    dsmem_bulk_copy(map_to_rank(r_base + static_cast<uint32_t>(rank * rpc) * RB, d), y_base + static_cast<uint32_t>(d * rpc) * RB,
+                                    static_cast<uint32_t>(rows_d) * RB, map_to_rank(recv_bar, d));
+            }
+        }
+        if (warp >= 4 && !skip && my_rows > 0) {
+            // the rows this CTA merges have arrived from every CTA of the cluster (complete_tx on recv_full)
+            if (mbar_wait_warp(recv_bar, 0, abort_flag, a.status)) {
+                // one warp per row, one lane per four columns
+                for (int lr = warp - 4; lr < my_rows; lr += G::kWGs * 4) {
+                    const RowInfo r = row_info(sp, sp.row_of(0, static_cast<int>(rank) * rpc + lr));
+                    float ms[8], wl[8];
+                    float mx = -INFINITY;
+                    #pragma unroll
+                    for (int s = 0; s < 8; ++s) {
+                        if (s < C) {
+                            const float2 t = ld_shared_v2(r_base + static_cast<uint32_t>(s * rpc + lr) * RB + HD * 4u);
+                            ms[s] = t.x; wl[s] = t.y;
+                            mx = fmaxf(mx, t.x);
+                        }
+                    }
+                    float l = 0.f;
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    #pragma unroll
+                    for (int s = 0; s < 8; ++s) {
+                        if (s < C) {
+                            const float w = ms[s] == -INFINITY ? 0.f : exp2f(ms[s] - mx);
+                            l += w * wl[s];
+                            if (lane * 4 < HD) {
+                                const float4 t = ld_shared_v4(r_base + static_cast<uint32_t>(s * rpc + lr) * RB + lane * 16u);
+                                acc.x += w * t.x; acc.y += w * t.y; acc.z += w * t.z; acc.w += w * t.w;
+                            }
+                        }
+                    }
+                    const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, r);
+                    const float inv = 1.f / l;
+                    if (lane * 4 < HD) {
+                        uint2 o;
+                        o.x = pack_bf16(acc.x * inv, acc.y * inv);
+                        o.y = pack_bf16(acc.z * inv, acc.w * inv);
+                        *reinterpret_cast<uint2*>(dst.o + lane * 4) = o;
+                    }
+                    if (dst.lse && lane == 0) *dst.lse = (mx + log2f(l)) * 0.6931471805599453f;
+                }
+            }
+        }
+        // nobody leaves while a copy into or out of its shared memory may still be in flight
+        cluster_arrive();
+        cluster_wait();
     }
 
     // ---- release TMEM ---------------------------------------------------------------------------
@@ -1015,16 +1169,17 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     plan->n_blocks = (q_rows + kBlockRows - 1) / kBlockRows;
     plan->mode = plan->n_blocks > 1 ? kMulti : (q_rows <= 64 ? kDual : kSingle);
     plan->tile_keys = plan->mode == kMulti ? 64 : 128;
-    plan->threads = kAuxThreads + (plan->mode == kMulti ? kMaxBlocks : 1) * kBlockRows;
+    plan->threads = kAuxThreads + (plan->mode == kMulti ? kMaxBlocks : (plan->mode == kDual ? 2 : 1)) * kBlockRows;
     // cluster size: the largest power of two that still fits the grid on the SMs in one wave
     const long long pairs = static_cast<long long>(p.batch) * p.n_heads;
     int c = 1;
     while (c < 8 && pairs * (c * 2) <= sm_count()) c *= 2;
     plan->cluster = c;
-    const int p_rows = plan->mode == kSingle ? q_rows : kBlockRows;
     const int q_smem_rows = plan->mode == kDual ? kBlockRows : q_rows;
-    const size_t qp = static_cast<size_t>(halves) * q_smem_rows * 128 +
-                      static_cast<size_t>(plan->n_blocks) * (plan->tile_keys / 64) * p_rows * 128;
+    const size_t p_total = plan->mode == kDual ? static_cast<size_t>(2) * 3 * 64 * 128                 // two warpgroups
+                         : plan->mode == kSingle ? static_cast<size_t>(2) * q_rows * 128               // two key halves
+                                                 : static_cast<size_t>(plan->n_blocks) * kBlockRows * 128;
+    const size_t qp = static_cast<size_t>(halves) * q_smem_rows * 128 + p_total;
     const size_t slot = static_cast<size_t>(halves) * plan->tile_keys * 128;
     // the MMAs of the last block read up to 128 rows past the start of their block: keep that inside the allocation
     const size_t overhang = static_cast<size_t>(kBlockRows) * 128;
@@ -1035,8 +1190,11 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     plan->n_vslots = slots - plan->n_kslots > kMaxSlots ? kMaxSlots : slots - plan->n_kslots;
     size_t bytes = qp + static_cast<size_t>(plan->n_kslots + plan->n_vslots) * slot;
     if (bytes < qp + overhang) bytes = qp + overhang;
-    const size_t merge = static_cast<size_t>(plan->n_blocks) * kBlockRows * (p.head_dim + 4) * 4;
-    if (c > 1 && merge > bytes) bytes = merge;
+    // rows of (head_dim + 4) floats staged for the merge once the pipeline is done
+    const size_t merge_rows = plan->mode == kMulti ? static_cast<size_t>(plan->n_blocks) * kBlockRows
+                            : plan->mode == kSingle ? 128 + 128 + 8 : 256 + 64 + 8;
+    const size_t merge = merge_rows * (p.head_dim + 4) * 4;
+    if ((c > 1 || plan->mode == kDual) && merge > bytes) bytes = merge;
     plan->smem = bytes + 1024;
     return plan->smem <= static_cast<size_t>(kMaxDynSmem);
 }
