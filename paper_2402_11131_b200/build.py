@@ -10,11 +10,12 @@ import sys
 PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
-LIB = os.path.join(PKG, "libss_msa.so")
-OBJ = os.path.join(PKG, "_build")
+TRACE = bool(os.environ.get("SS_TRACE"))       # developer build with in-kernel timestamps
+LIB = os.path.join(PKG, "libss_msa_trace.so" if TRACE else "libss_msa.so")
+OBJ = os.path.join(PKG, "_build_trace" if TRACE else "_build")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xcompiler", "-fPIC", "--use_fast_math", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
+              "-Xcompiler", "-fPIC", "--use_fast_math", "-I", os.path.join(ROOT, "include"), "-I", CSRC] + (["-DSS_TRACE"] if TRACE else [])
 
 
 def nvcc() -> str:

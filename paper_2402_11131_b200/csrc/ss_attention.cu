@@ -33,6 +33,19 @@
 
 namespace ss {
 
+// Developer build (-DSS_TRACE): per-role clock64 timestamps of the first CTAs, read back with
+// ss_trace_read.  Compiled out of the product library.
+#ifdef SS_TRACE
+constexpr int kTraceCtas = 16, kTraceRoles = 6, kTraceSlots = 160;
+__device__ long long g_trace[kTraceCtas][kTraceRoles][kTraceSlots];
+#define SS_TR(role, slot)                                                                                   \
+    do {                                                                                                    \
+        if (blockIdx.x < ss::kTraceCtas && (slot) < ss::kTraceSlots) ss::g_trace[blockIdx.x][role][slot] = clock64(); \
+    } while (0)
+#else
+#define SS_TR(role, slot) do { } while (0)
+#endif
+
 constexpr int kUnit = 16;            // split granularity (keys)
 constexpr int kBlockRows = 128;      // query rows per block (M of both MMAs)
 constexpr int kMaxBlocks = 3;        // 64 main rows + 256 stream rows = 320 rows at most
@@ -505,6 +518,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     const int n_blocks = a.n_blocks, nk = a.n_kslots, nv_slots = a.n_vslots;
     volatile int* abort_flag = &c.abort;
 
+    if (tid == 0) SS_TR(0, 0);
     // ---- shared-memory carve-up (1024-byte aligned: swizzle atoms) ----------------------------
     // Q and P keep only the rows that exist; an MMA that reads the rows of a 128-row block past them
     // picks up whatever follows in shared memory, which only ever reaches padding rows of S and O.
@@ -528,13 +542,18 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     // ---- prologue ---------------------------------------------------------------------------------
     // Everything up to the dependency wait touches no global memory, so under programmatic dependent
     // launch it overlaps the tail of the previous kernel in the stream.
-    if (tid == 0) {                                       // the barriers TMA completes on
+    if (tid == 0) {                                       // Q / K producer: the barriers its copies complete on
         mbar_init(smem_u32(&c.q_full), 1);
-        for (int s = 0; s < kMaxSlots; ++s) { mbar_init(smem_u32(&c.k_full[s]), 1); mbar_init(smem_u32(&c.v_full[s]), 1); }
+        for (int s = 0; s < kMaxSlots; ++s) mbar_init(smem_u32(&c.k_full[s]), 1);
         c.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        tma_prefetch_desc(&a.tm_qm); tma_prefetch_desc(&a.tm_k); tma_prefetch_desc(&a.tm_v);
-        if (a.gamma > 0) { tma_prefetch_desc(&a.tm_qs); tma_prefetch_desc(&a.tm_ks); tma_prefetch_desc(&a.tm_vs); }
+        tma_prefetch_desc(&a.tm_qm); tma_prefetch_desc(&a.tm_k);
+        if (a.gamma > 0) { tma_prefetch_desc(&a.tm_qs); tma_prefetch_desc(&a.tm_ks); }
+    } else if (tid == 96) {                               // V producer
+        for (int s = 0; s < kMaxSlots; ++s) mbar_init(smem_u32(&c.v_full[s]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        tma_prefetch_desc(&a.tm_v);
+        if (a.gamma > 0) tma_prefetch_desc(&a.tm_vs);
     } else if (tid == 64) {                               // every other barrier (first used after the CTA-wide sync)
         for (int s = 0; s < kMaxSlots; ++s) { mbar_init(smem_u32(&c.k_empty[s]), 1); mbar_init(smem_u32(&c.v_empty[s]), 1); }
         for (int s = 0; s < 2; ++s) {
@@ -545,8 +564,10 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
         mbar_init(smem_u32(&c.recv_full), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (tid == 0) SS_TR(0, 1);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (tid == 0) SS_TR(0, 2);
 
     if (tid == 0) {
         // the queries depend on nothing but (sequence, head): request them before the lengths are known
@@ -562,6 +583,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             }
         }
     }
+    if (tid == 0) SS_TR(0, 3);
     // per-sequence scalars (every thread reads them)
     int L = a.kv_len[b];
     int T = min(max(a.trees[b].n_nodes, 0), a.max_nodes);
@@ -582,7 +604,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
 
     const Span<TK> sp = make_span<TK>(a, L, T, static_cast<int>(rank), MODE == kDual);
 
-    // K tile j / V tile j of the span -> ring slot st (thread 0 only)
+    // K tile j / V tile j of the span -> ring slot st (K: thread 0, V: thread 96)
     auto load_k = [&](int j, int st) {
         const uint32_t bar = smem_u32(&c.k_full[st]);
         mbar_expect_tx(bar, G::kSlotBytes);
@@ -605,11 +627,15 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             else tma_load_3d(dst + hh * G::kBoxBytes, &a.tm_vs, hh * 64, h, static_cast<int>(spec_row0 + x), bar);
         }
     };
-    // the producer starts before the CTA-wide synchronisation: the first tiles need no hand-back
-    const int n_early = min(sp.n_tiles, min(nk, nv_slots));
+    if (tid == 0) SS_TR(0, 4);
+    // the producers start before the CTA-wide synchronisation: the first tiles need no hand-back
+    const int n_early_k = min(sp.n_tiles, nk), n_early_v = min(sp.n_tiles, nv_slots);
     if (tid == 0) {
-        for (int j = 0; j < n_early; ++j) { load_k(j, j); load_v(j, j); }
+        for (int j = 0; j < n_early_k; ++j) load_k(j, j);
+    } else if (tid == 96) {
+        for (int j = 0; j < n_early_v; ++j) load_v(j, j);
     }
+    if (tid == 0) SS_TR(0, 5);
     // kDual: the 64 zero rows in the middle of each warpgroup's P stay zero for the whole kernel
     if (MODE == kDual && tid >= kAuxThreads) {
         const int r = tid - kAuxThreads;                                  // 256 threads, 64 B each per warpgroup
@@ -623,30 +649,37 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     tc_fence_after();
     const uint32_t tmem = c.tmem_base;
     const uint32_t tmem_s = tmem + n_acc * G::kOCols;     // two S buffers of TK columns
+    if (tid == 0) SS_TR(0, 6);
 
-    // ================================= warp 0: TMA producer =====================================
+    // ============================ warp 0: K producer, warp 3: V producer ==========================
+    // Two rings, two threads: a K slot comes back as soon as S is queued, a V slot only after P V, and
+    // neither request waits behind the other.
     if (warp == 0) {
-        if (lane == 0 && sp.n_tiles > n_early) {
-            int jk = n_early, jv = n_early;               // next K tile / V tile to request
-            Ring rk, rv;                                  // their ring positions
-            rk.start(); rv.start();
-            for (int i = 0; i < n_early; ++i) { rk.advance(nk); rv.advance(nv_slots); }
+        if (lane == 0 && sp.n_tiles > n_early_k) {
+            Ring rk;
+            rk.start();
+            for (int i = 0; i < n_early_k; ++i) rk.advance(nk);
             bool ok = true;
-            while (ok && (jk < sp.n_tiles || jv < sp.n_tiles)) {
-                // K slots come back early (after S), so K runs ahead of V by at most one ring
-                if (jk < sp.n_tiles && (jk <= jv || jv >= sp.n_tiles)) {
-                    ok = rk.round == 0 || mbar_wait(smem_u32(&c.k_empty[rk.slot]), (rk.round - 1) & 1, abort_flag, a.status);
-                    if (ok) { load_k(jk++, rk.slot); rk.advance(nk); }
-                } else {
-                    ok = rv.round == 0 || mbar_wait(smem_u32(&c.v_empty[rv.slot]), (rv.round - 1) & 1, abort_flag, a.status);
-                    if (ok) { load_v(jv++, rv.slot); rv.advance(nv_slots); }
-                }
+            for (int j = n_early_k; ok && j < sp.n_tiles; ++j) {
+                ok = mbar_wait(smem_u32(&c.k_empty[rk.slot]), (rk.round - 1) & 1, abort_flag, a.status);
+                SS_TR(0, 8 + 2 * j);
+                if (ok) { load_k(j, rk.slot); rk.advance(nk); }
             }
-            if (!ok) {
-                // gave up: let the copies already in flight land before shared memory is reused or released
-                for (int s = 0; s < nk; ++s) mbar_drain(smem_u32(&c.k_full[s]), (s < rk.slot ? rk.round : rk.round - 1) & 1);
-                for (int s = 0; s < nv_slots; ++s) mbar_drain(smem_u32(&c.v_full[s]), (s < rv.slot ? rv.round : rv.round - 1) & 1);
+            // gave up: let the copies already in flight land before shared memory is reused or released
+            if (!ok) for (int s = 0; s < nk; ++s) mbar_drain(smem_u32(&c.k_full[s]), (s < rk.slot ? rk.round : rk.round - 1) & 1);
+        }
+    } else if (warp == 3) {
+        if (lane == 0 && sp.n_tiles > n_early_v) {
+            Ring rv;
+            rv.start();
+            for (int i = 0; i < n_early_v; ++i) rv.advance(nv_slots);
+            bool ok = true;
+            for (int j = n_early_v; ok && j < sp.n_tiles; ++j) {
+                ok = mbar_wait(smem_u32(&c.v_empty[rv.slot]), (rv.round - 1) & 1, abort_flag, a.status);
+                SS_TR(0, 9 + 2 * j);
+                if (ok) { load_v(j, rv.slot); rv.advance(nv_slots); }
             }
+            if (!ok) for (int s = 0; s < nv_slots; ++s) mbar_drain(smem_u32(&c.v_full[s]), (s < rv.slot ? rv.round : rv.round - 1) & 1);
         }
     }
     // ============================ warp 1: issues S = Q K^T =========================================
@@ -655,6 +688,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             // the query tile is always requested, so it is always awaited (shared memory is reused later)
             bool ok = mbar_wait(smem_u32(&c.q_full), 0, abort_flag, a.status);
             if (!ok) mbar_drain(smem_u32(&c.q_full), 0);
+            SS_TR(1, 0);
             ItemIter it = {0, 0u};
             it.begin(sp);
             Ring rk;
@@ -669,7 +703,9 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                     if (!mbar_wait(smem_u32(&c.k_full[rk.slot]), rk.round & 1, abort_flag, a.status)) break;
                     k_seen = true;
                 }
+                SS_TR(1, 8 + 4 * q);
                 if (q >= 2 && !mbar_wait(smem_u32(&c.s_free[buf]), ((q >> 1) - 1) & 1, abort_flag, a.status)) break;
+                SS_TR(1, 9 + 4 * q);
                 tc_fence_after();
                 const uint32_t qa = q_base + (MODE == kDual ? 0 : blk) * (kBlockRows * 128u);
                 const uint32_t ka = k_base + rk.slot * G::kSlotBytes;
@@ -679,8 +715,10 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                     tc_mma(tmem_s + buf * TK, desc_k_major(qa + hh * q_smem_rows * 128u + off),
                            desc_k_major(ka + hh * G::kBoxBytes + off), G::kIdescS, ks > 0);
                 }
+                SS_TR(1, 10 + 4 * q);
                 tc_commit(smem_u32(&c.s_full[blk][buf]));
                 if (it.last_of_tile()) tc_commit(smem_u32(&c.k_empty[rk.slot]));     // every S of tile j is queued: K may go
+                SS_TR(1, 11 + 4 * q);
             }
         }
     }
@@ -695,7 +733,8 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             int v_tile = it.j;
             for (int i = 0; i < v_tile; ++i) rv.advance(nv_slots);
             bool v_seen = false;
-            for (; !it.done(sp); it.next(sp)) {
+            int tq = 0;
+            for (; !it.done(sp); it.next(sp), ++tq) {
                 const int j = it.j, blk = it.blk();
                 const int nd = blk == 0 ? n_done0 : (blk == 1 ? n_done1 : n_done2);
                 while (v_tile < j) { rv.advance(nv_slots); ++v_tile; v_seen = false; }
@@ -703,7 +742,9 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                     if (!mbar_wait(smem_u32(&c.v_full[rv.slot]), rv.round & 1, abort_flag, a.status)) break;
                     v_seen = true;
                 }
+                SS_TR(2, 8 + 4 * tq);
                 if (!mbar_wait(smem_u32(&c.p_full[blk]), nd & 1, abort_flag, a.status)) break;
+                SS_TR(2, 9 + 4 * tq);
                 tc_fence_after();
                 const uint32_t pa = p_base + blk * p_bytes;
                 const uint32_t va = v_base + rv.slot * G::kSlotBytes;
@@ -711,9 +752,11 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 for (int ks = 0; ks < TK / 16; ++ks)
                     tc_mma(tmem + blk * G::kOCols, desc_k_major(pa + (ks >> 2) * p_half + (ks & 3) * 32u),
                            desc_mn_major(va + ks * 2048u, G::kBoxBytes), G::kIdescPV, (nd > 0 || ks > 0) ? 1u : 0u);
+                SS_TR(2, 10 + 4 * tq);
                 tc_commit(smem_u32(&c.o_done[blk]));
                 if (it.last_of_tile()) tc_commit(smem_u32(&c.v_empty[rv.slot]));     // last block of tile j: V may go
                 if (blk == 0) ++n_done0; else if (blk == 1) ++n_done1; else ++n_done2;
+                SS_TR(2, 11 + 4 * tq);
             }
         }
     }
@@ -755,6 +798,9 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             const int buf = q & 1;
             if (!mbar_wait_warp(smem_u32(&c.s_full[my_blk][buf]), (buf ? n_use1 : n_use0) & 1, abort_flag, a.status)) break;
             if (buf) ++n_use1; else ++n_use0;
+            [[maybe_unused]] const int trole = 3 + my_blk;
+            [[maybe_unused]] const bool tr_on = row_in_blk == 0 && my_blk < 2;
+            if (tr_on) SS_TR(trole, 8 + 6 * n_own);
             tc_fence_after();
             const uint32_t s_addr = tmem_s + lane_base + buf * TK;
             const int x = sp.first_key(j), nvk = sp.valid_keys(j);
@@ -785,6 +831,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                     l_run *= corr;
                 }
             }
+            if (tr_on) SS_TR(trole, 9 + 6 * n_own);
             if (G::kChunks == 1) {                      // the scores stay in registers: S can be overwritten
                 tc_fence_before();
                 __syncwarp();
@@ -796,6 +843,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 if (!mbar_wait_warp(smem_u32(&c.o_done[my_blk]), (n_own - 1) & 1, abort_flag, a.status)) break;
                 tc_fence_after();
             }
+            if (tr_on) SS_TR(trole, 10 + 6 * n_own);
             if (warp_active) {
                 if (n_own > 0 && __any_sync(0xffffffffu, need)) {
                     #pragma unroll
@@ -826,6 +874,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 }
                 l_run += sum;
             }
+            if (tr_on) SS_TR(trole, 11 + 6 * n_own);
             if (G::kChunks > 1) {                       // both passes have read S
                 tc_fence_before();
                 __syncwarp();
@@ -846,9 +895,11 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                     asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
                 }
             }
+            if (tr_on) SS_TR(trole, 12 + 6 * n_own);
             fence_async_smem();
             tc_fence_before();
             mbar_arrive(smem_u32(&c.p_full[my_blk]));
+            if (tr_on) SS_TR(trole, 13 + 6 * n_own);
             ++n_own;
         }
         // the block's last PV must have landed in TMEM before the accumulator is read
@@ -857,6 +908,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             tc_fence_after();
         }
     }
+    if (tid == kAuxThreads) SS_TR(5, 0);
     __syncwarp();     // the single-lane roles of warps 0..2 rejoin their warps
 
     // ======================================== epilogue ==========================================
@@ -969,13 +1021,14 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     } else {
         // ---- kSingle / kDual: one row block.  Rows travel as (O[HD], m, l) records of kRowBytes. ----
         constexpr uint32_t RB = G::kRowBytes;
+        constexpr int QW = HD / 4;                                             // columns one thread combines (kDual)
         const int nvr = sp.n_valid(0);
         const int rpc = (nvr + C - 1) / C;                                     // rows merged per CTA
         const int my_rows = max(0, min(rpc, nvr - static_cast<int>(rank) * rpc));
-        // staging in the shared memory the pipeline no longer needs (this CTA's MMAs are complete)
-        const uint32_t x_base = merge_base;                                    // kDual: [3 partials][64 rows]
-        const uint32_t y_base = merge_base + (MODE == kDual ? 192u : 0u) * RB; // rows to ship, in valid-row order
-        const uint32_t r_base = merge_base + (MODE == kDual ? 256u : 128u) * RB;   // received: [source CTA][rpc rows]
+        // staging in the shared memory the pipeline no longer needs
+        const uint32_t x_base = merge_base;                                    // kDual: [4 partials][64 rows]
+        const uint32_t y_base = merge_base + (MODE == kDual ? 256u : 0u) * RB; // rows to ship, in valid-row order
+        const uint32_t r_base = merge_base + (MODE == kDual ? 320u : 128u) * RB;   // received: [source CTA][rpc rows]
         const uint32_t recv_bar = smem_u32(&c.recv_full);
         if (tid == kAuxThreads) mbar_expect_tx(recv_bar, static_cast<uint32_t>(C * my_rows) * RB);
         if (warp >= 4) {
@@ -983,48 +1036,19 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             // copy must have landed and every MMA of the CTA must be complete before they are written
             mbar_wait_warp(smem_u32(&c.q_full), 0, abort_flag, a.status);
             if (MODE == kDual) named_barrier(2, G::kWGs * kBlockRows);
+        }
+        // Barrier A, arrival (every thread of the cluster, whatever happened above): this CTA's pipeline
+        // is finished, so the other CTAs may write its receive area, which its own staging never touches.
+        cluster_arrive();
+        if (warp >= 4) {
+            if (tid == kAuxThreads) SS_TR(5, 1);
             const int vi = ri.valid ? sp.valid_index(lrow) : -1;
             const bool any_valid = __any_sync(0xffffffffu, vi >= 0);
             const int pidx = my_blk * 2 + copy;                                // partial of the row inside this CTA
-            if (MODE == kDual && pidx != 0) {
-                // partials 1..3 go to X; partial 0's thread owns the row
-                const uint32_t xrow = x_base + static_cast<uint32_t>((pidx - 1) * 64 + lrow) * RB;
-                if (any_valid) {
-                    #pragma unroll
-                    for (int c0 = 0; c0 < HD; c0 += 16) {
-                        uint32_t orr[16];
-                        if (has_acc) { tmem_ld16<0>(o_addr + c0, orr); tmem_wait_ld(); }
-                        else { for (int i = 0; i < 16; ++i) orr[i] = 0u; }
-                        if (vi >= 0) {
-                            #pragma unroll
-                            for (int i = 0; i < 16; i += 4) st_shared_v4(xrow + (c0 + i) * 4u, orr[i], orr[i + 1], orr[i + 2], orr[i + 3]);
-                        }
-                    }
-                    if (vi >= 0) st_shared_v4(xrow + HD * 4u, __float_as_uint(m_run), __float_as_uint(l_run), 0u, 0u);
-                }
-            }
-            if (MODE == kDual) named_barrier(1, G::kWGs * kBlockRows);
-            if ((MODE != kDual || pidx == 0) && any_valid) {
-                // weights of the partials this thread combines
-                float w[4] = {1.f, 0.f, 0.f, 0.f};
-                float m_out = m_run, l_out = l_run;
-                if (MODE == kDual && vi >= 0) {
-                    float mp[4], lp[4];
-                    mp[0] = m_run; lp[0] = l_run;
-                    #pragma unroll
-                    for (int k = 1; k < 4; ++k) {
-                        const float2 t = ld_shared_v2(x_base + static_cast<uint32_t>((k - 1) * 64 + lrow) * RB + HD * 4u);
-                        mp[k] = t.x; lp[k] = t.y;
-                    }
-                    m_out = fmaxf(fmaxf(mp[0], mp[1]), fmaxf(mp[2], mp[3]));
-                    l_out = 0.f;
-                    #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        w[k] = mp[k] == -INFINITY ? 0.f : exp2f(mp[k] - m_out);
-                        l_out += w[k] * lp[k];
-                    }
-                }
-                const uint32_t yrow = y_base + static_cast<uint32_t>(vi >= 0 ? vi : 0) * RB;
+            // kDual: the four partials of a row go to X; kSingle: the row goes straight to Y
+            const uint32_t srow = MODE == kDual ? x_base + static_cast<uint32_t>(pidx * 64 + lrow) * RB
+                                                : y_base + static_cast<uint32_t>(vi >= 0 ? vi : 0) * RB;
+            if (any_valid) {
                 #pragma unroll
                 for (int c0 = 0; c0 < HD; c0 += 16) {
                     uint32_t orr[16];
@@ -1032,29 +1056,53 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                     else { for (int i = 0; i < 16; ++i) orr[i] = 0u; }
                     if (vi >= 0) {
                         #pragma unroll
-                        for (int i = 0; i < 16; i += 4) {
-                            float4 acc = make_float4(__uint_as_float(orr[i]) * w[0], __uint_as_float(orr[i + 1]) * w[0],
-                                                     __uint_as_float(orr[i + 2]) * w[0], __uint_as_float(orr[i + 3]) * w[0]);
-                            if (MODE == kDual) {
-                                #pragma unroll
-                                for (int k = 1; k < 4; ++k) {
-                                    const float4 t = ld_shared_v4(x_base + static_cast<uint32_t>((k - 1) * 64 + lrow) * RB + (c0 + i) * 4u);
-                                    acc.x += w[k] * t.x; acc.y += w[k] * t.y; acc.z += w[k] * t.z; acc.w += w[k] * t.w;
-                                }
-                            }
-                            st_shared_v4(yrow + (c0 + i) * 4u, __float_as_uint(acc.x), __float_as_uint(acc.y),
-                                         __float_as_uint(acc.z), __float_as_uint(acc.w));
-                        }
+                        for (int i = 0; i < 16; i += 4) st_shared_v4(srow + (c0 + i) * 4u, orr[i], orr[i + 1], orr[i + 2], orr[i + 3]);
                     }
                 }
-                if (vi >= 0) st_shared_v4(yrow + HD * 4u, __float_as_uint(m_out), __float_as_uint(l_out), 0u, 0u);
+                if (vi >= 0) st_shared_v4(srow + HD * 4u, __float_as_uint(m_run), __float_as_uint(l_run), 0u, 0u);
             }
+            if (tid == kAuxThreads) SS_TR(5, 2);
+            if (MODE == kDual) {
+                named_barrier(1, G::kWGs * kBlockRows);
+                // each of the row's four threads combines one quarter of the columns
+                if (vi >= 0) {
+                    float w[4], mp[4];
+                    float m_out = -INFINITY, l_out = 0.f;
+                    #pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const float2 t = ld_shared_v2(x_base + static_cast<uint32_t>(k * 64 + lrow) * RB + HD * 4u);
+                        mp[k] = t.x; w[k] = t.y;
+                        m_out = fmaxf(m_out, t.x);
+                    }
+                    #pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const float e = mp[k] == -INFINITY ? 0.f : exp2f(mp[k] - m_out);
+                        l_out += e * w[k];
+                        w[k] = e;
+                    }
+                    const uint32_t yrow = y_base + static_cast<uint32_t>(vi) * RB;
+                    #pragma unroll
+                    for (int i = 0; i < QW; i += 4) {
+                        const uint32_t col = static_cast<uint32_t>(pidx * QW + i) * 4u;
+                        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                        #pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const float4 t = ld_shared_v4(x_base + static_cast<uint32_t>(k * 64 + lrow) * RB + col);
+                            acc.x += w[k] * t.x; acc.y += w[k] * t.y; acc.z += w[k] * t.z; acc.w += w[k] * t.w;
+                        }
+                        st_shared_v4(yrow + col, __float_as_uint(acc.x), __float_as_uint(acc.y), __float_as_uint(acc.z), __float_as_uint(acc.w));
+                    }
+                    if (pidx == 0) st_shared_v4(yrow + HD * 4u, __float_as_uint(m_out), __float_as_uint(l_out), 0u, 0u);
+                }
+            }
+            if (tid == kAuxThreads) SS_TR(5, 3);
             fence_async_smem();                          // the rows are read by the bulk-copy engine
         }
-        // Barrier A (every thread of the cluster, whatever happened above): all CTAs are done with their
-        // pipelines and have staged their rows, so the receive areas can be written.
-        cluster_arrive();
+        // Barrier A, completion: every CTA of the cluster has finished its pipeline.  The CTA-wide named
+        // barrier orders the staged rows of all warpgroups before the one thread that ships them.
         cluster_wait();
+        if (warp >= 4) named_barrier(3, G::kWGs * kBlockRows);
+        if (tid == kAuxThreads) SS_TR(5, 4);
         if (tid == kAuxThreads) {
             for (int d = 0; d < C; ++d) {
                 const int rows_d = max(0, min(rpc, nvr - d * rpc));
@@ -1065,7 +1113,9 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
         }
         if (warp >= 4 && !skip && my_rows > 0) {
             // the rows this CTA merges have arrived from every CTA of the cluster (complete_tx on recv_full)
+            if (tid == kAuxThreads) SS_TR(5, 5);
             if (mbar_wait_warp(recv_bar, 0, abort_flag, a.status)) {
+                if (tid == kAuxThreads) SS_TR(5, 6);
                 // one warp per row, one lane per four columns
                 for (int lr = warp - 4; lr < my_rows; lr += G::kWGs * 4) {
                     const RowInfo r = row_info(sp, sp.row_of(0, static_cast<int>(rank) * rpc + lr));
@@ -1104,9 +1154,11 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 }
             }
         }
+        if (tid == kAuxThreads) SS_TR(5, 7);
         // nobody leaves while a copy into or out of its shared memory may still be in flight
         cluster_arrive();
         cluster_wait();
+        if (tid == kAuxThreads) SS_TR(5, 8);
     }
 
     // ---- release TMEM ---------------------------------------------------------------------------
@@ -1192,7 +1244,7 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     if (bytes < qp + overhang) bytes = qp + overhang;
     // rows of (head_dim + 4) floats staged for the merge once the pipeline is done
     const size_t merge_rows = plan->mode == kMulti ? static_cast<size_t>(plan->n_blocks) * kBlockRows
-                            : plan->mode == kSingle ? 128 + 128 + 8 : 256 + 64 + 8;
+                            : plan->mode == kSingle ? 128 + 128 + 8 : 256 + 64 + 64 + 8;
     const size_t merge = merge_rows * (p.head_dim + 4) * 4;
     if ((c > 1 || plan->mode == kDual) && merge > bytes) bytes = merge;
     plan->smem = bytes + 1024;
@@ -1315,3 +1367,15 @@ extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
         default: return ss::launch<128, ss::kMulti>(a, plan, pairs, s);
     }
 }
+
+#ifdef SS_TRACE
+// developer build only: copies the timestamp buffer to the host / clears it
+extern "C" int32_t ss_trace_read(long long* out) {
+    return cudaMemcpyFromSymbol(out, ss::g_trace, sizeof(ss::g_trace)) == cudaSuccess ? 0 : -1;
+}
+extern "C" int32_t ss_trace_clear() {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, ss::g_trace) != cudaSuccess) return -1;
+    return cudaMemset(p, 0, sizeof(ss::g_trace)) == cudaSuccess ? 0 : -1;
+}
+#endif
