@@ -38,6 +38,13 @@ namespace ss {
 #ifdef SS_TRACE
 constexpr int kTraceCtas = 16, kTraceRoles = 6, kTraceSlots = 160;
 __device__ long long g_trace[kTraceCtas][kTraceRoles][kTraceSlots];
+__device__ unsigned long long g_wall[8][6];      // first CTA start / last CTA end (globaltimer ns) of the last 8 launches
+__device__ unsigned long long g_key[8];           // launch identity: the output pointer
+__device__ __forceinline__ unsigned long long wall_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
 #define SS_TR(role, slot)                                                                                   \
     do {                                                                                                    \
         if (blockIdx.x < ss::kTraceCtas && (slot) < ss::kTraceSlots) ss::g_trace[blockIdx.x][role][slot] = clock64(); \
@@ -76,6 +83,8 @@ struct alignas(64) AttnArgs {
     const int* kv_capacity;
     const ss_tree_desc* trees;
     int* status;
+    int* counters;                   // [pairs] arrivals of a pair's CTAs (zero between calls)
+    float* partials;                 // [pairs][splits][rows][head_dim + 4]
 };
 
 struct Ctrl {
@@ -84,35 +93,17 @@ struct Ctrl {
     unsigned long long s_full[kMaxBlocks][2];   // per (block, S buffer): a warpgroup sees every phase of its own
     unsigned long long s_free[2];
     unsigned long long p_full[kMaxBlocks], o_done[kMaxBlocks];
-    unsigned long long recv_full;               // merge rows from every CTA of the cluster have landed (complete_tx)
     unsigned long long anc[SS_MAX_NODES];
-    float2 ml[kMaxBlocks][kBlockRows];   // (m, l) received for the rows this CTA merges: [block][src * rpc_max + lr]
     uint32_t tmem_base;
     int abort;
+    int is_last;                 // this CTA arrived last on its pair's counter
+    unsigned long long merge_full[2];   // a batch of the pair's partials has been copied into shared memory
 };
 
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ uint32_t cluster_rank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
-__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
-__device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void st_cluster_v4(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
-    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
-}
-__device__ __forceinline__ void st_cluster_v2(uint32_t addr, float x, float y) {
-    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(x), "f"(y) : "memory");
 }
 __device__ __forceinline__ float4 ld_shared_v4(uint32_t addr) {
     float4 v;
@@ -170,11 +161,6 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
 }
-// local shared memory -> shared memory of a CTA of the cluster, completing on that CTA's mbarrier
-__device__ __forceinline__ void dsmem_bulk_copy(uint32_t dst_cluster, uint32_t src_cta, uint32_t bytes, uint32_t bar_cluster) {
-    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst_cluster), "r"(src_cta), "r"(bytes), "r"(bar_cluster) : "memory");
-}
 __device__ __forceinline__ void named_barrier(int id, int threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
@@ -185,6 +171,11 @@ __device__ __forceinline__ float2 ld_shared_v2(uint32_t addr) {
     float2 v;
     asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
     return v;
+}
+// contiguous global memory -> shared memory, completing on an mbarrier of this CTA
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -512,13 +503,27 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int C = a.cluster;
-    const uint32_t rank = C > 1 ? cluster_rank() : 0u;
-    const int pair = blockIdx.x / C;
+    const uint32_t rank = blockIdx.x & (C - 1);            // C is a power of two
+    const int pair = blockIdx.x >> a.cluster_shift;
     const int b = pair / a.n_heads, h = pair - b * a.n_heads;
     const int n_blocks = a.n_blocks, nk = a.n_kslots, nv_slots = a.n_vslots;
     volatile int* abort_flag = &c.abort;
 
     if (tid == 0) SS_TR(0, 0);
+#ifdef SS_TRACE
+    __shared__ unsigned int s_launch;
+    if (tid == 0) {
+        const unsigned long long key = reinterpret_cast<unsigned long long>(a.o_main);
+        s_launch = 0;
+        for (unsigned int i = 0; i < 8; ++i) {
+            const unsigned long long old = atomicCAS(&g_key[i], 0ull, key);
+            if (old == 0ull || old == key) { s_launch = i; break; }
+        }
+        atomicMin(&g_wall[s_launch & 7][0], wall_ns());
+        atomicMax(&g_wall[s_launch & 7][2], wall_ns());      // last CTA start
+        if (blockIdx.x == 0) { g_wall[s_launch & 7][3] = wall_ns(); g_wall[s_launch & 7][4] = clock64(); }
+    }
+#endif
     // ---- shared-memory carve-up (1024-byte aligned: swizzle atoms) ----------------------------
     // Q and P keep only the rows that exist; an MMA that reads the rows of a 128-row block past them
     // picks up whatever follows in shared memory, which only ever reaches padding rows of S and O.
@@ -561,12 +566,20 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             for (int k = 0; k < kMaxBlocks; ++k) mbar_init(smem_u32(&c.s_full[k][s]), 1);
         }
         for (int s = 0; s < kMaxBlocks; ++s) { mbar_init(smem_u32(&c.p_full[s]), kBlockRows); mbar_init(smem_u32(&c.o_done[s]), 1); }
-        mbar_init(smem_u32(&c.recv_full), 1);
+        mbar_init(smem_u32(&c.merge_full[0]), 1);
+        mbar_init(smem_u32(&c.merge_full[1]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (tid == 0) SS_TR(0, 1);
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // One thread waits for the previous kernel of the stream; the others sleep on the CTA barrier (a
+    // whole parked grid polling the dependency slows the kernel it waits for).  Only then may the next
+    // kernel be scheduled: every CTA of this grid is resident and past its wait, so CTAs of a later
+    // grid can never hold an SM that this grid still needs.
+    if (tid == 0) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    }
+    __syncthreads();
     if (tid == 0) SS_TR(0, 2);
 
     if (tid == 0) {
@@ -585,10 +598,11 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     }
     if (tid == 0) SS_TR(0, 3);
     // per-sequence scalars (every thread reads them)
-    int L = a.kv_len[b];
-    int T = min(max(a.trees[b].n_nodes, 0), a.max_nodes);
-    const long long slot0 = a.kv_start[b];
-    const int cap = a.kv_capacity != nullptr ? a.kv_capacity[b] : 0x7fffffff;
+    // (read through L2: under an early launch the SM's L1 may predate the previous kernel's last writes)
+    int L = __ldcg(a.kv_len + b);
+    int T = min(max(__ldcg(&a.trees[b].n_nodes), 0), a.max_nodes);
+    const long long slot0 = __ldcg(a.kv_start + b);
+    const int cap = a.kv_capacity != nullptr ? __ldcg(a.kv_capacity + b) : 0x7fffffff;
     constexpr uint32_t kTmemCols = 512;
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&c.tmem_base)), "r"(kTmemCols) : "memory");
@@ -600,7 +614,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
         if (tid == 0) set_status(a.status, SS_ERR_CAPACITY);
         L = 0; T = 0;
     }
-    if (tid >= kAuxThreads && tid < kAuxThreads + SS_MAX_NODES) c.anc[tid - kAuxThreads] = a.trees[b].anc_mask[tid - kAuxThreads];
+    if (tid >= kAuxThreads && tid < kAuxThreads + SS_MAX_NODES) c.anc[tid - kAuxThreads] = __ldcg(&a.trees[b].anc_mask[tid - kAuxThreads]);
 
     const Span<TK> sp = make_span<TK>(a, L, T, static_cast<int>(rank), MODE == kDual);
 
@@ -912,9 +926,114 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     __syncwarp();     // the single-lane roles of warps 0..2 rejoin their warps
 
     // ======================================== epilogue ==========================================
+    // Every CTA of a split pair leaves one un-normalised partial (O, m, l) per valid row in the
+    // workspace (it stays in L2); the CTA that arrives last on the pair's counter combines them and
+    // writes the output.  Nobody waits for anybody: the other CTAs exit at once and free their SMs.
     const bool has_acc = (warp >= 4) && n_own > 0;     // otherwise the partial is (m = -inf, l = 0, O = 0)
     const uint32_t o_addr = tmem + lane_base + (warp >= 4 ? my_blk : 0) * G::kOCols;
-    if (C == 1 && MODE != kDual) {
+    constexpr int RP = G::kMergePitch;                                         // floats per partial row: O, m, l, pad
+    constexpr int QW = HD / 4;                                                 // columns one thread combines (kDual)
+    const int rows_cap = MODE == kDual ? 64 : n_blocks * kBlockRows;           // partial rows per CTA
+    float* const part_pair = a.partials + static_cast<size_t>(pair) * C * rows_cap * RP;
+    float* const part_mine = part_pair + static_cast<size_t>(rank) * rows_cap * RP;
+    const int wg_threads = G::kWGs * kBlockRows;
+    // row of the partial this thread is responsible for (block-local valid-row number), -1: none
+    const int vi = (warp >= 4 && ri.valid) ? sp.valid_index(rblk * kBlockRows + lrow) : -1;
+    const int pidx = my_blk * 2 + copy;                                        // kDual: partial of the row inside the CTA
+
+    // kDual staging area X: [source][64 rows][RP floats]; sources are the four CTA-local partials of a
+    // row, later the partials of the pair's CTAs.  A thread combines one quarter of its row's columns;
+    // with `carry` the running (m, l, acc) counts as one more source.
+    const uint32_t x_base = merge_base;
+    auto combine_x = [&](int n_src, bool carry, float& m_c, float& l_c, float4 (&acc)[QW / 4]) {
+        constexpr uint32_t RBx = RP * 4;
+        float w[4], mp[4], lp[4];
+        float m_new = carry ? m_c : -INFINITY;
+        #pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            if (k < n_src) {
+                const float2 t = ld_shared_v2(x_base + static_cast<uint32_t>(k * 64 + lrow) * RBx + HD * 4u);
+                mp[k] = t.x; lp[k] = t.y;
+                m_new = fmaxf(m_new, t.x);
+            }
+        }
+        const float wc = (carry && m_c != -INFINITY) ? exp2f(m_c - m_new) : 0.f;
+        float l_new = wc * l_c;
+        #pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            w[k] = (k < n_src && mp[k] != -INFINITY) ? exp2f(mp[k] - m_new) : 0.f;     // 0: saw no visible key
+            if (k < n_src) l_new += w[k] * lp[k];
+        }
+        #pragma unroll
+        for (int i = 0; i < QW / 4; ++i) {
+            const uint32_t col = static_cast<uint32_t>(pidx * QW + i * 4) * 4u;
+            float4 r = carry ? make_float4(acc[i].x * wc, acc[i].y * wc, acc[i].z * wc, acc[i].w * wc) : make_float4(0.f, 0.f, 0.f, 0.f);
+            #pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if (k < n_src) {
+                    const float4 t = ld_shared_v4(x_base + static_cast<uint32_t>(k * 64 + lrow) * RBx + col);
+                    r.x += w[k] * t.x; r.y += w[k] * t.y; r.z += w[k] * t.z; r.w += w[k] * t.w;
+                }
+            }
+            acc[i] = r;
+        }
+        m_c = m_new;
+        l_c = l_new;
+    };
+    if (MODE == kDual) {
+        if (warp >= 4) {
+            // The staging area overlaps the query tile, P and the K/V slots: the query copy must have
+            // landed and every MMA of the CTA must be complete before it is written.
+            mbar_wait_warp(smem_u32(&c.q_full), 0, abort_flag, a.status);
+            named_barrier(2, wg_threads);
+            if (tid == kAuxThreads) SS_TR(5, 1);
+            const bool any_valid = __any_sync(0xffffffffu, vi >= 0);
+            constexpr uint32_t RB = RP * 4;
+            const uint32_t srow = x_base + static_cast<uint32_t>(pidx * 64 + lrow) * RB;
+            if (any_valid) {
+                #pragma unroll
+                for (int c0 = 0; c0 < HD; c0 += 16) {
+                    uint32_t orr[16];
+                    if (has_acc) { tmem_ld16<0>(o_addr + c0, orr); tmem_wait_ld(); }
+                    else { for (int i = 0; i < 16; ++i) orr[i] = 0u; }
+                    if (vi >= 0) {
+                        #pragma unroll
+                        for (int i = 0; i < 16; i += 4) st_shared_v4(srow + (c0 + i) * 4u, orr[i], orr[i + 1], orr[i + 2], orr[i + 3]);
+                    }
+                }
+                if (vi >= 0) st_shared_v4(srow + HD * 4u, __float_as_uint(m_run), __float_as_uint(l_run), 0u, 0u);
+            }
+            if (tid == kAuxThreads) SS_TR(5, 2);
+            named_barrier(1, wg_threads);
+            // each of the row's four threads combines one quarter of the columns
+            if (vi >= 0) {
+                float m_out = -INFINITY, l_out = 0.f;
+                float4 acc[QW / 4];
+                combine_x(4, false, m_out, l_out, acc);
+                if (C == 1) {
+                    // the pair was not split: this is the result
+                    if (!skip) {
+                        const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, ri);
+                        const float inv = 1.f / l_out;
+                        #pragma unroll
+                        for (int i = 0; i < QW / 4; ++i) {
+                            uint2 o;
+                            o.x = pack_bf16(acc[i].x * inv, acc[i].y * inv);
+                            o.y = pack_bf16(acc[i].z * inv, acc[i].w * inv);
+                            *reinterpret_cast<uint2*>(dst.o + pidx * QW + i * 4) = o;
+                        }
+                        if (dst.lse && pidx == 0) *dst.lse = (m_out + log2f(l_out)) * 0.6931471805599453f;
+                    }
+                } else {
+                    float* dst = part_mine + static_cast<size_t>(lrow) * RP;     // same row order as the staging area
+                    #pragma unroll
+                    for (int i = 0; i < QW / 4; ++i) __stcg(reinterpret_cast<float4*>(dst + pidx * QW + i * 4), acc[i]);
+                    if (pidx == 0) __stcg(reinterpret_cast<float2*>(dst + HD), make_float2(m_out, l_out));
+                }
+            }
+            if (tid == kAuxThreads) SS_TR(5, 3);
+        }
+    } else if (C == 1) {
         // the pair was not split: normalise and write this thread's row
         if (warp >= 4 && __any_sync(0xffffffffu, ri.valid) && !skip) {
             const float inv = 1.f / l_run;
@@ -941,226 +1060,164 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 *reinterpret_cast<uint4*>(dst.o + c0 + 8) = hi;
             }
         }
-    } else if (MODE == kMulti) {
-        // Every thread of the cluster passes both barriers, whatever happened above.
-        // Barrier A: all CTAs are done with their pipelines, so shared memory can be reused.
-        cluster_arrive();
-        const int n_src = C * G::kCopies;                       // partials per row
-        const int rpc_max = kBlockRows / n_src;                 // row stride of the receive buffers
-        // valid row number vi of the block goes to CTA vi / rpc, local row vi % rpc
-        int vi = -1;
-        uint32_t remote = 0, ml_remote = 0;
-        bool sender = false;
-        if (warp >= 4) {
-            const int nvr = sp.n_valid(rblk);
-            const int rpc = (nvr + C - 1) / C;
-            vi = ri.valid ? sp.valid_index(rblk * kBlockRows + lrow) : -1;
-            sender = __any_sync(0xffffffffu, vi >= 0);
-            if (vi >= 0) {
-                const uint32_t dst_rank = vi / rpc;
-                const int lr = vi - dst_rank * rpc;
-                const int src = static_cast<int>(rank) * G::kCopies + copy;
-                // receiver layout: [block][source][local row][kMergePitch floats]
-                remote = map_to_rank(merge_base + (((my_blk * n_src + src) * rpc_max + lr) * G::kMergePitch) * 4u, dst_rank);
-                ml_remote = map_to_rank(smem_u32(&c.ml[my_blk][src * rpc_max + lr]), dst_rank);
-            }
-        }
-        {
-            cluster_wait();
-            if (sender) {
-                #pragma unroll
-                for (int c0 = 0; c0 < HD; c0 += 16) {
-                    uint32_t orr[16];
-                    if (has_acc) { tmem_ld16<0>(o_addr + c0, orr); tmem_wait_ld(); }
-                    else { for (int i = 0; i < 16; ++i) orr[i] = 0u; }
-                    if (vi >= 0) {
-                        #pragma unroll
-                        for (int i = 0; i < 16; i += 4)
-                            st_cluster_v4(remote + (c0 + i) * 4u, orr[i], orr[i + 1], orr[i + 2], orr[i + 3]);
-                    }
-                }
-                if (vi >= 0) st_cluster_v2(ml_remote, m_run, l_run);
-            }
-        }
-        // Barrier B: every partial has been delivered.
-        cluster_arrive();
-        cluster_wait();
-        if (warp >= 4 && !skip) {
-            const int nvr = sp.n_valid(rblk);
-            const int rpc = (nvr + C - 1) / C;
-            const int wq = warp & 3;
-            // one warp per row, one lane per four columns
-            for (int lr = wq; lr < rpc; lr += 4) {
-                const int v = static_cast<int>(rank) * rpc + lr;
-                if (v >= nvr) break;
-                const RowInfo r = row_info(sp, sp.row_of(rblk, v));
-                float mx = -INFINITY;
-                for (int s = 0; s < n_src; ++s) mx = fmaxf(mx, c.ml[my_blk][s * rpc_max + lr].x);
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                float l = 0.f;
-                for (int s = 0; s < n_src; ++s) {
-                    const float2 ml = c.ml[my_blk][s * rpc_max + lr];
-                    const float w = exp2f(ml.x - mx);         // 0 for a partial that saw no visible key
-                    l += w * ml.y;
-                    if (lane * 4 < HD) {
-                        const float4 x4 = ld_shared_v4(merge_base + (((my_blk * n_src + s) * rpc_max + lr) * G::kMergePitch + lane * 4) * 4u);
-                        acc.x += w * x4.x; acc.y += w * x4.y; acc.z += w * x4.z; acc.w += w * x4.w;
-                    }
-                }
-                const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, r);
-                const float inv = 1.f / l;
-                if (lane * 4 < HD) {
-                    uint2 o;
-                    o.x = pack_bf16(acc.x * inv, acc.y * inv);
-                    o.y = pack_bf16(acc.z * inv, acc.w * inv);
-                    *reinterpret_cast<uint2*>(dst.o + lane * 4) = o;
-                }
-                if (dst.lse && lane == 0) *dst.lse = (mx + log2f(l)) * 0.6931471805599453f;
-            }
-        }
     } else {
-        // ---- kSingle / kDual: one row block.  Rows travel as (O[HD], m, l) records of kRowBytes. ----
-        constexpr uint32_t RB = G::kRowBytes;
-        constexpr int QW = HD / 4;                                             // columns one thread combines (kDual)
-        const int nvr = sp.n_valid(0);
-        const int rpc = (nvr + C - 1) / C;                                     // rows merged per CTA
-        const int my_rows = max(0, min(rpc, nvr - static_cast<int>(rank) * rpc));
-        // staging in the shared memory the pipeline no longer needs
-        const uint32_t x_base = merge_base;                                    // kDual: [4 partials][64 rows]
-        const uint32_t y_base = merge_base + (MODE == kDual ? 256u : 0u) * RB; // rows to ship, in valid-row order
-        const uint32_t r_base = merge_base + (MODE == kDual ? 320u : 128u) * RB;   // received: [source CTA][rpc rows]
-        const uint32_t recv_bar = smem_u32(&c.recv_full);
-        if (tid == kAuxThreads) mbar_expect_tx(recv_bar, static_cast<uint32_t>(C * my_rows) * RB);
-        if (warp >= 4) {
-            // the staging areas overlap the query tile and the other warpgroup's P and K/V slots: the query
-            // copy must have landed and every MMA of the CTA must be complete before they are written
-            mbar_wait_warp(smem_u32(&c.q_full), 0, abort_flag, a.status);
-            if (MODE == kDual) named_barrier(2, G::kWGs * kBlockRows);
-        }
-        // Barrier A, arrival (every thread of the cluster, whatever happened above): this CTA's pipeline
-        // is finished, so the other CTAs may write its receive area, which its own staging never touches.
-        cluster_arrive();
-        if (warp >= 4) {
-            if (tid == kAuxThreads) SS_TR(5, 1);
-            const int vi = ri.valid ? sp.valid_index(lrow) : -1;
-            const bool any_valid = __any_sync(0xffffffffu, vi >= 0);
-            const int pidx = my_blk * 2 + copy;                                // partial of the row inside this CTA
-            // kDual: the four partials of a row go to X; kSingle: the row goes straight to Y
-            const uint32_t srow = MODE == kDual ? x_base + static_cast<uint32_t>(pidx * 64 + lrow) * RB
-                                                : y_base + static_cast<uint32_t>(vi >= 0 ? vi : 0) * RB;
-            if (any_valid) {
-                #pragma unroll
-                for (int c0 = 0; c0 < HD; c0 += 16) {
-                    uint32_t orr[16];
-                    if (has_acc) { tmem_ld16<0>(o_addr + c0, orr); tmem_wait_ld(); }
-                    else { for (int i = 0; i < 16; ++i) orr[i] = 0u; }
-                    if (vi >= 0) {
-                        #pragma unroll
-                        for (int i = 0; i < 16; i += 4) st_shared_v4(srow + (c0 + i) * 4u, orr[i], orr[i + 1], orr[i + 2], orr[i + 3]);
-                    }
-                }
-                if (vi >= 0) st_shared_v4(srow + HD * 4u, __float_as_uint(m_run), __float_as_uint(l_run), 0u, 0u);
-            }
-            if (tid == kAuxThreads) SS_TR(5, 2);
-            if (MODE == kDual) {
-                named_barrier(1, G::kWGs * kBlockRows);
-                // each of the row's four threads combines one quarter of the columns
+        // kSingle / kMulti, split pair: every thread stores its row's partial
+        if (warp >= 4 && __any_sync(0xffffffffu, vi >= 0)) {
+            float* dst = part_mine + static_cast<size_t>(rblk * kBlockRows + (vi >= 0 ? vi : 0)) * RP;
+            #pragma unroll
+            for (int c0 = 0; c0 < HD; c0 += 16) {
+                uint32_t orr[16];
+                if (has_acc) { tmem_ld16<0>(o_addr + c0, orr); tmem_wait_ld(); }
+                else { for (int i = 0; i < 16; ++i) orr[i] = 0u; }
                 if (vi >= 0) {
-                    float w[4], mp[4];
-                    float m_out = -INFINITY, l_out = 0.f;
                     #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const float2 t = ld_shared_v2(x_base + static_cast<uint32_t>(k * 64 + lrow) * RB + HD * 4u);
-                        mp[k] = t.x; w[k] = t.y;
-                        m_out = fmaxf(m_out, t.x);
-                    }
-                    #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const float e = mp[k] == -INFINITY ? 0.f : exp2f(mp[k] - m_out);
-                        l_out += e * w[k];
-                        w[k] = e;
-                    }
-                    const uint32_t yrow = y_base + static_cast<uint32_t>(vi) * RB;
-                    #pragma unroll
-                    for (int i = 0; i < QW; i += 4) {
-                        const uint32_t col = static_cast<uint32_t>(pidx * QW + i) * 4u;
-                        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                        #pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            const float4 t = ld_shared_v4(x_base + static_cast<uint32_t>(k * 64 + lrow) * RB + col);
-                            acc.x += w[k] * t.x; acc.y += w[k] * t.y; acc.z += w[k] * t.z; acc.w += w[k] * t.w;
-                        }
-                        st_shared_v4(yrow + col, __float_as_uint(acc.x), __float_as_uint(acc.y), __float_as_uint(acc.z), __float_as_uint(acc.w));
-                    }
-                    if (pidx == 0) st_shared_v4(yrow + HD * 4u, __float_as_uint(m_out), __float_as_uint(l_out), 0u, 0u);
+                    for (int i = 0; i < 16; i += 4)
+                        __stcg(reinterpret_cast<float4*>(dst + c0 + i), make_float4(__uint_as_float(orr[i]), __uint_as_float(orr[i + 1]),
+                                                                                   __uint_as_float(orr[i + 2]), __uint_as_float(orr[i + 3])));
                 }
             }
-            if (tid == kAuxThreads) SS_TR(5, 3);
-            fence_async_smem();                          // the rows are read by the bulk-copy engine
+            if (vi >= 0) __stcg(reinterpret_cast<float2*>(dst + HD), make_float2(m_run, l_run));
         }
-        // Barrier A, completion: every CTA of the cluster has finished its pipeline.  The CTA-wide named
-        // barrier orders the staged rows of all warpgroups before the one thread that ships them.
-        cluster_wait();
-        if (warp >= 4) named_barrier(3, G::kWGs * kBlockRows);
-        if (tid == kAuxThreads) SS_TR(5, 4);
+    }
+
+    if (C > 1 && warp >= 4) {
+        // arrive on the pair's counter; the last CTA combines
+        __threadfence();
+        named_barrier(3, wg_threads);
         if (tid == kAuxThreads) {
-            for (int d = 0; d < C; ++d) {
-                const int rows_d = max(0, min(rpc, nvr - d * rpc));
-                if (rows_d > 0)
-                    dsmem_bulk_copy(map_to_rank(r_base + static_cast<uint32_t>(rank * rpc) * RB, d), y_base + static_cast<uint32_t>(d * rpc) * RB,
-                                    static_cast<uint32_t>(rows_d) * RB, map_to_rank(recv_bar, d));
-            }
+            const int prev = atomicAdd(&a.counters[pair], 1);
+            const int last = (prev == C - 1);
+            if (last) a.counters[pair] = 0;              // ready for the next call
+            __threadfence();
+            c.is_last = last;
         }
-        if (warp >= 4 && !skip && my_rows > 0) {
-            // the rows this CTA merges have arrived from every CTA of the cluster (complete_tx on recv_full)
-            if (tid == kAuxThreads) SS_TR(5, 5);
-            if (mbar_wait_warp(recv_bar, 0, abort_flag, a.status)) {
-                if (tid == kAuxThreads) SS_TR(5, 6);
-                // one warp per row, one lane per four columns
-                for (int lr = warp - 4; lr < my_rows; lr += G::kWGs * 4) {
-                    const RowInfo r = row_info(sp, sp.row_of(0, static_cast<int>(rank) * rpc + lr));
-                    float ms[8], wl[8];
-                    float mx = -INFINITY;
-                    #pragma unroll
-                    for (int s = 0; s < 8; ++s) {
-                        if (s < C) {
-                            const float2 t = ld_shared_v2(r_base + static_cast<uint32_t>(s * rpc + lr) * RB + HD * 4u);
-                            ms[s] = t.x; wl[s] = t.y;
-                            mx = fmaxf(mx, t.x);
-                        }
+        named_barrier(3, wg_threads);
+        if (tid == kAuxThreads) SS_TR(5, 4);
+        if (c.is_last && !skip) {
+            if (MODE == kDual) {
+                // The partials of the pair's CTAs are contiguous in the workspace: bulk-copy them into the
+                // staging area (up to four at a time) and combine from shared memory.
+                constexpr uint32_t RB = RP * 4;
+                const uint32_t mbar = smem_u32(&c.merge_full[0]);
+                float m_c = -INFINITY, l_c = 0.f;
+                float4 acc[QW / 4];
+                bool ok = true;
+                int round = 0;
+                for (int s0 = 0; s0 < C; s0 += 4, ++round) {
+                    const int ns = min(4, C - s0);
+                    if (round > 0) named_barrier(1, wg_threads);          // everyone has read the previous batch
+                    if (tid == kAuxThreads) {
+                        asm volatile("fence.proxy.async;" ::: "memory");  // generic accesses to X and to the partials come first
+                        mbar_expect_tx(mbar, static_cast<uint32_t>(ns) * 64u * RB);
+                        for (int k = 0; k < ns; ++k)
+                            bulk_load(x_base + static_cast<uint32_t>(k) * 64u * RB, part_pair + static_cast<size_t>(s0 + k) * rows_cap * RP, 64u * RB, mbar);
                     }
-                    float l = 0.f;
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    ok = ok && mbar_wait_warp(mbar, round & 1, abort_flag, a.status);
+                    if (ok && vi >= 0) combine_x(ns, round > 0, m_c, l_c, acc);
+                }
+                if (tid == kAuxThreads) SS_TR(5, 7);
+                if (ok && vi >= 0) {
+                    const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, ri);
+                    const float inv = 1.f / l_c;
                     #pragma unroll
-                    for (int s = 0; s < 8; ++s) {
-                        if (s < C) {
-                            const float w = ms[s] == -INFINITY ? 0.f : exp2f(ms[s] - mx);
-                            l += w * wl[s];
-                            if (lane * 4 < HD) {
-                                const float4 t = ld_shared_v4(r_base + static_cast<uint32_t>(s * rpc + lr) * RB + lane * 16u);
-                                acc.x += w * t.x; acc.y += w * t.y; acc.z += w * t.z; acc.w += w * t.w;
+                    for (int i = 0; i < QW / 4; ++i) {
+                        uint2 o;
+                        o.x = pack_bf16(acc[i].x * inv, acc[i].y * inv);
+                        o.y = pack_bf16(acc[i].z * inv, acc[i].w * inv);
+                        *reinterpret_cast<uint2*>(dst.o + pidx * QW + i * 4) = o;
+                    }
+                    if (dst.lse && pidx == 0) *dst.lse = (m_c + log2f(l_c)) * 0.6931471805599453f;
+                }
+                if (tid == kAuxThreads) SS_TR(5, 8);
+            } else {
+                // kSingle / kMulti: the partial rows stream through two shared-memory buffers, 32 rows of
+                // every CTA of the pair per round; the copy of round i+1 runs while round i is combined.
+                constexpr int RR = 32;
+                constexpr uint32_t RB = RP * 4;
+                const uint32_t buf_bytes = static_cast<uint32_t>(C) * RR * RB;
+                const size_t cta_stride = static_cast<size_t>(rows_cap) * RP;
+                mbar_wait_warp(smem_u32(&c.q_full), 0, abort_flag, a.status);      // the query copy may alias the buffers
+                int n_rounds = 0;
+                for (int k = 0; k < n_blocks; ++k) n_rounds += (sp.n_valid(k) + RR - 1) / RR;
+                // round -> (block, first valid-row number)
+                auto round_rows = [&](int i, int& blk, int& r0) {
+                    blk = 0;
+                    for (;;) {
+                        const int n = (sp.n_valid(blk) + RR - 1) / RR;
+                        if (i < n) break;
+                        i -= n; ++blk;
+                    }
+                    r0 = i * RR;
+                };
+                auto issue_round = [&](int i) {
+                    int blk, r0;
+                    round_rows(i, blk, r0);
+                    const uint32_t mbar = smem_u32(&c.merge_full[i & 1]);
+                    asm volatile("fence.proxy.async;" ::: "memory");      // generic accesses to the buffer and to the partials come first
+                    mbar_expect_tx(mbar, buf_bytes);
+                    for (int sidx = 0; sidx < C; ++sidx)
+                        bulk_load(merge_base + (i & 1) * buf_bytes + static_cast<uint32_t>(sidx) * RR * RB,
+                                  part_pair + sidx * cta_stride + static_cast<size_t>(blk * kBlockRows + r0) * RP, RR * RB, mbar);
+                };
+                named_barrier(1, wg_threads);                             // every warpgroup is past its pipeline
+                if (tid == kAuxThreads && n_rounds > 0) issue_round(0);
+                bool ok = true;
+                for (int i = 0; i < n_rounds; ++i) {                      // every thread runs every round: the barriers stay matched
+                    if (i + 1 < n_rounds) {
+                        named_barrier(1, wg_threads);                     // everyone has read buffer (i + 1) & 1
+                        if (tid == kAuxThreads) issue_round(i + 1);
+                    }
+                    ok = ok && mbar_wait_warp(smem_u32(&c.merge_full[i & 1]), (i >> 1) & 1, abort_flag, a.status);
+                    if (!ok) continue;
+                    int blk, r0;
+                    round_rows(i, blk, r0);
+                    const int nvr = sp.n_valid(blk);
+                    const uint32_t xb = merge_base + (i & 1) * buf_bytes;
+                    // work item: (row of the round, group of four columns)
+                    for (int w = tid - kAuxThreads; w < RR * (HD / 4); w += wg_threads) {
+                        const int rr = w / (HD / 4), g = w - rr * (HD / 4);
+                        if (r0 + rr >= nvr) continue;
+                        float ms[4], ls[4];
+                        float mx = -INFINITY;
+                        #pragma unroll
+                        for (int sidx = 0; sidx < 4; ++sidx) {
+                            if (sidx < C) {
+                                const float2 t = ld_shared_v2(xb + static_cast<uint32_t>(sidx * RR + rr) * RB + HD * 4u);
+                                ms[sidx] = t.x; ls[sidx] = t.y;
+                                mx = fmaxf(mx, t.x);
                             }
                         }
-                    }
-                    const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, r);
-                    const float inv = 1.f / l;
-                    if (lane * 4 < HD) {
+                        float l = 0.f;
+                        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                        #pragma unroll
+                        for (int sidx = 0; sidx < 4; ++sidx) {
+                            if (sidx < C) {
+                                const float wgt = ms[sidx] == -INFINITY ? 0.f : exp2f(ms[sidx] - mx);   // 0: saw no visible key
+                                l += wgt * ls[sidx];
+                                const float4 t = ld_shared_v4(xb + static_cast<uint32_t>(sidx * RR + rr) * RB + g * 16u);
+                                acc.x += wgt * t.x; acc.y += wgt * t.y; acc.z += wgt * t.z; acc.w += wgt * t.w;
+                            }
+                        }
+                        const RowInfo r = row_info(sp, sp.row_of(blk, r0 + rr));
+                        const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, r);
+                        const float inv = 1.f / l;
                         uint2 o;
                         o.x = pack_bf16(acc.x * inv, acc.y * inv);
                         o.y = pack_bf16(acc.z * inv, acc.w * inv);
-                        *reinterpret_cast<uint2*>(dst.o + lane * 4) = o;
+                        *reinterpret_cast<uint2*>(dst.o + g * 4) = o;
+                        if (dst.lse && g == 0) *dst.lse = (mx + log2f(l)) * 0.6931471805599453f;
                     }
-                    if (dst.lse && lane == 0) *dst.lse = (mx + log2f(l)) * 0.6931471805599453f;
                 }
             }
         }
-        if (tid == kAuxThreads) SS_TR(5, 7);
-        // nobody leaves while a copy into or out of its shared memory may still be in flight
-        cluster_arrive();
-        cluster_wait();
-        if (tid == kAuxThreads) SS_TR(5, 8);
+        if (tid == kAuxThreads) SS_TR(5, 5);
     }
 
+#ifdef SS_TRACE
+    if (tid == 0) atomicMax(&g_wall[s_launch & 7][1], wall_ns());
+    if (tid == 0) atomicMin(&g_wall[s_launch & 7][5], wall_ns());      // first CTA end
+    if (tid == 0 && blockIdx.x == 0) { g_wall[s_launch & 7][3] = wall_ns() - g_wall[s_launch & 7][3]; g_wall[s_launch & 7][4] = clock64() - g_wall[s_launch & 7][4]; }
+#endif
     // ---- release TMEM ---------------------------------------------------------------------------
     tc_fence_before();
     __syncthreads();
@@ -1208,6 +1265,7 @@ static bool make_map(CUtensorMap* out, const void* basep, int d, long long n1, l
 struct AttnPlan {
     int tmax8, spec_rows, n_blocks, mode, tile_keys, n_kslots, n_vslots, cluster, threads;
     size_t smem;
+    size_t counter_bytes, partial_bytes;       // workspace after its header
 };
 
 static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
@@ -1222,10 +1280,11 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     plan->mode = plan->n_blocks > 1 ? kMulti : (q_rows <= 64 ? kDual : kSingle);
     plan->tile_keys = plan->mode == kMulti ? 64 : 128;
     plan->threads = kAuxThreads + (plan->mode == kMulti ? kMaxBlocks : (plan->mode == kDual ? 2 : 1)) * kBlockRows;
-    // cluster size: the largest power of two that still fits the grid on the SMs in one wave
+    // CTAs per (sequence, head) pair: the largest power of two that still fits the grid on the SMs in one wave
     const long long pairs = static_cast<long long>(p.batch) * p.n_heads;
     int c = 1;
-    while (c < 8 && pairs * (c * 2) <= sm_count()) c *= 2;
+    const int c_max = plan->mode == kDual ? 8 : 4;          // the merge of the other variants combines at most four partials
+    while (c < c_max && pairs * (c * 2) <= sm_count()) c *= 2;
     plan->cluster = c;
     const int q_smem_rows = plan->mode == kDual ? kBlockRows : q_rows;
     const size_t p_total = plan->mode == kDual ? static_cast<size_t>(2) * 3 * 64 * 128                 // two warpgroups
@@ -1242,12 +1301,16 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     plan->n_vslots = slots - plan->n_kslots > kMaxSlots ? kMaxSlots : slots - plan->n_kslots;
     size_t bytes = qp + static_cast<size_t>(plan->n_kslots + plan->n_vslots) * slot;
     if (bytes < qp + overhang) bytes = qp + overhang;
-    // rows of (head_dim + 4) floats staged for the merge once the pipeline is done
-    const size_t merge_rows = plan->mode == kMulti ? static_cast<size_t>(plan->n_blocks) * kBlockRows
-                            : plan->mode == kSingle ? 128 + 128 + 8 : 256 + 64 + 64 + 8;
-    const size_t merge = merge_rows * (p.head_dim + 4) * 4;
-    if ((c > 1 || plan->mode == kDual) && merge > bytes) bytes = merge;
+    // kDual stages its four CTA-local partials of every row ((head_dim + 4) floats) once the pipeline is done
+    // (the other variants stream the partials of a split pair through two buffers of 32 rows per CTA of the pair)
+    const size_t stage = plan->mode == kDual ? static_cast<size_t>(4) * 64 * (p.head_dim + 4) * 4
+                                             : static_cast<size_t>(2) * c * 32 * (p.head_dim + 4) * 4;
+    if ((plan->mode == kDual || c > 1) && stage > bytes) bytes = stage;
     plan->smem = bytes + 1024;
+    // workspace: one arrival counter per pair; one partial row per (pair, CTA of the pair, query row)
+    const size_t rows_cap = plan->mode == kDual ? 64 : static_cast<size_t>(plan->n_blocks) * kBlockRows;
+    plan->counter_bytes = (static_cast<size_t>(pairs) * sizeof(int32_t) + 255) / 256 * 256;
+    plan->partial_bytes = c > 1 ? static_cast<size_t>(pairs) * c * rows_cap * (p.head_dim + 4) * 4 : 0;
     return plan->smem <= static_cast<size_t>(kMaxDynSmem);
 }
 
@@ -1268,17 +1331,13 @@ static int32_t launch(const AttnArgs& args, const AttnPlan& plan, long long pair
     // always more than half of an SM's shared memory: one CTA per SM, so a CTA never queues for TMEM
     cfg.dynamicSmemBytes = plan.smem < 120 * 1024 ? 120 * 1024 : plan.smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = static_cast<unsigned>(plan.cluster);
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
+    cudaLaunchAttribute attr[1];
     // programmatic dependent launch: the CTAs may be scheduled while the previous kernel of the stream
     // drains; the kernel touches global memory only after its griddepcontrol.wait, so stream order holds
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 2;
+    cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, msa_attention_kernel<HD, MODE>, args) == cudaSuccess ? SS_OK : SS_ERR_CUDA;
 }
 
@@ -1287,7 +1346,7 @@ static int32_t launch(const AttnArgs& args, const AttnPlan& plan, long long pair
 extern "C" size_t ss_msa_attention_workspace_bytes(const ss_attn_params* p) {
     ss::AttnPlan plan;
     if (p == nullptr || !ss::make_plan(*p, &plan)) return 0;
-    return ss::kWsHeaderBytes;     // the status word; split-KV partials never leave the chip
+    return ss::kWsHeaderBytes + plan.counter_bytes + plan.partial_bytes;
 }
 
 extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
@@ -1345,6 +1404,8 @@ extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
     a.kv_start = reinterpret_cast<const long long*>(p->kv_start);
     a.kv_len = p->kv_len; a.kv_capacity = p->kv_capacity; a.trees = p->trees;
     a.status = reinterpret_cast<int*>(p->workspace);
+    a.counters = reinterpret_cast<int*>(static_cast<char*>(p->workspace) + ss::kWsHeaderBytes);
+    a.partials = reinterpret_cast<float*>(static_cast<char*>(p->workspace) + ss::kWsHeaderBytes + plan.counter_bytes);
     const long long pairs = static_cast<long long>(p->batch) * H;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (plan.mode == ss::kDual) {
@@ -1376,6 +1437,14 @@ extern "C" int32_t ss_trace_read(long long* out) {
 extern "C" int32_t ss_trace_clear() {
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, ss::g_trace) != cudaSuccess) return -1;
-    return cudaMemset(p, 0, sizeof(ss::g_trace)) == cudaSuccess ? 0 : -1;
+    if (cudaMemset(p, 0, sizeof(ss::g_trace)) != cudaSuccess) return -1;
+    unsigned long long wall[8][6];
+    for (int i = 0; i < 8; ++i) { wall[i][0] = ~0ull; wall[i][1] = 0ull; wall[i][2] = 0ull; wall[i][3] = 0ull; wall[i][4] = 0ull; wall[i][5] = ~0ull; }
+    unsigned long long keys[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    if (cudaMemcpyToSymbol(ss::g_wall, wall, sizeof(wall)) != cudaSuccess) return -1;
+    return cudaMemcpyToSymbol(ss::g_key, keys, sizeof(keys)) == cudaSuccess ? 0 : -1;
+}
+extern "C" int32_t ss_trace_wall(unsigned long long* out) {
+    return cudaMemcpyFromSymbol(out, ss::g_wall, sizeof(ss::g_wall)) == cudaSuccess ? 0 : -1;
 }
 #endif
