@@ -101,6 +101,16 @@ int32_t ss_tree_build(const int32_t* parent, int32_t n_nodes, int32_t gamma, ss_
  * If kv_capacity is given and L_b + T_b > kv_capacity[b], sequence b is skipped and the status word
  * is set to SS_ERR_CAPACITY.
  * Errors (nothing launched): SS_ERR_INVALID_ARG, SS_ERR_UNSUPPORTED, SS_ERR_WORKSPACE, SS_ERR_CUDA. */
+/* ss_attn_params.flags.
+ * SS_ATTN_PREFIX_STABLE: the caller promises that no kernel that may still be running when this call's
+ * kernel is scheduled writes the cached prefix (slots below kv_len of every sequence), kv_start, kv_len,
+ * kv_capacity or the tree descriptors.  The call is launched so that it can be scheduled while the
+ * previous kernel of the stream drains (programmatic dependent launch); with the promise it reads the
+ * lengths and starts streaming the prefix during that time.  Queries, the tree nodes' K/V, the stream K/V
+ * and every output keep plain stream order either way.  A decode step satisfies the promise naturally:
+ * the kernels before a layer's attention write this step's queries and tree-node K/V, never the prefix. */
+#define SS_ATTN_PREFIX_STABLE 1u
+
 typedef struct ss_attn_params {
     int32_t batch, n_heads, head_dim, gamma;
     int32_t max_nodes;              /* row stride (in nodes) of the q/o/lse arrays, <= SS_MAX_NODES */
@@ -122,6 +132,7 @@ typedef struct ss_attn_params {
     float* lse_spec;
     void* workspace;
     size_t workspace_bytes;
+    uint32_t flags;                 /* SS_ATTN_* bits, 0 for none */
 } ss_attn_params;
 
 /* Bytes of workspace ss_msa_attention needs for these shapes (pointers in *p are not read). */

@@ -26,6 +26,8 @@ SS_ERR_CAPACITY = -5
 SS_ERR_CUDA = -6
 SS_ERR_DEVICE_TIMEOUT = -7
 
+SS_ATTN_PREFIX_STABLE = 1
+
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libss_msa.so")
 _lib = None
 
@@ -54,7 +56,7 @@ class AttnParams(C.Structure):
                 ("kv_slot_stride", C.c_int64), ("kv_head_stride", C.c_int64), ("kv_total_slots", C.c_int64),
                 ("kv_start", C.c_void_p), ("kv_len", C.c_void_p), ("kv_capacity", C.c_void_p),
                 ("trees", C.c_void_p), ("lse_main", C.c_void_p), ("lse_spec", C.c_void_p),
-                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("flags", C.c_uint32)]
 
 
 class CacheLayout(C.Structure):
@@ -142,7 +144,7 @@ def workspace(n_bytes: int, device="cuda") -> torch.Tensor:
 # ---- device -------------------------------------------------------------------------------------
 def make_attn_params(*, q_main, o_main, k_cache, v_cache, kv_start, kv_len, trees, gamma, sm_scale,
                      q_spec=None, k_spec=None, v_spec=None, o_spec=None, kv_capacity=None, lse_main=None,
-                     lse_spec=None, workspace=None) -> AttnParams:
+                     lse_spec=None, workspace=None, prefix_stable=False) -> AttnParams:
     """Fills ss_attn_params from tensors.  q_main/o_main: bf16 [B][Tmax][H][d]; *_spec: bf16
     [B][Tmax][gamma][H][d]; k_cache/v_cache: bf16 [slots][H][d] (any slot/head stride, d contiguous)."""
     B, Tmax, H, d = q_main.shape
@@ -159,6 +161,7 @@ def make_attn_params(*, q_main, o_main, k_cache, v_cache, kv_start, kv_len, tree
     p.lse_main, p.lse_spec = _ptr(lse_main), _ptr(lse_spec)
     p.workspace = _ptr(workspace)
     p.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    p.flags = SS_ATTN_PREFIX_STABLE if prefix_stable else 0
     return p
 
 

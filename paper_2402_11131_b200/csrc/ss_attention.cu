@@ -73,6 +73,7 @@ struct alignas(64) AttnArgs {
     int n_blocks, cluster, cluster_shift;   // cluster = 1 << cluster_shift
     int n_kslots, n_vslots;          // ring depths
     int head_coord;                  // 1, or 0 when all heads share one K/V (head stride 0)
+    int prefix_stable;               // the caller's SS_ATTN_PREFIX_STABLE promise
     float scale_log2;                // sm_scale * log2(e)
     __nv_bfloat16* o_main;
     __nv_bfloat16* o_spec;
@@ -96,7 +97,7 @@ struct Ctrl {
     unsigned long long anc[SS_MAX_NODES];
     uint32_t tmem_base;
     int abort;
-    int is_last;                 // this CTA arrived last on its pair's counter
+    int merge_ok;                // the pair's other CTAs arrived in time
     unsigned long long merge_full[2];   // a batch of the pair's partials has been copied into shared memory
 };
 
@@ -575,46 +576,35 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     // whole parked grid polling the dependency slows the kernel it waits for).  Only then may the next
     // kernel be scheduled: every CTA of this grid is resident and past its wait, so CTAs of a later
     // grid can never hold an SM that this grid still needs.
-    if (tid == 0) {
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    }
-    __syncthreads();
-    if (tid == 0) SS_TR(0, 2);
-
-    if (tid == 0) {
-        // the queries depend on nothing but (sequence, head): request them before the lengths are known
-        const uint32_t qbar = smem_u32(&c.q_full);
-        mbar_expect_tx(qbar, G::kCopies * G::kHalves * q_rows * 128u);
-        #pragma unroll
-        for (int cp = 0; cp < G::kCopies; ++cp) {
-            #pragma unroll
-            for (int hh = 0; hh < G::kHalves; ++hh) {
-                const uint32_t dst = q_base + hh * q_smem_rows * 128u + cp * 64u * 128u;
-                tma_load_3d(dst, &a.tm_qm, hh * 64, h, b * a.max_nodes, qbar);
-                if (a.gamma > 0) tma_load_3d(dst + a.tmax8 * 128u, &a.tm_qs, hh * 64, h, static_cast<int>(spec_row0), qbar);
-            }
+    auto dependency_wait = [&]() {
+        if (tid == 0) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
         }
+        __syncthreads();
+    };
+    // Without the caller's promise nothing is read before the wait.  With it (prefix_stable: nothing
+    // still in flight writes the cached prefix, the lengths or the trees) the lengths are read and the
+    // first prefix tiles requested right away, so HBM streams while the previous kernel drains.
+    if (!a.prefix_stable) dependency_wait();
+    if (tid == 0) SS_TR(0, 2);
+    constexpr uint32_t kTmemCols = 512;
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&c.tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    if (tid == 0) SS_TR(0, 3);
     // per-sequence scalars (every thread reads them)
     // (read through L2: under an early launch the SM's L1 may predate the previous kernel's last writes)
     int L = __ldcg(a.kv_len + b);
     int T = min(max(__ldcg(&a.trees[b].n_nodes), 0), a.max_nodes);
     const long long slot0 = __ldcg(a.kv_start + b);
     const int cap = a.kv_capacity != nullptr ? __ldcg(a.kv_capacity + b) : 0x7fffffff;
-    constexpr uint32_t kTmemCols = 512;
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&c.tmem_base)), "r"(kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
     bool skip = false;                                    // sequence over its slot capacity: nothing read or written
     if (L < 0 || L + T > cap) {
         skip = true;
-        if (tid == 0) set_status(a.status, SS_ERR_CAPACITY);
         L = 0; T = 0;
     }
-    if (tid >= kAuxThreads && tid < kAuxThreads + SS_MAX_NODES) c.anc[tid - kAuxThreads] = __ldcg(&a.trees[b].anc_mask[tid - kAuxThreads]);
+    if (tid == 0) SS_TR(0, 3);
 
     const Span<TK> sp = make_span<TK>(a, L, T, static_cast<int>(rank), MODE == kDual);
 
@@ -641,14 +631,38 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             else tma_load_3d(dst + hh * G::kBoxBytes, &a.tm_vs, hh * 64, h, static_cast<int>(spec_row0 + x), bar);
         }
     };
-    if (tid == 0) SS_TR(0, 4);
     // the producers start before the CTA-wide synchronisation: the first tiles need no hand-back
     const int n_early_k = min(sp.n_tiles, nk), n_early_v = min(sp.n_tiles, nv_slots);
-    if (tid == 0) {
-        for (int j = 0; j < n_early_k; ++j) load_k(j, j);
-    } else if (tid == 96) {
-        for (int j = 0; j < n_early_v; ++j) load_v(j, j);
+    // before the dependency wait only tiles that lie wholly inside the cached prefix may be requested
+    auto prefix_only = [&](int j) { return sp.is_cache(j) && sp.first_key(j) + TK <= sp.L; };
+    int n_pre = 0;                                        // early tiles this producer thread has requested
+    if (a.prefix_stable) {
+        if (tid == 0) {
+            while (n_pre < n_early_k && prefix_only(n_pre)) { load_k(n_pre, n_pre); ++n_pre; }
+        } else if (tid == 96) {
+            while (n_pre < n_early_v && prefix_only(n_pre)) { load_v(n_pre, n_pre); ++n_pre; }
+        }
+        dependency_wait();
     }
+    if (skip && tid == 0) set_status(a.status, SS_ERR_CAPACITY);
+    if (tid == 0) {
+        // the rest of the first tiles, then the queries
+        for (int j = n_pre; j < n_early_k; ++j) load_k(j, j);
+        const uint32_t qbar = smem_u32(&c.q_full);
+        mbar_expect_tx(qbar, G::kCopies * G::kHalves * q_rows * 128u);
+        #pragma unroll
+        for (int cp = 0; cp < G::kCopies; ++cp) {
+            #pragma unroll
+            for (int hh = 0; hh < G::kHalves; ++hh) {
+                const uint32_t dst = q_base + hh * q_smem_rows * 128u + cp * 64u * 128u;
+                tma_load_3d(dst, &a.tm_qm, hh * 64, h, b * a.max_nodes, qbar);
+                if (a.gamma > 0) tma_load_3d(dst + a.tmax8 * 128u, &a.tm_qs, hh * 64, h, static_cast<int>(spec_row0), qbar);
+            }
+        }
+    } else if (tid == 96) {
+        for (int j = n_pre; j < n_early_v; ++j) load_v(j, j);
+    }
+    if (tid >= kAuxThreads && tid < kAuxThreads + SS_MAX_NODES) c.anc[tid - kAuxThreads] = __ldcg(&a.trees[b].anc_mask[tid - kAuxThreads]);
     if (tid == 0) SS_TR(0, 5);
     // kDual: the 64 zero rows in the middle of each warpgroup's P stay zero for the whole kernel
     if (MODE == kDual && tid >= kAuxThreads) {
@@ -1081,132 +1095,101 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     }
 
     if (C > 1 && warp >= 4) {
-        // arrive on the pair's counter; the last CTA combines
+        // Arrive on the pair's counter, then wait (bounded) until the pair's other CTAs have arrived too:
+        // they were launched together and need nothing from this CTA, so the wait is short.  Each CTA then
+        // combines its own share of the rows, so the tail of the kernel is a C-th of a single merger's.
         __threadfence();
         named_barrier(3, wg_threads);
         if (tid == kAuxThreads) {
-            const int prev = atomicAdd(&a.counters[pair], 1);
-            const int last = (prev == C - 1);
-            if (last) a.counters[pair] = 0;              // ready for the next call
-            __threadfence();
-            c.is_last = last;
+            unsigned int* cnt = reinterpret_cast<unsigned int*>(a.counters) + pair;
+            const unsigned int prev = atomicAdd(cnt, 1u);
+            const unsigned int target = (prev | static_cast<unsigned int>(C - 1)) + 1u;   // this call's C arrivals end here
+            bool ok = true;
+            const long long t0 = clock64();
+            for (;;) {
+                unsigned int now;
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(now) : "l"(cnt) : "memory");
+                if (static_cast<int>(now - target) >= 0) break;
+                if (*abort_flag || clock64() - t0 > kWaitCycles) { ok = false; break; }
+                __nanosleep(32);
+            }
+            if (!ok) { c.abort = 1; set_status(a.status, SS_ERR_DEVICE_TIMEOUT); }
+            c.merge_ok = ok ? 1 : 0;
         }
         named_barrier(3, wg_threads);
         if (tid == kAuxThreads) SS_TR(5, 4);
-        if (c.is_last && !skip) {
-            if (MODE == kDual) {
-                // The partials of the pair's CTAs are contiguous in the workspace: bulk-copy them into the
-                // staging area (up to four at a time) and combine from shared memory.
-                constexpr uint32_t RB = RP * 4;
-                const uint32_t mbar = smem_u32(&c.merge_full[0]);
-                float m_c = -INFINITY, l_c = 0.f;
-                float4 acc[QW / 4];
-                bool ok = true;
-                int round = 0;
-                for (int s0 = 0; s0 < C; s0 += 4, ++round) {
-                    const int ns = min(4, C - s0);
-                    if (round > 0) named_barrier(1, wg_threads);          // everyone has read the previous batch
-                    if (tid == kAuxThreads) {
-                        asm volatile("fence.proxy.async;" ::: "memory");  // generic accesses to X and to the partials come first
-                        mbar_expect_tx(mbar, static_cast<uint32_t>(ns) * 64u * RB);
-                        for (int k = 0; k < ns; ++k)
-                            bulk_load(x_base + static_cast<uint32_t>(k) * 64u * RB, part_pair + static_cast<size_t>(s0 + k) * rows_cap * RP, 64u * RB, mbar);
-                    }
-                    ok = ok && mbar_wait_warp(mbar, round & 1, abort_flag, a.status);
-                    if (ok && vi >= 0) combine_x(ns, round > 0, m_c, l_c, acc);
+        if (c.merge_ok && !skip) {
+            // This CTA's share: rows [first, first + share) of the pair's partial rows.  They stream through two
+            // shared-memory buffers, RR rows of every CTA of the pair per round (bulk copies from L2); the copy
+            // of round i + 1 runs while round i is combined.
+            constexpr uint32_t RB = RP * 4;
+            const int share = rows_cap >> a.cluster_shift;
+            const int first = static_cast<int>(rank) * share;
+            const int RR = min(share, C == 8 ? 16 : 32);
+            const int n_rounds = share / RR;
+            const uint32_t buf_bytes = static_cast<uint32_t>(C * RR) * RB;
+            const size_t cta_stride = static_cast<size_t>(rows_cap) * RP;
+            mbar_wait_warp(smem_u32(&c.q_full), 0, abort_flag, a.status);      // the query copy may alias the buffers
+            auto issue_round = [&](int i) {
+                const uint32_t mbar = smem_u32(&c.merge_full[i & 1]);
+                asm volatile("fence.proxy.async;" ::: "memory");      // generic accesses to the buffer and to the partials come first
+                mbar_expect_tx(mbar, buf_bytes);
+                for (int sidx = 0; sidx < C; ++sidx)
+                    bulk_load(merge_base + (i & 1) * buf_bytes + static_cast<uint32_t>(sidx * RR) * RB,
+                              part_pair + sidx * cta_stride + static_cast<size_t>(first + i * RR) * RP, static_cast<uint32_t>(RR) * RB, mbar);
+            };
+            // partial row number -> query row; false for a padding row
+            auto out_row = [&](int idx, RowInfo& r) -> bool {
+                if (MODE == kDual) { r = row_info(sp, idx); return r.valid; }
+                const int blk = idx / kBlockRows, v = idx - blk * kBlockRows;
+                if (v >= sp.n_valid(blk)) return false;
+                r = row_info(sp, sp.row_of(blk, v));
+                return true;
+            };
+            named_barrier(1, wg_threads);                             // every warpgroup is done with the staging area
+            if (tid == kAuxThreads) issue_round(0);
+            bool ok = true;
+            for (int i = 0; i < n_rounds; ++i) {                      // every thread runs every round: the barriers stay matched
+                if (i + 1 < n_rounds) {
+                    named_barrier(1, wg_threads);                     // everyone has read buffer (i + 1) & 1
+                    if (tid == kAuxThreads) issue_round(i + 1);
                 }
-                if (tid == kAuxThreads) SS_TR(5, 7);
-                if (ok && vi >= 0) {
-                    const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, ri);
-                    const float inv = 1.f / l_c;
+                ok = ok && mbar_wait_warp(smem_u32(&c.merge_full[i & 1]), (i >> 1) & 1, abort_flag, a.status);
+                if (!ok) continue;
+                const uint32_t xb = merge_base + (i & 1) * buf_bytes;
+                // work item: (row of the round, group of four columns)
+                for (int w = tid - kAuxThreads; w < RR * (HD / 4); w += wg_threads) {
+                    const int rr = w / (HD / 4), g = w - rr * (HD / 4);
+                    RowInfo r;
+                    if (!out_row(first + i * RR + rr, r)) continue;
+                    float ms[8], ls[8];
+                    float mx = -INFINITY;
                     #pragma unroll
-                    for (int i = 0; i < QW / 4; ++i) {
-                        uint2 o;
-                        o.x = pack_bf16(acc[i].x * inv, acc[i].y * inv);
-                        o.y = pack_bf16(acc[i].z * inv, acc[i].w * inv);
-                        *reinterpret_cast<uint2*>(dst.o + pidx * QW + i * 4) = o;
-                    }
-                    if (dst.lse && pidx == 0) *dst.lse = (m_c + log2f(l_c)) * 0.6931471805599453f;
-                }
-                if (tid == kAuxThreads) SS_TR(5, 8);
-            } else {
-                // kSingle / kMulti: the partial rows stream through two shared-memory buffers, 32 rows of
-                // every CTA of the pair per round; the copy of round i+1 runs while round i is combined.
-                constexpr int RR = 32;
-                constexpr uint32_t RB = RP * 4;
-                const uint32_t buf_bytes = static_cast<uint32_t>(C) * RR * RB;
-                const size_t cta_stride = static_cast<size_t>(rows_cap) * RP;
-                mbar_wait_warp(smem_u32(&c.q_full), 0, abort_flag, a.status);      // the query copy may alias the buffers
-                int n_rounds = 0;
-                for (int k = 0; k < n_blocks; ++k) n_rounds += (sp.n_valid(k) + RR - 1) / RR;
-                // round -> (block, first valid-row number)
-                auto round_rows = [&](int i, int& blk, int& r0) {
-                    blk = 0;
-                    for (;;) {
-                        const int n = (sp.n_valid(blk) + RR - 1) / RR;
-                        if (i < n) break;
-                        i -= n; ++blk;
-                    }
-                    r0 = i * RR;
-                };
-                auto issue_round = [&](int i) {
-                    int blk, r0;
-                    round_rows(i, blk, r0);
-                    const uint32_t mbar = smem_u32(&c.merge_full[i & 1]);
-                    asm volatile("fence.proxy.async;" ::: "memory");      // generic accesses to the buffer and to the partials come first
-                    mbar_expect_tx(mbar, buf_bytes);
-                    for (int sidx = 0; sidx < C; ++sidx)
-                        bulk_load(merge_base + (i & 1) * buf_bytes + static_cast<uint32_t>(sidx) * RR * RB,
-                                  part_pair + sidx * cta_stride + static_cast<size_t>(blk * kBlockRows + r0) * RP, RR * RB, mbar);
-                };
-                named_barrier(1, wg_threads);                             // every warpgroup is past its pipeline
-                if (tid == kAuxThreads && n_rounds > 0) issue_round(0);
-                bool ok = true;
-                for (int i = 0; i < n_rounds; ++i) {                      // every thread runs every round: the barriers stay matched
-                    if (i + 1 < n_rounds) {
-                        named_barrier(1, wg_threads);                     // everyone has read buffer (i + 1) & 1
-                        if (tid == kAuxThreads) issue_round(i + 1);
-                    }
-                    ok = ok && mbar_wait_warp(smem_u32(&c.merge_full[i & 1]), (i >> 1) & 1, abort_flag, a.status);
-                    if (!ok) continue;
-                    int blk, r0;
-                    round_rows(i, blk, r0);
-                    const int nvr = sp.n_valid(blk);
-                    const uint32_t xb = merge_base + (i & 1) * buf_bytes;
-                    // work item: (row of the round, group of four columns)
-                    for (int w = tid - kAuxThreads; w < RR * (HD / 4); w += wg_threads) {
-                        const int rr = w / (HD / 4), g = w - rr * (HD / 4);
-                        if (r0 + rr >= nvr) continue;
-                        float ms[4], ls[4];
-                        float mx = -INFINITY;
-                        #pragma unroll
-                        for (int sidx = 0; sidx < 4; ++sidx) {
-                            if (sidx < C) {
-                                const float2 t = ld_shared_v2(xb + static_cast<uint32_t>(sidx * RR + rr) * RB + HD * 4u);
-                                ms[sidx] = t.x; ls[sidx] = t.y;
-                                mx = fmaxf(mx, t.x);
-                            }
+                    for (int sidx = 0; sidx < 8; ++sidx) {
+                        if (sidx < C) {
+                            const float2 t = ld_shared_v2(xb + static_cast<uint32_t>(sidx * RR + rr) * RB + HD * 4u);
+                            ms[sidx] = t.x; ls[sidx] = t.y;
+                            mx = fmaxf(mx, t.x);
                         }
-                        float l = 0.f;
-                        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                        #pragma unroll
-                        for (int sidx = 0; sidx < 4; ++sidx) {
-                            if (sidx < C) {
-                                const float wgt = ms[sidx] == -INFINITY ? 0.f : exp2f(ms[sidx] - mx);   // 0: saw no visible key
-                                l += wgt * ls[sidx];
-                                const float4 t = ld_shared_v4(xb + static_cast<uint32_t>(sidx * RR + rr) * RB + g * 16u);
-                                acc.x += wgt * t.x; acc.y += wgt * t.y; acc.z += wgt * t.z; acc.w += wgt * t.w;
-                            }
-                        }
-                        const RowInfo r = row_info(sp, sp.row_of(blk, r0 + rr));
-                        const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, r);
-                        const float inv = 1.f / l;
-                        uint2 o;
-                        o.x = pack_bf16(acc.x * inv, acc.y * inv);
-                        o.y = pack_bf16(acc.z * inv, acc.w * inv);
-                        *reinterpret_cast<uint2*>(dst.o + g * 4) = o;
-                        if (dst.lse && g == 0) *dst.lse = (mx + log2f(l)) * 0.6931471805599453f;
                     }
+                    float l = 0.f;
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    #pragma unroll
+                    for (int sidx = 0; sidx < 8; ++sidx) {
+                        if (sidx < C) {
+                            const float wgt = ms[sidx] == -INFINITY ? 0.f : exp2f(ms[sidx] - mx);   // 0: saw no visible key
+                            l += wgt * ls[sidx];
+                            const float4 t = ld_shared_v4(xb + static_cast<uint32_t>(sidx * RR + rr) * RB + g * 16u);
+                            acc.x += wgt * t.x; acc.y += wgt * t.y; acc.z += wgt * t.z; acc.w += wgt * t.w;
+                        }
+                    }
+                    const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, r);
+                    const float inv = 1.f / l;
+                    uint2 o;
+                    o.x = pack_bf16(acc.x * inv, acc.y * inv);
+                    o.y = pack_bf16(acc.z * inv, acc.w * inv);
+                    *reinterpret_cast<uint2*>(dst.o + g * 4) = o;
+                    if (dst.lse && g == 0) *dst.lse = (mx + log2f(l)) * 0.6931471805599453f;
                 }
             }
         }
@@ -1283,8 +1266,7 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     // CTAs per (sequence, head) pair: the largest power of two that still fits the grid on the SMs in one wave
     const long long pairs = static_cast<long long>(p.batch) * p.n_heads;
     int c = 1;
-    const int c_max = plan->mode == kDual ? 8 : 4;          // the merge of the other variants combines at most four partials
-    while (c < c_max && pairs * (c * 2) <= sm_count()) c *= 2;
+    while (c < 8 && pairs * (c * 2) <= sm_count()) c *= 2;
     plan->cluster = c;
     const int q_smem_rows = plan->mode == kDual ? kBlockRows : q_rows;
     const size_t p_total = plan->mode == kDual ? static_cast<size_t>(2) * 3 * 64 * 128                 // two warpgroups
@@ -1302,10 +1284,11 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     size_t bytes = qp + static_cast<size_t>(plan->n_kslots + plan->n_vslots) * slot;
     if (bytes < qp + overhang) bytes = qp + overhang;
     // kDual stages its four CTA-local partials of every row ((head_dim + 4) floats) once the pipeline is done
-    // (the other variants stream the partials of a split pair through two buffers of 32 rows per CTA of the pair)
-    const size_t stage = plan->mode == kDual ? static_cast<size_t>(4) * 64 * (p.head_dim + 4) * 4
-                                             : static_cast<size_t>(2) * c * 32 * (p.head_dim + 4) * 4;
-    if ((plan->mode == kDual || c > 1) && stage > bytes) bytes = stage;
+    const size_t stage = static_cast<size_t>(4) * 64 * (p.head_dim + 4) * 4;
+    if (plan->mode == kDual && stage > bytes) bytes = stage;
+    // every CTA of a split pair streams its share of the pair's partial rows through two buffers
+    const size_t merge_bufs = static_cast<size_t>(2) * c * (c == 8 ? 16 : 32) * (p.head_dim + 4) * 4;
+    if (c > 1 && merge_bufs > bytes) bytes = merge_bufs;
     plan->smem = bytes + 1024;
     // workspace: one arrival counter per pair; one partial row per (pair, CTA of the pair, query row)
     const size_t rows_cap = plan->mode == kDual ? 64 : static_cast<size_t>(plan->n_blocks) * kBlockRows;
@@ -1397,6 +1380,7 @@ extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
     a.cluster_shift = 0;
     while ((1 << a.cluster_shift) < plan.cluster) ++a.cluster_shift;
     a.head_coord = shared_heads ? 0 : 1;
+    a.prefix_stable = (p->flags & SS_ATTN_PREFIX_STABLE) ? 1 : 0;
     a.scale_log2 = p->sm_scale * 1.4426950408889634f;
     a.o_main = static_cast<__nv_bfloat16*>(p->o_main);
     a.o_spec = static_cast<__nv_bfloat16*>(p->o_spec);

@@ -18,15 +18,19 @@ class DeviceStep:
     """All inputs of one step on the device, with per-layer ss_attn_params prepared once.
 
     layers          layer indices of the workload to materialise (default: all of them)
+    prefix_stable   pass SS_ATTN_PREFIX_STABLE to the attention calls (true for every use in this repo:
+                    what runs before an attention call never writes the cached prefix)
     distinct_slabs  if set, layer l draws its KV slab from random substream (l % distinct_slabs):
                     every layer still owns its own device memory, only the host generation is shared
     """
 
     def __init__(self, st: StepInputs, layers: Optional[List[int]] = None, distinct_slabs: Optional[int] = None,
-                 device: str = "cuda", with_lse: bool = False, pinned_host: bool = False):
+                 device: str = "cuda", with_lse: bool = False, pinned_host: bool = False, prefix_stable: bool = True):
         api.lib()
         c = st.cfg
         self.st, self.cfg, self.device = st, c, device
+        # SS_ATTN_PREFIX_STABLE: nothing in flight before an attention call writes the prefix, lengths or trees
+        self.prefix_stable = prefix_stable
         self.layers = list(range(c.n_layers)) if layers is None else list(layers)
         nl = len(self.layers)
         B, T, H, d, g = c.batch, c.n_nodes, c.n_heads, c.head_dim, c.gamma
@@ -103,7 +107,7 @@ class DeviceStep:
             kv_start=self.kv_start, kv_len=self.kv_len, kv_capacity=self.kv_capacity, trees=self.trees,
             gamma=self.cfg.gamma if msa else 0, sm_scale=self.st.sm_scale,
             q_spec=self.q_spec[i], k_spec=self.k_spec[i], v_spec=self.v_spec[i], o_spec=self.o_spec[i],
-            lse_main=self.lse_main[i], lse_spec=self.lse_spec[i], workspace=ws)
+            lse_main=self.lse_main[i], lse_spec=self.lse_spec[i], workspace=ws, prefix_stable=self.prefix_stable)
 
     # ---- the hot path -------------------------------------------------------------------------
     def run_attention(self, stream=None, only: Optional[List[int]] = None) -> int:

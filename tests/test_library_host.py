@@ -32,7 +32,7 @@ def test_every_declared_symbol_is_exported(lib):
 def test_struct_sizes_match_the_header(lib):
     assert C.sizeof(api.TreeDesc) == 16 + 4 * 64 + 4 * 64 + 8 * 64
     assert C.sizeof(api.CacheLayout) == 40
-    assert C.sizeof(api.AttnParams) == 24 + 8 * 8 + 3 * 8 + 8 * 8
+    assert C.sizeof(api.AttnParams) == 24 + 8 * 8 + 3 * 8 + 8 * 8 + 8      # ... + flags (padded to 8)
 
 
 def test_tree_build_paper_mask_example(lib):
