@@ -1098,10 +1098,12 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
         // Arrive on the pair's counter, then wait (bounded) until the pair's other CTAs have arrived too:
         // they were launched together and need nothing from this CTA, so the wait is short.  Each CTA then
         // combines its own share of the rows, so the tail of the kernel is a C-th of a single merger's.
-        __threadfence();
+        // (the CTA barrier orders every thread's partial stores before the one thread whose device-scope
+        //  fence and arrival then publish them)
         named_barrier(3, wg_threads);
         if (tid == kAuxThreads) {
             unsigned int* cnt = reinterpret_cast<unsigned int*>(a.counters) + pair;
+            __threadfence();
             const unsigned int prev = atomicAdd(cnt, 1u);
             const unsigned int target = (prev | static_cast<unsigned int>(C - 1)) + 1u;   // this call's C arrivals end here
             bool ok = true;
