@@ -187,7 +187,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    from paper_2402_11131_b200 import api, build, workloads as W
+    from paper_2402_11131_b200 import api, build, replicas, workloads as W
     from paper_2402_11131_b200.step import DeviceStep
     if rank == 0:
         build.build()
@@ -276,9 +276,7 @@ def main():
     compact_ms = time_graph(g_compact, K, 3)
     clocks = sampler.stop() if rank == 0 else None
     if world > 1:
-        t = torch.tensor([step_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        step_ms = float(t.item())
+        step_ms = replicas.max_over_ranks(step_ms, "cuda")
         dist.barrier()
     status = api.ss_status(dev.attn_ws, stream) or api.ss_status(dev.verify_ws, stream)
     if status != 0:
@@ -423,9 +421,8 @@ def time_e2e(dev, stream, reps, world):
     torch.cuda.synchronize()
     dt = (time.perf_counter() - t0) / reps
     if world > 1:
-        t = torch.tensor([dt], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dt = float(t.item())
+        from paper_2402_11131_b200 import replicas
+        dt = replicas.max_over_ranks(dt, "cuda")
     acc = dev.accept_len.cpu().numpy()
     step_bytes = (sum(dev.attention_bytes(i) for i in range(nl)) + dev.verify_bytes() + dev.compact_bytes(acc))
     return {"value": world * step_bytes / dt / 1e9, "unit": UNIT, "ms_per_step": dt * 1e3,

@@ -23,7 +23,8 @@
  *   - A workspace must be zero-filled once (cudaMemset) before its first use; each call leaves
  *     it ready for the next.  Word 0 of a workspace is the device status word: a kernel that
  *     detects a broken invariant (sequence over capacity, a wait that ran out) stores its
- *     SS_ERR_* code there and returns instead of faulting.
+ *     SS_ERR_* code there and returns instead of faulting.  After SS_ERR_DEVICE_TIMEOUT the
+ *     workspace's arrival counters are undefined: zero-fill it again before reuse.
  *   - Two calls that share a workspace must not overlap on the device.
  */
 #ifndef SS_MSA_H_
@@ -97,7 +98,11 @@ int32_t ss_tree_build(const int32_t* parent, int32_t n_nodes, int32_t gamma, ss_
  *   lse_main float[batch][max_nodes][n_heads], lse_spec float[batch][max_nodes][gamma][n_heads]:
  *                                  optional natural-log sum-exp of the scaled scores (NULL to skip).
  * Scores are sm_scale * <q, k>; softmax statistics and both products accumulate in fp32.
- * Reads nothing past slot kv_start[b]+L_b+T_b-1; writes only o_*, lse_* and the workspace.
+ * The workspace holds, besides the status word, one arrival counter per (sequence, head) pair and the
+ * partial rows of pairs whose keys are split over several CTAs (ss_msa_attention_workspace_bytes).
+ * Reads no K/V row past slot kv_start[b]+L_b+T_b-1 whose value can reach an output (a tile may touch
+ * later slots of the slab; what it finds there is masked or cleared); writes only o_*, lse_* and the
+ * workspace.
  * If kv_capacity is given and L_b + T_b > kv_capacity[b], sequence b is skipped and the status word
  * is set to SS_ERR_CAPACITY.
  * Errors (nothing launched): SS_ERR_INVALID_ARG, SS_ERR_UNSUPPORTED, SS_ERR_WORKSPACE, SS_ERR_CUDA. */

@@ -1,31 +1,39 @@
 // Tree-masked multi-stream attention, one layer (Eq. 1, Eq. 2): split-KV flash-decode for sm_100a.
 //
-// Work decomposition.  A thread-block cluster of C CTAs owns one (sequence, head) pair.  The pair's
-// keys are the cached slots [0, L+T) (prefix, then this step's tree nodes, masked by ancestry) and
-// the T*gamma transient stream keys (node-major).  They are cut into 16-key units and CTA r of the
-// cluster takes units [U*r/C, U*(r+1)/C), so every CTA of a pair streams the same number of bytes.
+// Work decomposition.  C CTAs (a power of two, chosen so that the grid fills the SMs once) share one
+// (sequence, head) pair.  The pair's keys are the cached slots [0, L+T) (prefix, then this step's tree
+// nodes, masked by ancestry) and the T*gamma transient stream keys (node-major).  They are cut into
+// 16-key units and CTA r takes units [U*r/C, U*(r+1)/C), so every CTA of a pair streams the same number
+// of bytes.
 //
 // Inside a CTA.  ALL query rows of the head -- T main rows, then the T*gamma stream rows -- sit in
 // shared memory as up to three 128-row blocks, so each K/V tile that TMA brings in is used by every
 // (node x stream) row: the prefix crosses HBM once per head, not once per stream.
-//   thread 0    TMA producer: Q once, then K tiles and V tiles into two independent rings
-//               (mbarrier complete_tx); swizzle-128B boxes straight from the caller's strided tensors.
-//               A K slot is handed back as soon as S has been computed, a V slot after P V.
+//   threads 0, 96  TMA producers of the K ring and of the V ring (mbarrier complete_tx); swizzle-128B
+//               boxes straight from the caller's strided tensors.  A K slot is handed back as soon
+//               as S is queued, a V slot after P V.  Thread 0 also requests Q once.
 //   warp 1      tcgen05 issuer of S = Q K^T (128 x TK x d) into one of two TMEM buffers;
-//   warp 2      tcgen05 issuer of O += P V (128 x d x TK) into the block's TMEM accumulator;
+//   warp 2      tcgen05 issuer of O += P V (128 x d x TK) into a TMEM accumulator;
 //               tcgen05.commit arrives on the mbarriers that hand buffers back.  TK = 128 keys when
 //               the head has one row block (N = 128 MMAs run at the full tensor rate), 64 otherwise.
-//   warps 4..   one warpgroup per 128-row block, one thread per query row: tcgen05.ld of the S row,
-//               tree / stream mask from the node's 64-bit ancestor word, online softmax in fp32
-//               registers (the running maximum is only raised when it would grow by more than 2^8,
-//               which keeps the TMEM accumulator untouched on almost every tile), P as bf16 into a
-//               swizzled shared-memory tile that feeds the second MMA.
-// Split-KV merge.  Each CTA ends with un-normalised (m, l, O) per row.  The valid rows of every
-// block are dealt out to the C CTAs of the cluster: all CTAs push a row's partial into the shared
-// memory of the CTA that merges it (st.shared::cluster), one cluster barrier, then that CTA combines
-// the C partials and writes bf16 output.  No CTA ever spins on another: the only cross-CTA waits are
-// hardware cluster barriers that every thread reaches unconditionally; every mbarrier wait is
-// bounded and reports SS_ERR_DEVICE_TIMEOUT.
+//   warps 4..   softmax warpgroups, one thread per TMEM lane: tcgen05.ld of the S row, tree / stream
+//               mask from the node's 64-bit ancestor word, online softmax in fp32 registers (the
+//               running maximum is only raised when it would grow by more than 2^8, which keeps the
+//               TMEM accumulator untouched on almost every tile), P as bf16 into a swizzled
+//               shared-memory tile that feeds the second MMA.
+// Three variants (enum Mode) map rows to warpgroups: one warpgroup per 128-row block (up to three
+// blocks); one block of 65..128 rows; and, for heads of at most 64 rows, the rows twice in one block
+// (the two copies split every tile's keys) with two warpgroups ping-ponging on alternate tiles.
+//
+// Split-KV merge.  Each CTA ends with un-normalised (m, l, O) per row, combines what it holds for a
+// row locally, and leaves one partial row in the workspace (it stays in L2).  It then arrives on the
+// pair's counter and waits, bounded, for the pair's other CTAs (launched with it, needing nothing
+// from it); each CTA combines its own share of the rows and writes bf16 output.
+//
+// Launch.  Programmatic dependent launch: one thread of each CTA waits for the previous kernel of
+// the stream; before that wait the kernel touches global memory only under the caller's
+// SS_ATTN_PREFIX_STABLE promise (lengths, trees and wholly-prefix K/V tiles).  Every wait in the
+// kernel is bounded and reports SS_ERR_DEVICE_TIMEOUT.
 #include <cuda.h>
 #include <cuda_bf16.h>
 

@@ -201,6 +201,47 @@ def test_attention_strided_cache_views(cuda, oracle):
     assert_attention_close(oracle, st, st.layer(0), dev, 0)
 
 
+def test_attention_without_the_prefix_promise_gives_the_same_bits(cuda, oracle):
+    """flags = 0 (nothing read before the dependency wait) and SS_ATTN_PREFIX_STABLE differ only in
+    when the prefix tiles are requested: the outputs are bit-identical, for every kernel variant
+    (<= 64 rows, one block of 65..128 rows, several blocks)."""
+    api, DeviceStep = cuda
+    cases = [dict(prefix_len=700, n_nodes=16, gamma=3, max_depth=3, n_heads=8, head_dim=128),      # 64 rows
+             dict(prefix_len=500, n_nodes=32, gamma=3, max_depth=4, n_heads=6, head_dim=64),       # 128 rows
+             dict(prefix_len=400, n_nodes=40, gamma=4, max_depth=4, n_heads=5, head_dim=80)]       # 200 rows
+    for k, kw in enumerate(cases):
+        cfg = W.custom_config("promise%d" % k, n_layers=2, n_msa_layers=1, config_id=640 + k, **kw)
+        st = W.make_step(cfg)
+        outs = []
+        for promise in (False, True):
+            dev = DeviceStep(st, prefix_stable=promise)
+            for _ in range(2):                                  # back to back: the second call overlaps the first
+                dev.run_attention()
+            assert api.ss_status(dev.attn_ws) == 0
+            outs.append([dev.o_main[0].clone(), dev.o_main[1].clone(), dev.o_spec[1].clone()])
+            if promise:
+                for i in range(2):
+                    assert_attention_close(oracle, st, st.layer(i), dev, i)
+        for x, y in zip(*outs):
+            assert torch.equal(x.view(torch.int16), y.view(torch.int16))
+
+
+@pytest.mark.parametrize("n_heads,expect_split", [(1, 8), (3, 8), (20, 4), (40, 2), (100, 1)])
+def test_attention_every_split_factor(cuda, oracle, n_heads, expect_split):
+    """The number of CTAs per (sequence, head) pair follows the head count (8, 4, 2, 1): every merge
+    path, including pairs whose CTAs get no keys at all (8 CTAs, 5 key units)."""
+    api, DeviceStep = cuda
+    for k, (L, T, g) in enumerate([(70, 6, 1), (900, 40, 4)]):
+        cfg = W.custom_config("split%d_%d" % (n_heads, k), n_layers=2, n_msa_layers=1, prefix_len=L, n_nodes=T,
+                              gamma=g, max_depth=3, n_heads=n_heads, head_dim=64, config_id=660 + k)
+        st = W.make_step(cfg)
+        dev = DeviceStep(st, with_lse=True)
+        dev.run_attention()
+        assert api.ss_status(dev.attn_ws) == 0
+        for i in range(2):
+            assert_attention_close(oracle, st, st.layer(i), dev, i, check_lse=True)
+
+
 # ---- verification ---------------------------------------------------------------------------------
 def _verify_and_compare(api, dev, st, oracle):
     dev.run_verify()
