@@ -66,7 +66,7 @@ constexpr int kBlockRows = 128;      // query rows per block (M of both MMAs)
 constexpr int kMaxBlocks = 3;        // 64 main rows + 256 stream rows = 320 rows at most
 constexpr int kMaxSlots = 4;         // slots per ring (K ring, V ring)
 constexpr int kAuxThreads = 128;     // warps 0..3: producer, MMA issuer, two spare
-constexpr int kMaxDynSmem = 232448 - 4096;  // 227 KB per CTA less the static control block
+constexpr int kMaxDynSmem = 232448 - 1024;  // 227 KB per CTA less the static control block
 constexpr float kRescaleStep = 8.f;  // raise the running maximum only when it grows by more than 2^8
 constexpr long long kWaitCycles = 2000000000ll;   // bound of every mbarrier wait (~1 s)
 
@@ -185,6 +185,14 @@ __device__ __forceinline__ float2 ld_shared_v2(uint32_t addr) {
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// shared memory -> contiguous global memory; the calling thread commits and waits for the whole group
+__device__ __forceinline__ void bulk_store(void* dst, uint32_t src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_store_wait_all() {
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -967,6 +975,9 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     // row, later the partials of the pair's CTAs.  A thread combines one quarter of its row's columns;
     // with `carry` the running (m, l, acc) counts as one more source.
     const uint32_t x_base = merge_base;
+    constexpr uint32_t RB = RP * 4;                                            // bytes of a partial row
+    // outgoing partial rows of this CTA, as they lie in the workspace (kDual: after the staging area)
+    const uint32_t y_base = merge_base + (MODE == kDual ? 4u * 64u * RB : 0u);
     auto combine_x = [&](int n_src, bool carry, float& m_c, float& l_c, float4 (&acc)[QW / 4]) {
         constexpr uint32_t RBx = RP * 4;
         float w[4], mp[4], lp[4];
@@ -1047,10 +1058,13 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                         if (dst.lse && pidx == 0) *dst.lse = (m_out + log2f(l_out)) * 0.6931471805599453f;
                     }
                 } else {
-                    float* dst = part_mine + static_cast<size_t>(lrow) * RP;     // same row order as the staging area
+                    // the partial row goes to the outgoing area Y, in the staging area's row order
+                    const uint32_t yrow = y_base + static_cast<uint32_t>(lrow) * RB;
                     #pragma unroll
-                    for (int i = 0; i < QW / 4; ++i) __stcg(reinterpret_cast<float4*>(dst + pidx * QW + i * 4), acc[i]);
-                    if (pidx == 0) __stcg(reinterpret_cast<float2*>(dst + HD), make_float2(m_out, l_out));
+                    for (int i = 0; i < QW / 4; ++i)
+                        st_shared_v4(yrow + static_cast<uint32_t>(pidx * QW + i * 4) * 4u, __float_as_uint(acc[i].x), __float_as_uint(acc[i].y),
+                                     __float_as_uint(acc[i].z), __float_as_uint(acc[i].w));
+                    if (pidx == 0) st_shared_v4(yrow + HD * 4u, __float_as_uint(m_out), __float_as_uint(l_out), 0u, 0u);
                 }
             }
             if (tid == kAuxThreads) SS_TR(5, 3);
@@ -1083,7 +1097,9 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             }
         }
     } else {
-        // kSingle / kMulti, split pair: every thread stores its row's partial
+        // kSingle / kMulti, split pair: every thread stores its row's partial straight from TMEM (a
+        // warpgroup that is done does not wait for the others; staging the rows in shared memory first
+        // would, and measured slower)
         if (warp >= 4 && __any_sync(0xffffffffu, vi >= 0)) {
             float* dst = part_mine + static_cast<size_t>(rblk * kBlockRows + (vi >= 0 ? vi : 0)) * RP;
             #pragma unroll
@@ -1106,11 +1122,18 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
         // Arrive on the pair's counter, then wait (bounded) until the pair's other CTAs have arrived too:
         // they were launched together and need nothing from this CTA, so the wait is short.  Each CTA then
         // combines its own share of the rows, so the tail of the kernel is a C-th of a single merger's.
-        // (the CTA barrier orders every thread's partial stores before the one thread whose device-scope
-        //  fence and arrival then publish them)
+        // The CTA barrier orders every thread's partial rows before the one thread whose device-scope fence
+        // and arrival publish them.  kDual: the rows wait in Y and that thread ships them to the workspace
+        // in whole lines with one bulk copy.
+        if (MODE == kDual) fence_async_smem();
         named_barrier(3, wg_threads);
         if (tid == kAuxThreads) {
             unsigned int* cnt = reinterpret_cast<unsigned int*>(a.counters) + pair;
+            if (MODE == kDual) {
+                bulk_store(part_mine, y_base, 64u * RB);
+                bulk_store_wait_all();
+                asm volatile("fence.proxy.async;" ::: "memory");
+            }
             __threadfence();
             const unsigned int prev = atomicAdd(cnt, 1u);
             const unsigned int target = (prev | static_cast<unsigned int>(C - 1)) + 1u;   // this call's C arrivals end here
@@ -1289,13 +1312,16 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     int slots = static_cast<int>((kMaxDynSmem - 1024 - qp) / slot);
     if (slots > 2 * kMaxSlots) slots = 2 * kMaxSlots;
     if (slots < 4) return false;
-    plan->n_kslots = slots / 2 > 2 ? 2 : slots / 2;          // K comes back right after S: two slots suffice
+    // a K slot is held until every row block has its S queued, a V slot until the last P V: split evenly
+    plan->n_kslots = slots / 2 > kMaxSlots ? kMaxSlots : slots / 2;
     plan->n_vslots = slots - plan->n_kslots > kMaxSlots ? kMaxSlots : slots - plan->n_kslots;
     size_t bytes = qp + static_cast<size_t>(plan->n_kslots + plan->n_vslots) * slot;
     if (bytes < qp + overhang) bytes = qp + overhang;
     // kDual stages its four CTA-local partials of every row ((head_dim + 4) floats) once the pipeline is done
-    const size_t stage = static_cast<size_t>(4) * 64 * (p.head_dim + 4) * 4;
-    if (plan->mode == kDual && stage > bytes) bytes = stage;
+    // after the pipeline kDual stages its four CTA-local partials of every row and the outgoing row (5 x 64 rows)
+    const size_t row_bytes = static_cast<size_t>(p.head_dim + 4) * 4;
+    const size_t stage = plan->mode == kDual ? 5 * 64 * row_bytes : 0;
+    if (stage > bytes) bytes = stage;
     // every CTA of a split pair streams its share of the pair's partial rows through two buffers
     const size_t merge_bufs = static_cast<size_t>(2) * c * (c == 8 ? 16 : 32) * (p.head_dim + 4) * 4;
     if (c > 1 && merge_bufs > bytes) bytes = merge_bufs;
