@@ -307,7 +307,9 @@ def main():
                    "parallelism": "replicas" if world > 1 else "single_gpu",
                    "l2": "every layer streams its own KV slab; a step touches %.0f MB, far more than the 126 MB L2"
                          % (step_bytes / 1e6),
-                   "launch": "whole step replayed as one CUDA graph"},
+                   "launch": "whole step replayed as one CUDA graph; attention launched with programmatic dependent launch",
+                   "attention_flags": "SS_ATTN_PREFIX_STABLE (nothing in flight before an attention call writes a cached prefix)",
+                   "component_timings": "us_plain_layer / us_msa_layer stream a different slab per launch (cold); us_verify / us_compact replay one kernel on L2-warm data"},
         "step_bytes": step_bytes, "pct_of_8TBs": value / world / 8000.0 * 100,
         "us_per_layer": attn_ms * 1e3 / nl,
         "us_plain_layer": None if plain_ms is None else plain_ms * 1e3 / len(plain_idx),
@@ -319,7 +321,9 @@ def main():
         "clocks": clocks,
         "roofline": {"kernel": "msa_attention_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
-                     "bytes_per_launch": attn_bytes / nl, "us_per_launch": attn_launch_us, "traffic": ncu_traffic()},
+                     "bytes_per_launch": attn_bytes / nl, "us_per_launch": attn_launch_us,
+                     "timed": "CUDA events around replays of a graph of the step's %d attention launches, right after the timed region" % nl,
+                     "traffic": ncu_traffic() if args.workload == "7b" else None},
         "e2e": e2e,
     }
     if not args.no_cpu_baseline and world == 1:
