@@ -1,34 +1,37 @@
-// Tree-masked multi-stream attention, one layer (Eq. 1, Eq. 2): split-KV flash-decode for sm_100a.
+// Tree-masked multi-stream attention, one layer (Eq. 1, Eq. 2): flash-decode for sm_100a.
 //
-// Work decomposition.  C CTAs (a power of two, chosen so that the grid fills the SMs once) share one
-// (sequence, head) pair.  The pair's keys are the cached slots [0, L+T) (prefix, then this step's tree
-// nodes, masked by ancestry) and the T*gamma transient stream keys (node-major).  They are cut into
-// 16-key units and CTA r takes units [U*r/C, U*(r+1)/C), so every CTA of a pair streams the same number
-// of bytes.
+// Work decomposition.  The query rows of a (sequence, head) pair -- T main rows, then the T*gamma
+// stream rows -- form one tile when there are at most 64 of them, else blocks of 128 rows that go to
+// separate CTAs (a block streams the keys it can see: the cached slots, and the stream keys of its own
+// nodes).  C CTAs (a power of two, chosen so that the grid fills the SMs once) share the keys of a
+// block: the cached slots [0, L+T) (prefix, then this step's tree nodes, masked by ancestry) and the
+// block's transient stream keys (node-major) are cut into 16-key units and CTA r takes units
+// [U*r/C, U*(r+1)/C), so every CTA of a block streams the same number of bytes.  The CTAs of a pair
+// run in the same wave, so a K/V tile crosses HBM once and is served from L2 to the other row blocks.
 //
-// Inside a CTA.  ALL query rows of the head -- T main rows, then the T*gamma stream rows -- sit in
-// shared memory as up to three 128-row blocks, so each K/V tile that TMA brings in is used by every
-// (node x stream) row: the prefix crosses HBM once per head, not once per stream.
+// Inside a CTA.
 //   threads 0, 96  TMA producers of the K ring and of the V ring (mbarrier complete_tx); swizzle-128B
 //               boxes straight from the caller's strided tensors.  A K slot is handed back as soon
 //               as S is queued, a V slot after P V.  Thread 0 also requests Q once.
-//   warp 1      tcgen05 issuer of S = Q K^T (128 x TK x d) into one of two TMEM buffers;
-//   warp 2      tcgen05 issuer of O += P V (128 x d x TK) into a TMEM accumulator;
-//               tcgen05.commit arrives on the mbarriers that hand buffers back.  TK = 128 keys when
-//               the head has one row block (N = 128 MMAs run at the full tensor rate), 64 otherwise.
-//   warps 4..   softmax warpgroups, one thread per TMEM lane: tcgen05.ld of the S row, tree / stream
-//               mask from the node's 64-bit ancestor word, online softmax in fp32 registers (the
-//               running maximum is only raised when it would grow by more than 2^8, which keeps the
-//               TMEM accumulator untouched on almost every tile), P as bf16 into a swizzled
-//               shared-memory tile that feeds the second MMA.
-// Three variants (enum Mode) map rows to warpgroups: one warpgroup per 128-row block (up to three
-// blocks); one block of 65..128 rows; and, for heads of at most 64 rows, the rows twice in one block
-// (the two copies split every tile's keys) with two warpgroups ping-ponging on alternate tiles.
+//   warp 1      tcgen05 issuer of S = Q K^T (128 x 128 keys x d) into one of two TMEM buffers;
+//   warp 2      tcgen05 issuer of O += P V into the TMEM accumulator of a warpgroup;
+//               tcgen05.commit arrives on the mbarriers that hand buffers back.
+//   warps 4..11 two softmax warpgroups, one thread per TMEM lane: tcgen05.ld of 64 scores of the row,
+//               tree / stream mask from the node's 64-bit ancestor word, online softmax in fp32
+//               registers (the running maximum is only raised when it would grow by more than 2^8,
+//               which keeps the TMEM accumulator untouched on almost every tile), P as bf16 into a
+//               swizzled shared-memory tile that feeds the second MMA.
+// Two variants (enum Mode) map rows and keys to the warpgroups.  kPair: a block of up to 128 rows; of
+// every 128-key tile warpgroup 0 takes keys 0..63 and warpgroup 1 keys 64..127, each with its own P
+// tile, running maximum and accumulator.  kDual, for heads of at most 64 rows: the block holds the
+// rows twice (copy 0 takes keys 0..63, copy 1 keys 64..127) and the two warpgroups take alternate
+// tiles.  Either way all four sub-partitions of the SM share a tile's exponentials.
 //
 // Split-KV merge.  Each CTA ends with un-normalised (m, l, O) per row, combines what it holds for a
-// row locally, and leaves one partial row in the workspace (it stays in L2).  It then arrives on the
-// pair's counter and waits, bounded, for the pair's other CTAs (launched with it, needing nothing
-// from it); each CTA combines its own share of the rows and writes bf16 output.
+// row locally, and -- when the keys were split -- leaves one partial row in the workspace (it stays in
+// L2).  It then arrives on the block's counter and waits, bounded, for the other CTAs of the block
+// (launched with it, needing nothing from it); each CTA combines its own share of the rows and writes
+// bf16 output.
 //
 // Launch.  Programmatic dependent launch: one thread of each CTA waits for the previous kernel of
 // the stream; before that wait the kernel touches global memory only under the caller's
@@ -63,22 +66,24 @@ __device__ __forceinline__ unsigned long long wall_ns() {
 
 constexpr int kUnit = 16;            // split granularity (keys)
 constexpr int kBlockRows = 128;      // query rows per block (M of both MMAs)
-constexpr int kMaxBlocks = 3;        // 64 main rows + 256 stream rows = 320 rows at most
+constexpr int kTileKeys = 128;       // keys per tile: N = 128 MMAs run at the full tensor rate
 constexpr int kMaxSlots = 4;         // slots per ring (K ring, V ring)
-constexpr int kAuxThreads = 128;     // warps 0..3: producer, MMA issuer, two spare
+constexpr int kAuxThreads = 128;     // warps 0..3: producers and MMA issuers
 constexpr int kMaxDynSmem = 232448 - 1024;  // 227 KB per CTA less the static control block
 constexpr float kRescaleStep = 8.f;  // raise the running maximum only when it grows by more than 2^8
 constexpr long long kWaitCycles = 2000000000ll;   // bound of every mbarrier wait (~1 s)
 
 struct alignas(64) AttnArgs {
-    CUtensorMap tm_k, tm_v;          // cache slab    dims (d, H, slots)        box (64, 1, TK)
+    CUtensorMap tm_k, tm_v;          // cache slab    dims (d, H, slots)        box (64, 1, 128)
     CUtensorMap tm_qm;               // q_main        dims (d, H, B*Tmax)       box (64, 1, tmax8)
-    CUtensorMap tm_qs;               // q_spec        dims (d, H, B*Tmax*g)     box (64, 1, spec_rows)
-    CUtensorMap tm_ks, tm_vs;        // k_spec/v_spec dims (d, H, B*Tmax*g)     box (64, 1, TK)
+    CUtensorMap tm_qs;               // q_spec        dims (d, H, B*Tmax*g)     box (64, 1, s0rows): stream rows of block 0
+    CUtensorMap tm_qs1;              // q_spec        the same tensor           box (64, 1, 128): later row blocks
+    CUtensorMap tm_ks, tm_vs;        // k_spec/v_spec dims (d, H, B*Tmax*g)     box (64, 1, 128)
     int batch, n_heads, gamma, max_nodes;
-    int tmax8;                       // max_nodes rounded up to 8: first stream row in shared memory
-    int spec_rows;                   // max_nodes * gamma rounded up to 8 (rows of the q_spec box)
-    int n_blocks, cluster, cluster_shift;   // cluster = 1 << cluster_shift
+    int tmax8;                       // max_nodes rounded up to 8: first stream row of the head's query tile
+    int s0rows;                      // stream rows that share block 0 with the main rows
+    int n_blocks;                    // 128-row blocks per head (kPair), 1 for kDual
+    int cluster, cluster_shift;      // CTAs that share a block's keys; cluster = 1 << cluster_shift
     int n_kslots, n_vslots;          // ring depths
     int head_coord;                  // 1, or 0 when all heads share one K/V (head stride 0)
     int prefix_stable;               // the caller's SS_ATTN_PREFIX_STABLE promise
@@ -92,21 +97,21 @@ struct alignas(64) AttnArgs {
     const int* kv_capacity;
     const ss_tree_desc* trees;
     int* status;
-    int* counters;                   // [pairs] arrivals of a pair's CTAs (zero between calls)
-    float* partials;                 // [pairs][splits][rows][head_dim + 4]
+    int* counters;                   // [groups] arrivals of a block's CTAs (monotonic)
+    float* partials;                 // [groups][splits][rows][head_dim + 4]
 };
 
 struct Ctrl {
     unsigned long long q_full;
     unsigned long long k_full[kMaxSlots], k_empty[kMaxSlots], v_full[kMaxSlots], v_empty[kMaxSlots];
-    unsigned long long s_full[kMaxBlocks][2];   // per (block, S buffer): a warpgroup sees every phase of its own
+    unsigned long long s_full[2][2];            // per (warpgroup, S buffer): a warpgroup sees every phase of its own
     unsigned long long s_free[2];
-    unsigned long long p_full[kMaxBlocks], o_done[kMaxBlocks];
+    unsigned long long p_full[2], o_done[2];    // per warpgroup
     unsigned long long anc[SS_MAX_NODES];
     uint32_t tmem_base;
     int abort;
-    int merge_ok;                // the pair's other CTAs arrived in time
-    unsigned long long merge_full[2];   // a batch of the pair's partials has been copied into shared memory
+    int merge_ok;                // the block's other CTAs arrived in time
+    unsigned long long merge_full[2];   // a batch of the block's partials has been copied into shared memory
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -269,52 +274,23 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int n, bool b_mn_major) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// The CTA's share of the pair's keys, as a list of tiles of TK keys.  Every role derives it from
-// the same few numbers, so no tile list is ever stored.
-template <int TK>
+// The CTA's share of its row block's keys, as a list of tiles of kTileKeys keys.  Every role derives
+// it from the same few numbers, so no tile list is ever stored.
 struct Span {
-    int L, T, n_stream;            // prefix length, tree nodes, stream keys (T * gamma)
+    int L, T, n_stream;            // prefix length, tree nodes, stream keys of the sequence (T * gamma)
     int kc0, kc1;                  // cache keys [kc0, kc1) (indices into [0, L+T))
     int ks0, ks1;                  // stream keys [ks0, ks1) (indices into [0, T*gamma))
     int n_cache_tiles, n_tiles;
-    int tmax8, gamma, n_blocks;
-    int spec_end;                  // valid rows: [0, T) and [tmax8, spec_end)
-    unsigned valid_blocks;         // bit b set: row block b holds a valid row
-    bool pingpong;                 // one row block served by two warpgroups that take alternate tiles
+    int tmax8, gamma;
+    int spec_end;                  // valid rows of the head: [0, T) and [tmax8, spec_end)
+    int row0;                      // first row of this CTA's block
 
     __device__ __forceinline__ bool is_cache(int j) const { return j < n_cache_tiles; }
     __device__ __forceinline__ int first_key(int j) const {
-        return j < n_cache_tiles ? kc0 + j * TK : ks0 + (j - n_cache_tiles) * TK;
+        return j < n_cache_tiles ? kc0 + j * kTileKeys : ks0 + (j - n_cache_tiles) * kTileKeys;
     }
     __device__ __forceinline__ int valid_keys(int j) const {
-        return min(TK, (j < n_cache_tiles ? kc1 : ks1) - first_key(j));
-    }
-    // bit b set: row block b holds a row that can see a key of tile j
-    __device__ __forceinline__ unsigned active_mask(int j) const {
-        if (pingpong) return 1u << (j & 1);
-        if (j < n_cache_tiles) return valid_blocks;
-        // stream key s is seen by the stream rows s .. (end of its node's group)
-        const int s0 = first_key(j), s_last = s0 + valid_keys(j) - 1;
-        const int row_lo = tmax8 + s0, row_hi = tmax8 + (s_last / gamma) * gamma + gamma - 1;
-        unsigned m = 0;
-        for (int b = 0; b < n_blocks; ++b)
-            if (row_lo < (b + 1) * kBlockRows && row_hi >= b * kBlockRows) m |= 1u << b;
-        return m;
-    }
-    // valid rows of a block, numbered 0 .. n_valid-1 (main rows first, then stream rows)
-    __device__ __forceinline__ int main_in_block(int blk) const { return blk == 0 ? T : 0; }
-    __device__ __forceinline__ int n_valid(int blk) const {
-        const int r0 = blk * kBlockRows, r1 = r0 + kBlockRows;
-        return main_in_block(blk) + max(0, min(spec_end, r1) - max(tmax8, r0));
-    }
-    __device__ __forceinline__ int valid_index(int row) const {      // -1 for a padding row
-        const int blk = row / kBlockRows, r0 = blk * kBlockRows;
-        if (row < tmax8) return row < T ? row - r0 : -1;
-        return row < spec_end ? main_in_block(blk) + row - max(tmax8, r0) : -1;
-    }
-    __device__ __forceinline__ int row_of(int blk, int vi) const {
-        const int r0 = blk * kBlockRows, mb = main_in_block(blk);
-        return vi < mb ? r0 + vi : max(tmax8, r0) + (vi - mb);
+        return min(kTileKeys, (j < n_cache_tiles ? kc1 : ks1) - first_key(j));
     }
 };
 
@@ -327,57 +303,31 @@ struct Ring {
     }
 };
 
-// (tile, block) items in tile-major order, only the active ones
-struct ItemIter {
-    int j;
-    unsigned m;
-    template <class S>
-    __device__ __forceinline__ void begin(const S& sp) {
-        j = 0;
-        m = sp.n_tiles > 0 ? sp.active_mask(0) : 0u;
-        skip_empty(sp);
-    }
-    template <class S>
-    __device__ __forceinline__ void skip_empty(const S& sp) {
-        while (m == 0u && j < sp.n_tiles) {
-            ++j;
-            m = j < sp.n_tiles ? sp.active_mask(j) : 0u;
-        }
-    }
-    template <class S>
-    __device__ __forceinline__ bool done(const S& sp) const { return j >= sp.n_tiles; }
-    __device__ __forceinline__ int blk() const { return __ffs(m) - 1; }
-    __device__ __forceinline__ bool last_of_tile() const { return (m & (m - 1u)) == 0u; }
-    template <class S>
-    __device__ __forceinline__ void next(const S& sp) {
-        m &= m - 1u;
-        skip_empty(sp);
-    }
-};
-
-template <int TK>
-__device__ __forceinline__ Span<TK> make_span(const AttnArgs& a, int L, int T, int rank, bool pingpong) {
-    Span<TK> s;
-    s.pingpong = pingpong;
-    s.L = L; s.T = T; s.gamma = a.gamma; s.tmax8 = a.tmax8; s.n_blocks = a.n_blocks;
+__device__ __forceinline__ Span make_span(const AttnArgs& a, int L, int T, int rank, int rb) {
+    Span s;
+    s.L = L; s.T = T; s.gamma = a.gamma; s.tmax8 = a.tmax8;
     s.n_stream = T * a.gamma;
     s.spec_end = a.tmax8 + s.n_stream;
-    const int ec = L + T;
-    const int uc = (ec + kUnit - 1) / kUnit, us = (s.n_stream + kUnit - 1) / kUnit;
+    s.row0 = rb * kBlockRows;
+    // stream rows [x0, x1) of the block (numbered from the first stream row); row x = (node, stream) sees
+    // the stream keys node*gamma .. x, so the block sees the keys from its first node's first stream on
+    const int x0 = max(s.row0, s.tmax8) - s.tmax8, x1 = min(s.row0 + kBlockRows, s.spec_end) - s.tmax8;
+    int slo = 0, shi = 0;
+    if (x1 > x0) { slo = x0 / a.gamma * a.gamma; shi = x1; }
+    const bool any_row = s.row0 < T || x1 > x0;           // a block without a valid row streams nothing
+    const int ec = any_row ? L + T : 0;
+    const int uc = (ec + kUnit - 1) / kUnit, us = (shi - slo + kUnit - 1) / kUnit;
     const int u = uc + us;
-    // u < 2^28 and rank < 8: the products fit 32 bits; the cluster size is a power of two
+    // u < 2^28 and rank < 8: the products fit 32 bits; the split factor is a power of two
     const int u0 = static_cast<int>((static_cast<unsigned>(u) * static_cast<unsigned>(rank)) >> a.cluster_shift);
     const int u1 = static_cast<int>((static_cast<unsigned>(u) * static_cast<unsigned>(rank + 1)) >> a.cluster_shift);
     s.kc0 = min(u0, uc) * kUnit;
     s.kc1 = min(min(u1, uc) * kUnit, ec);
-    s.ks0 = (max(u0, uc) - uc) * kUnit;
-    s.ks1 = min((max(u1, uc) - uc) * kUnit, s.n_stream);
-    s.n_cache_tiles = s.kc1 > s.kc0 ? (s.kc1 - s.kc0 + TK - 1) / TK : 0;
-    const int nst = s.ks1 > s.ks0 ? (s.ks1 - s.ks0 + TK - 1) / TK : 0;
+    s.ks0 = slo + (max(u0, uc) - uc) * kUnit;
+    s.ks1 = min(slo + (max(u1, uc) - uc) * kUnit, shi);
+    s.n_cache_tiles = s.kc1 > s.kc0 ? (s.kc1 - s.kc0 + kTileKeys - 1) / kTileKeys : 0;
+    const int nst = s.ks1 > s.ks0 ? (s.ks1 - s.ks0 + kTileKeys - 1) / kTileKeys : 0;
     s.n_tiles = s.n_cache_tiles + nst;
-    s.valid_blocks = 0;
-    for (int b = 0; b < a.n_blocks; ++b)
-        if (s.n_valid(b) > 0) s.valid_blocks |= 1u << b;
     return s;
 }
 
@@ -387,8 +337,7 @@ struct RowInfo {
     bool valid;
     int node, stream;              // stream 0 = main row, 1..gamma = speculative stream
 };
-template <int TK>
-__device__ __forceinline__ RowInfo row_info(const Span<TK>& s, int row) {
+__device__ __forceinline__ RowInfo row_info(const Span& s, int row) {
     RowInfo r;
     if (row < s.tmax8) {
         r.valid = row < s.T; r.node = row; r.stream = 0;
@@ -464,30 +413,32 @@ __device__ __forceinline__ float chunk_exp_store(const uint32_t (&v)[64], float 
     return (sum[0] + sum[1]) + (sum[2] + sum[3]);
 }
 
-// Kernel variants.  kMulti: up to three 128-row blocks, 64-key tiles.  kSingle: one block of 65..128
-// rows, 128-key tiles.  kDual: at most 64 rows: the block holds the rows twice, copy 0 takes keys
-// 0..63 of every 128-key tile and copy 1 keys 64..127 (P is zero in the other half), so all four
-// sub-partitions share the exponentials; and two warpgroups, each with its own accumulator, take
-// alternate tiles, so one tile's softmax overlaps the other's MMAs.  The four partials a row then has
-// inside the CTA are combined before the cluster-wide merge.
-enum Mode { kMulti = 0, kSingle = 1, kDual = 2 };
+// Kernel variants.  kPair: a block of up to 128 rows; warpgroup w takes keys 64w .. 64w+63 of every
+// tile, with its own P tile (64 keys wide), running maximum and accumulator.  kDual: at most 64 rows:
+// the block holds the rows twice, copy 0 takes keys 0..63 of a tile and copy 1 keys 64..127 (P is zero
+// in the other half), and the two warpgroups, each with its own accumulator, take alternate tiles, so
+// one tile's softmax overlaps the other's MMAs.  The partials a row then has inside the CTA (two, four)
+// are combined before the merge across CTAs.
+enum Mode { kPair = 0, kDual = 2 };
 
 template <int HD, int MODE>
 struct Geo {
-    static constexpr int TK = MODE == kMulti ? 64 : 128;          // keys per tile
     static constexpr int kHalves = HD > 64 ? 2 : 1;               // 64-element boxes along head_dim
-    static constexpr int kBoxBytes = TK * 128;                    // one TMA box: TK rows x 128 B
+    static constexpr int kBoxBytes = kTileKeys * 128;             // one TMA box: 128 keys x 128 B
     static constexpr int kSlotBytes = kHalves * kBoxBytes;        // one K tile (or one V tile)
     static constexpr int kKSteps = HD / 16;                       // MMA K steps of S = Q K^T
-    static constexpr int kMergePitch = HD + 4;                    // floats per row in the merge buffer
-    static constexpr uint32_t kIdescS = idesc_bf16(TK, false);
+    static constexpr int kMergePitch = HD + 4;                    // floats per partial row: O, m, l, pad
+    static constexpr uint32_t kIdescS = idesc_bf16(kTileKeys, false);
     static constexpr uint32_t kIdescPV = idesc_bf16(HD, true);
-    static constexpr int kOCols = 128;                            // TMEM columns reserved per block accumulator
-    static constexpr int kWGs = MODE == kMulti ? kMaxBlocks : (MODE == kDual ? 2 : 1);   // softmax warpgroups
-    static constexpr int kThreads = kAuxThreads + kWGs * kBlockRows;
+    static constexpr int kOCols = 128;                            // TMEM columns reserved per accumulator
+    static constexpr int kThreads = kAuxThreads + 2 * kBlockRows; // two softmax warpgroups
     static constexpr int kCopies = MODE == kDual ? 2 : 1;
-    static constexpr int kRowBytes = kMergePitch * 4;             // one merge row: O, then (m, l)
-    static constexpr int kChunks = MODE == kSingle ? 2 : 1;       // 64-key chunks of a tile one thread handles
+    // P of one warpgroup, 128 B rows of 64 keys (swizzled).  kPair: 128 rows.  kDual: [copy-0 rows 0..63 |
+    // 64 zero rows | copy-1 rows 0..63]; the MMA reads keys 0..63 from the first 128 rows and keys 64..127
+    // from the last 128 rows, so each copy's other half is zero.
+    static constexpr uint32_t kPBytes = MODE == kDual ? 3u * 64u * 128u : 128u * 128u;
+    static constexpr int kRowsCap = MODE == kDual ? 64 : kBlockRows;   // partial rows a CTA ships
+    static constexpr int kSplitCol = ((HD / 16 + 1) / 2) * 16;    // kPair: warpgroup 0 finishes columns [0, kSplitCol)
 };
 
 // destination of a row's output and log-sum-exp
@@ -510,20 +461,32 @@ __device__ __forceinline__ OutPtr out_ptr(const AttnArgs& a, int b, int h, long 
     return p;
 }
 
+// 16 fp32 values scaled and packed to bf16 -> 32 bytes at dst
+__device__ __forceinline__ void store_bf16x16(__nv_bfloat16* dst, const float (&v)[16]) {
+    uint4 lo, hi;
+    lo.x = pack_bf16(v[0], v[1]);   lo.y = pack_bf16(v[2], v[3]);   lo.z = pack_bf16(v[4], v[5]);   lo.w = pack_bf16(v[6], v[7]);
+    hi.x = pack_bf16(v[8], v[9]);   hi.y = pack_bf16(v[10], v[11]); hi.z = pack_bf16(v[12], v[13]); hi.w = pack_bf16(v[14], v[15]);
+    *reinterpret_cast<uint4*>(dst) = lo;
+    *reinterpret_cast<uint4*>(dst + 8) = hi;
+}
+
 // ---------------------------------------------------------------------------------------------
 template <int HD, int MODE>
 __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kernel(const __grid_constant__ AttnArgs a) {
     using G = Geo<HD, MODE>;
-    constexpr int TK = G::TK;
+    constexpr int TK = kTileKeys;
+    constexpr bool kIsDual = MODE == kDual;
     extern __shared__ unsigned char smem_raw[];
     __shared__ Ctrl c;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int C = a.cluster;
     const uint32_t rank = blockIdx.x & (C - 1);            // C is a power of two
-    const int pair = blockIdx.x >> a.cluster_shift;
+    const int group = blockIdx.x >> a.cluster_shift;       // (pair, row block): the CTAs that share its keys
+    const int rb = kIsDual ? 0 : group % a.n_blocks;
+    const int pair = kIsDual ? group : group / a.n_blocks;
     const int b = pair / a.n_heads, h = pair - b * a.n_heads;
-    const int n_blocks = a.n_blocks, nk = a.n_kslots, nv_slots = a.n_vslots;
+    const int nk = a.n_kslots, nv_slots = a.n_vslots;
     volatile int* abort_flag = &c.abort;
 
     if (tid == 0) SS_TR(0, 0);
@@ -542,22 +505,14 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     }
 #endif
     // ---- shared-memory carve-up (1024-byte aligned: swizzle atoms) ----------------------------
-    // Q and P keep only the rows that exist; an MMA that reads the rows of a 128-row block past them
-    // picks up whatever follows in shared memory, which only ever reaches padding rows of S and O.
+    // The query tile always has room for 128 rows; rows past the ones that exist hold whatever shared
+    // memory held, which only ever reaches padding rows of S and O.
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t q_rows = a.tmax8 + a.spec_rows;                      // rows of the head's query tile
-    const uint32_t q_smem_rows = MODE == kDual ? kBlockRows : q_rows;   // kDual: second copy at row 64
-    // P of one warpgroup, 128 B rows of 64 keys (swizzled).  kMulti / kSingle: [key half][p_rows].
-    // kDual: [copy-0 rows 0..63 | 64 zero rows | copy-1 rows 0..63]; the MMA reads keys 0..63 from the
-    // first 128 rows and keys 64..127 from the last 128 rows, so each copy's other half is zero.
-    const uint32_t p_rows = MODE == kMulti ? kBlockRows : q_rows;
-    const uint32_t p_half = MODE == kDual ? 64u * 128u : p_rows * 128u;    // byte offset of the second key half
-    const uint32_t p_bytes = MODE == kDual ? 3u * 64u * 128u : (TK / 64) * p_rows * 128u;
-    const int n_acc = MODE == kDual ? 2 : n_blocks;                        // accumulators = warpgroups in use
-    const uint32_t q_base = base;                                       // [half][q_smem_rows][128 B]
-    const uint32_t p_base = q_base + G::kHalves * q_smem_rows * 128u;   // [warpgroup][p_bytes]
-    const uint32_t k_base = p_base + n_acc * p_bytes;                   // [slot][half][TK][128 B]
-    const uint32_t v_base = k_base + nk * G::kSlotBytes;                // [slot][half][TK][128 B]
+    constexpr uint32_t kQHalfBytes = kBlockRows * 128u;
+    const uint32_t q_base = base;                                       // [half][128 rows][128 B]; kDual: second copy at row 64
+    const uint32_t p_base = q_base + G::kHalves * kQHalfBytes;          // [warpgroup][kPBytes]
+    const uint32_t k_base = p_base + 2u * G::kPBytes;                   // [slot][half][128 keys][128 B]
+    const uint32_t v_base = k_base + nk * G::kSlotBytes;                // [slot][half][128 keys][128 B]
     const uint32_t merge_base = base;                                   // aliases everything above, after the main loop
     const long long spec_row0 = static_cast<long long>(b) * a.max_nodes * a.gamma;   // first stream row of the sequence
 
@@ -570,7 +525,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
         c.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         tma_prefetch_desc(&a.tm_qm); tma_prefetch_desc(&a.tm_k);
-        if (a.gamma > 0) { tma_prefetch_desc(&a.tm_qs); tma_prefetch_desc(&a.tm_ks); }
+        if (a.gamma > 0) { tma_prefetch_desc(&a.tm_qs); tma_prefetch_desc(&a.tm_qs1); tma_prefetch_desc(&a.tm_ks); }
     } else if (tid == 96) {                               // V producer
         for (int s = 0; s < kMaxSlots; ++s) mbar_init(smem_u32(&c.v_full[s]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -579,12 +534,13 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     } else if (tid == 64) {                               // every other barrier (first used after the CTA-wide sync)
         for (int s = 0; s < kMaxSlots; ++s) { mbar_init(smem_u32(&c.k_empty[s]), 1); mbar_init(smem_u32(&c.v_empty[s]), 1); }
         for (int s = 0; s < 2; ++s) {
-            mbar_init(smem_u32(&c.s_free[s]), 4);
-            for (int k = 0; k < kMaxBlocks; ++k) mbar_init(smem_u32(&c.s_full[k][s]), 1);
+            mbar_init(smem_u32(&c.s_free[s]), kIsDual ? 4 : 8);          // warps that read an S buffer
+            mbar_init(smem_u32(&c.s_full[0][s]), 1);
+            mbar_init(smem_u32(&c.s_full[1][s]), 1);
+            mbar_init(smem_u32(&c.p_full[s]), kBlockRows);
+            mbar_init(smem_u32(&c.o_done[s]), 1);
+            mbar_init(smem_u32(&c.merge_full[s]), 1);
         }
-        for (int s = 0; s < kMaxBlocks; ++s) { mbar_init(smem_u32(&c.p_full[s]), kBlockRows); mbar_init(smem_u32(&c.o_done[s]), 1); }
-        mbar_init(smem_u32(&c.merge_full[0]), 1);
-        mbar_init(smem_u32(&c.merge_full[1]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (tid == 0) SS_TR(0, 1);
@@ -604,7 +560,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     // first prefix tiles requested right away, so HBM streams while the previous kernel drains.
     if (!a.prefix_stable) dependency_wait();
     if (tid == 0) SS_TR(0, 2);
-    constexpr uint32_t kTmemCols = 512;
+    constexpr uint32_t kTmemCols = 512;                   // two accumulators and two S buffers of 128 columns
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&c.tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -622,7 +578,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     }
     if (tid == 0) SS_TR(0, 3);
 
-    const Span<TK> sp = make_span<TK>(a, L, T, static_cast<int>(rank), MODE == kDual);
+    const Span sp = make_span(a, L, T, static_cast<int>(rank), rb);
 
     // K tile j / V tile j of the span -> ring slot st (K: thread 0, V: thread 96)
     auto load_k = [&](int j, int st) {
@@ -662,17 +618,23 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     }
     if (skip && tid == 0) set_status(a.status, SS_ERR_CAPACITY);
     if (tid == 0) {
-        // the rest of the first tiles, then the queries
+        // the rest of the first tiles, then the queries of the block
         for (int j = n_pre; j < n_early_k; ++j) load_k(j, j);
         const uint32_t qbar = smem_u32(&c.q_full);
-        mbar_expect_tx(qbar, G::kCopies * G::kHalves * q_rows * 128u);
+        const bool with_spec = a.gamma > 0 && a.s0rows > 0;
+        const uint32_t rows = rb > 0 ? kBlockRows : a.tmax8 + (with_spec ? a.s0rows : 0);
+        mbar_expect_tx(qbar, G::kCopies * G::kHalves * rows * 128u);
         #pragma unroll
         for (int cp = 0; cp < G::kCopies; ++cp) {
             #pragma unroll
             for (int hh = 0; hh < G::kHalves; ++hh) {
-                const uint32_t dst = q_base + hh * q_smem_rows * 128u + cp * 64u * 128u;
-                tma_load_3d(dst, &a.tm_qm, hh * 64, h, b * a.max_nodes, qbar);
-                if (a.gamma > 0) tma_load_3d(dst + a.tmax8 * 128u, &a.tm_qs, hh * 64, h, static_cast<int>(spec_row0), qbar);
+                const uint32_t dst = q_base + hh * kQHalfBytes + cp * 64u * 128u;
+                if (rb > 0) {
+                    tma_load_3d(dst, &a.tm_qs1, hh * 64, h, static_cast<int>(spec_row0 + rb * kBlockRows - a.tmax8), qbar);
+                } else {
+                    tma_load_3d(dst, &a.tm_qm, hh * 64, h, b * a.max_nodes, qbar);
+                    if (with_spec) tma_load_3d(dst + a.tmax8 * 128u, &a.tm_qs, hh * 64, h, static_cast<int>(spec_row0), qbar);
+                }
             }
         }
     } else if (tid == 96) {
@@ -681,9 +643,9 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     if (tid >= kAuxThreads && tid < kAuxThreads + SS_MAX_NODES) c.anc[tid - kAuxThreads] = __ldcg(&a.trees[b].anc_mask[tid - kAuxThreads]);
     if (tid == 0) SS_TR(0, 5);
     // kDual: the 64 zero rows in the middle of each warpgroup's P stay zero for the whole kernel
-    if (MODE == kDual && tid >= kAuxThreads) {
+    if (kIsDual && tid >= kAuxThreads) {
         const int r = tid - kAuxThreads;                                  // 256 threads, 64 B each per warpgroup
-        const uint32_t dst = p_base + (r >> 7) * p_bytes + 64u * 128u + (r & 127) * 64u;
+        const uint32_t dst = p_base + (r >> 7) * G::kPBytes + 64u * 128u + (r & 127) * 64u;
         #pragma unroll
         for (int i = 0; i < 4; ++i) st_shared_v4(dst + i * 16, 0u, 0u, 0u, 0u);
         fence_async_smem();
@@ -692,8 +654,20 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = c.tmem_base;
-    const uint32_t tmem_s = tmem + n_acc * G::kOCols;     // two S buffers of TK columns
+    const uint32_t tmem_s = tmem + 2 * G::kOCols;         // two S buffers of 128 columns
     if (tid == 0) SS_TR(0, 6);
+
+    // per-thread partial of this CTA's key span, kept for the merge (softmax warps only)
+    float m_run = -INFINITY, l_run = 0.f;
+    int n_own = 0;
+    const int wg = (warp - 4) >> 2;                                           // softmax warpgroup 0 / 1
+    const int row_in_blk = ((warp & 3) << 5) | lane;                          // TMEM lane of this thread
+    const int copy = kIsDual ? (row_in_blk >> 6) : 0;
+    const int lrow = kIsDual ? (row_in_blk & 63) : row_in_blk;                // row of the block this thread works for
+    const int chunk = kIsDual ? copy : wg;                                    // 64-key half of a tile this thread handles
+    const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    RowInfo ri;
+    ri.valid = false; ri.node = 0; ri.stream = 0;
 
     // ============================ warp 0: K producer, warp 3: V producer ==========================
     // Two rings, two threads: a K slot comes back as soon as S is queued, a V slot only after P V, and
@@ -726,148 +700,120 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             if (!ok) for (int s = 0; s < nv_slots; ++s) mbar_drain(smem_u32(&c.v_full[s]), (s < rv.slot ? rv.round : rv.round - 1) & 1);
         }
     }
-    // ============================ warp 1: issues S = Q K^T =========================================
+    // ============================ warp 1: issues S = Q K^T, one MMA group per tile ================
     else if (warp == 1) {
         if (lane == 0) {
             // the query tile is always requested, so it is always awaited (shared memory is reused later)
             bool ok = mbar_wait(smem_u32(&c.q_full), 0, abort_flag, a.status);
             if (!ok) mbar_drain(smem_u32(&c.q_full), 0);
             SS_TR(1, 0);
-            ItemIter it = {0, 0u};
-            it.begin(sp);
             Ring rk;
             rk.start();
-            int k_tile = it.j;                            // tile the ring position belongs to
-            for (int i = 0; i < k_tile; ++i) rk.advance(nk);
-            bool k_seen = false;
-            for (int q = 0; ok && !it.done(sp); ++q, it.next(sp)) {
-                const int j = it.j, blk = it.blk(), buf = q & 1;
-                while (k_tile < j) { rk.advance(nk); ++k_tile; k_seen = false; }
-                if (!k_seen) {
-                    if (!mbar_wait(smem_u32(&c.k_full[rk.slot]), rk.round & 1, abort_flag, a.status)) break;
-                    k_seen = true;
-                }
-                SS_TR(1, 8 + 4 * q);
-                if (q >= 2 && !mbar_wait(smem_u32(&c.s_free[buf]), ((q >> 1) - 1) & 1, abort_flag, a.status)) break;
-                SS_TR(1, 9 + 4 * q);
+            for (int j = 0; ok && j < sp.n_tiles; ++j, rk.advance(nk)) {
+                const int buf = j & 1;
+                if (!mbar_wait(smem_u32(&c.k_full[rk.slot]), rk.round & 1, abort_flag, a.status)) break;
+                SS_TR(1, 8 + 4 * j);
+                if (j >= 2 && !mbar_wait(smem_u32(&c.s_free[buf]), ((j >> 1) - 1) & 1, abort_flag, a.status)) break;
+                SS_TR(1, 9 + 4 * j);
                 tc_fence_after();
-                const uint32_t qa = q_base + (MODE == kDual ? 0 : blk) * (kBlockRows * 128u);
                 const uint32_t ka = k_base + rk.slot * G::kSlotBytes;
                 #pragma unroll
                 for (int ks = 0; ks < G::kKSteps; ++ks) {
                     const uint32_t hh = ks >> 2, off = (ks & 3) * 32u;
-                    tc_mma(tmem_s + buf * TK, desc_k_major(qa + hh * q_smem_rows * 128u + off),
+                    tc_mma(tmem_s + buf * TK, desc_k_major(q_base + hh * kQHalfBytes + off),
                            desc_k_major(ka + hh * G::kBoxBytes + off), G::kIdescS, ks > 0);
                 }
-                SS_TR(1, 10 + 4 * q);
-                tc_commit(smem_u32(&c.s_full[blk][buf]));
-                if (it.last_of_tile()) tc_commit(smem_u32(&c.k_empty[rk.slot]));     // every S of tile j is queued: K may go
-                SS_TR(1, 11 + 4 * q);
+                SS_TR(1, 10 + 4 * j);
+                if (kIsDual) {
+                    tc_commit(smem_u32(&c.s_full[buf][buf]));            // tile j belongs to warpgroup j & 1
+                } else {
+                    tc_commit(smem_u32(&c.s_full[0][buf]));
+                    tc_commit(smem_u32(&c.s_full[1][buf]));
+                }
+                tc_commit(smem_u32(&c.k_empty[rk.slot]));                // S of tile j is queued: K may go
+                SS_TR(1, 11 + 4 * j);
             }
         }
     }
     // ============================ warp 2: issues O += P V ==========================================
     else if (warp == 2) {
         if (lane == 0) {
-            ItemIter it = {0, 0u};
-            it.begin(sp);
-            int n_done0 = 0, n_done1 = 0, n_done2 = 0;   // PV batches issued per block
             Ring rv;
             rv.start();
-            int v_tile = it.j;
-            for (int i = 0; i < v_tile; ++i) rv.advance(nv_slots);
-            bool v_seen = false;
-            int tq = 0;
-            for (; !it.done(sp); it.next(sp), ++tq) {
-                const int j = it.j, blk = it.blk();
-                const int nd = blk == 0 ? n_done0 : (blk == 1 ? n_done1 : n_done2);
-                while (v_tile < j) { rv.advance(nv_slots); ++v_tile; v_seen = false; }
-                if (!v_seen) {
-                    if (!mbar_wait(smem_u32(&c.v_full[rv.slot]), rv.round & 1, abort_flag, a.status)) break;
-                    v_seen = true;
-                }
-                SS_TR(2, 8 + 4 * tq);
-                if (!mbar_wait(smem_u32(&c.p_full[blk]), nd & 1, abort_flag, a.status)) break;
-                SS_TR(2, 9 + 4 * tq);
-                tc_fence_after();
-                const uint32_t pa = p_base + blk * p_bytes;
+            bool ok = true;
+            for (int j = 0; ok && j < sp.n_tiles; ++j, rv.advance(nv_slots)) {
+                if (!mbar_wait(smem_u32(&c.v_full[rv.slot]), rv.round & 1, abort_flag, a.status)) break;
+                SS_TR(2, 8 + 4 * j);
                 const uint32_t va = v_base + rv.slot * G::kSlotBytes;
-                #pragma unroll
-                for (int ks = 0; ks < TK / 16; ++ks)
-                    tc_mma(tmem + blk * G::kOCols, desc_k_major(pa + (ks >> 2) * p_half + (ks & 3) * 32u),
-                           desc_mn_major(va + ks * 2048u, G::kBoxBytes), G::kIdescPV, (nd > 0 || ks > 0) ? 1u : 0u);
-                SS_TR(2, 10 + 4 * tq);
-                tc_commit(smem_u32(&c.o_done[blk]));
-                if (it.last_of_tile()) tc_commit(smem_u32(&c.v_empty[rv.slot]));     // last block of tile j: V may go
-                if (blk == 0) ++n_done0; else if (blk == 1) ++n_done1; else ++n_done2;
-                SS_TR(2, 11 + 4 * tq);
+                if (kIsDual) {
+                    // the whole tile for warpgroup j & 1: keys 0..63 from copy 0's rows, 64..127 from copy 1's
+                    const int w = j & 1;
+                    if (!mbar_wait(smem_u32(&c.p_full[w]), (j >> 1) & 1, abort_flag, a.status)) break;
+                    SS_TR(2, 9 + 4 * j);
+                    tc_fence_after();
+                    const uint32_t pa = p_base + w * G::kPBytes;
+                    #pragma unroll
+                    for (int ks = 0; ks < TK / 16; ++ks)
+                        tc_mma(tmem + w * G::kOCols, desc_k_major(pa + (ks >> 2) * (64u * 128u) + (ks & 3) * 32u),
+                               desc_mn_major(va + ks * 2048u, G::kBoxBytes), G::kIdescPV, (j >= 2 || ks > 0) ? 1u : 0u);
+                    tc_commit(smem_u32(&c.o_done[w]));
+                } else {
+                    // keys 64w .. 64w+63 into the accumulator of warpgroup w
+                    #pragma unroll
+                    for (int w = 0; w < 2; ++w) {
+                        if (!mbar_wait(smem_u32(&c.p_full[w]), j & 1, abort_flag, a.status)) { ok = false; break; }
+                        if (w == 0) SS_TR(2, 9 + 4 * j);
+                        tc_fence_after();
+                        const uint32_t pa = p_base + w * G::kPBytes;
+                        #pragma unroll
+                        for (int ks = 0; ks < 4; ++ks)
+                            tc_mma(tmem + w * G::kOCols, desc_k_major(pa + ks * 32u),
+                                   desc_mn_major(va + (w * 4 + ks) * 2048u, G::kBoxBytes), G::kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
+                        tc_commit(smem_u32(&c.o_done[w]));
+                    }
+                    if (!ok) break;
+                }
+                SS_TR(2, 10 + 4 * j);
+                tc_commit(smem_u32(&c.v_empty[rv.slot]));                // P V of tile j is queued: V may go when it completes
+                SS_TR(2, 11 + 4 * j);
             }
         }
     }
-    // ============================ warps 4..: softmax warpgroups =================================
-    // per-thread partial of this CTA's key span, kept for the merge
-    float m_run = -INFINITY, l_run = 0.f;
-    int n_own = 0;
-    const int my_blk = (warp - 4) >> 2;
-    const int row_in_blk = ((warp & 3) << 5) | lane;                          // TMEM lane of this thread
-    const int copy = MODE == kDual ? (row_in_blk >> 6) : 0;
-    const int lrow = MODE == kDual ? (row_in_blk & 63) : row_in_blk;          // row of the block this thread works for
-    const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    RowInfo ri;
-    ri.valid = false; ri.node = 0; ri.stream = 0;
-    const int rblk = MODE == kDual ? 0 : my_blk;                              // row block (kDual: both warpgroups serve block 0)
-    if (warp >= 4) {
-        ri = row_info(sp, rblk * kBlockRows + lrow);
+    // ============================ warps 4..11: softmax warpgroups ==============================
+    else if (warp >= 4) {
+        ri = row_info(sp, sp.row0 + lrow);
         const unsigned long long anc = ri.valid ? c.anc[ri.node] : 0ull;
         // a warp whose 32 rows are all padding skips the arithmetic but keeps the barrier protocol
         const bool warp_active = __any_sync(0xffffffffu, ri.valid);
-        const uint32_t o_addr = tmem + lane_base + my_blk * G::kOCols;
-        const uint32_t p_row = MODE == kDual ? p_base + my_blk * p_bytes + copy * (128u * 128u) + lrow * 128u
-                                             : p_base + my_blk * p_bytes + row_in_blk * 128u;
-        const bool p_row_ok = MODE == kDual || static_cast<uint32_t>(row_in_blk) < p_rows;   // rows past p_rows are padding: never stored
-        ItemIter it = {0, 0u};
-        it.begin(sp);
-        int prev_tile = -1;
-        int n_use0 = 0, n_use1 = 0;                    // S buffers of this block consumed so far, per buffer
-        Ring rv;                                       // V ring position of tile v_tile
+        const uint32_t o_addr = tmem + lane_base + wg * G::kOCols;
+        const uint32_t p_row = kIsDual ? p_base + wg * G::kPBytes + copy * (128u * 128u) + lrow * 128u
+                                       : p_base + wg * G::kPBytes + row_in_blk * 128u;
+        Ring rv;                                       // V ring position of tile j
         rv.start();
-        int v_tile = it.j;
-        for (int i = 0; i < v_tile; ++i) rv.advance(nv_slots);
-        for (int q = 0; !it.done(sp); ++q, it.next(sp)) {
-            const int j = it.j;
-            const bool first_of_tile = (j != prev_tile);
-            prev_tile = j;
+        int v_tile = 0;
+        for (int j = kIsDual ? wg : 0; j < sp.n_tiles; j += kIsDual ? 2 : 1) {
             while (v_tile < j) { rv.advance(nv_slots); ++v_tile; }
-            if (it.blk() != my_blk) continue;
-            const int buf = q & 1;
-            if (!mbar_wait_warp(smem_u32(&c.s_full[my_blk][buf]), (buf ? n_use1 : n_use0) & 1, abort_flag, a.status)) break;
-            if (buf) ++n_use1; else ++n_use0;
-            [[maybe_unused]] const int trole = 3 + my_blk;
-            [[maybe_unused]] const bool tr_on = row_in_blk == 0 && my_blk < 2;
+            const int buf = j & 1;
+            // uses of (warpgroup, buffer) so far: j >> 1 in either variant
+            if (!mbar_wait_warp(smem_u32(&c.s_full[wg][buf]), (j >> 1) & 1, abort_flag, a.status)) break;
+            [[maybe_unused]] const int trole = 3 + wg;
+            [[maybe_unused]] const bool tr_on = row_in_blk == 0;
             if (tr_on) SS_TR(trole, 8 + 6 * n_own);
             tc_fence_after();
-            const uint32_t s_addr = tmem_s + lane_base + buf * TK;
+            const uint32_t s_addr = tmem_s + lane_base + buf * TK + chunk * 64;
             const int x = sp.first_key(j), nvk = sp.valid_keys(j);
             const bool cache = sp.is_cache(j);
             const bool masked = !cache || x + TK > sp.L || nvk < TK;
-            // chunk ch of this thread covers keys x + 64 * (copy + ch) ...
-            unsigned long long vis[G::kChunks];
-            #pragma unroll
-            for (int ch = 0; ch < G::kChunks; ++ch)
-                vis[ch] = masked ? visible_mask(cache, x + (copy + ch) * 64, nvk - (copy + ch) * 64, sp.L, sp.gamma, ri, anc) : ~0ull;
+            const unsigned long long vis = masked ? visible_mask(cache, x + chunk * 64, nvk - chunk * 64, sp.L, sp.gamma, ri, anc) : ~0ull;
 
             uint32_t sr[64];
             float corr = 1.f;
             bool need = false;
-            // ---- pass 1: the tile's maximum ----------------------------------------------------------
+            // ---- pass 1: the maximum of this thread's 64 scores ----------------------------------------
             if (warp_active) {
-                float mx = -INFINITY;
-                #pragma unroll
-                for (int ch = 0; ch < G::kChunks; ++ch) {
-                    tmem_ld64(s_addr + (copy + ch) * 64, sr);
-                    tmem_wait_ld();
-                    mx = fmaxf(mx, masked ? chunk_max<true>(sr, a.scale_log2, vis[ch]) : chunk_max<false>(sr, a.scale_log2, 0ull));
-                }
+                tmem_ld64(s_addr, sr);
+                tmem_wait_ld();
+                const float mx = masked ? chunk_max<true>(sr, a.scale_log2, vis) : chunk_max<false>(sr, a.scale_log2, 0ull);
                 need = mx > m_run + kRescaleStep;
                 if (need) {
                     corr = exp2f(m_run - mx);           // 0 when nothing was visible so far
@@ -876,15 +822,14 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 }
             }
             if (tr_on) SS_TR(trole, 9 + 6 * n_own);
-            if (G::kChunks == 1) {                      // the scores stay in registers: S can be overwritten
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&c.s_free[buf]));
-            }
-            // the previous PV of this block must be complete: it read the P tile that is about to
+            // the scores stay in registers: S can be overwritten
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&c.s_free[buf]));
+            // the previous PV of this warpgroup must be complete: it read the P tile that is about to
             // be overwritten, and it wrote the accumulator that a raised maximum rescales
             if (n_own > 0) {
-                if (!mbar_wait_warp(smem_u32(&c.o_done[my_blk]), (n_own - 1) & 1, abort_flag, a.status)) break;
+                if (!mbar_wait_warp(smem_u32(&c.o_done[wg]), (n_own - 1) & 1, abort_flag, a.status)) break;
                 tc_fence_after();
             }
             if (tr_on) SS_TR(trole, 10 + 6 * n_own);
@@ -903,38 +848,22 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 }
                 // ---- pass 2: P = exp2(S - m) as bf16, row sum -------------------------------------------
                 const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
-                float sum = 0.f;
-                #pragma unroll
-                for (int ch = 0; ch < G::kChunks; ++ch) {
-                    if (G::kChunks > 1) {
-                        tmem_ld64(s_addr + ch * 64, sr);
-                        tmem_wait_ld();
-                    }
-                    if (p_row_ok) {
-                        const uint32_t dst = p_row + ch * p_half;
-                        sum += masked ? chunk_exp_store<true>(sr, a.scale_log2, m_use, vis[ch], dst, row_in_blk)
-                                      : chunk_exp_store<false>(sr, a.scale_log2, m_use, 0ull, dst, row_in_blk);
-                    }
-                }
-                l_run += sum;
+                l_run += masked ? chunk_exp_store<true>(sr, a.scale_log2, m_use, vis, p_row, row_in_blk)
+                                : chunk_exp_store<false>(sr, a.scale_log2, m_use, 0ull, p_row, row_in_blk);
             }
             if (tr_on) SS_TR(trole, 11 + 6 * n_own);
-            if (G::kChunks > 1) {                       // both passes have read S
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&c.s_free[buf]));
-            }
             // V rows past the end of the sequence's keys may hold anything (even NaN patterns): P is 0
-            // there, but 0 * NaN is NaN, so the first block to use such a tile clears them.  Rows that
-            // only lie past this CTA's share of the keys are real data and need nothing.
+            // there, but 0 * NaN is NaN, so the warpgroup clears the ones its P V reads (kDual: the whole
+            // tile, kPair: its half).  Rows that only lie past this CTA's share of the keys are real data.
             const int region_left = (cache ? sp.L + sp.T : sp.n_stream) - x;      // real rows in the tile
-            if (first_of_tile && region_left < TK) {
+            const int fix_lo = max(region_left, kIsDual ? 0 : wg * 64), fix_hi = kIsDual ? TK : wg * 64 + 64;
+            if (fix_lo < fix_hi) {
                 if (!mbar_wait_warp(smem_u32(&c.v_full[rv.slot]), rv.round & 1, abort_flag, a.status)) break;
                 const uint32_t vdst = v_base + rv.slot * G::kSlotBytes;
                 constexpr int kPieceShift = G::kHalves == 2 ? 4 : 3;              // 16-byte pieces per row: 8 per half
-                const int n_pieces = (TK - region_left) << kPieceShift;
+                const int n_pieces = (fix_hi - fix_lo) << kPieceShift;
                 for (int i = row_in_blk; i < n_pieces; i += kBlockRows) {
-                    const int r = region_left + (i >> kPieceShift), pc = i & ((1 << kPieceShift) - 1);
+                    const int r = fix_lo + (i >> kPieceShift), pc = i & ((1 << kPieceShift) - 1);
                     const uint32_t dst = vdst + (pc >> 3) * G::kBoxBytes + r * 128u + ((pc & 7) << 4);
                     asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
                 }
@@ -942,86 +871,78 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             if (tr_on) SS_TR(trole, 12 + 6 * n_own);
             fence_async_smem();
             tc_fence_before();
-            mbar_arrive(smem_u32(&c.p_full[my_blk]));
+            mbar_arrive(smem_u32(&c.p_full[wg]));
             if (tr_on) SS_TR(trole, 13 + 6 * n_own);
             ++n_own;
         }
-        // the block's last PV must have landed in TMEM before the accumulator is read
+        // the warpgroup's last PV must have landed in TMEM before the accumulator is read
         if (n_own > 0) {
-            mbar_wait_warp(smem_u32(&c.o_done[my_blk]), (n_own - 1) & 1, abort_flag, a.status);
+            mbar_wait_warp(smem_u32(&c.o_done[wg]), (n_own - 1) & 1, abort_flag, a.status);
             tc_fence_after();
         }
     }
     if (tid == kAuxThreads) SS_TR(5, 0);
-    __syncwarp();     // the single-lane roles of warps 0..2 rejoin their warps
+    __syncwarp();     // the single-lane roles of warps 0..3 rejoin their warps
 
     // ======================================== epilogue ==========================================
-    // Every CTA of a split pair leaves one un-normalised partial (O, m, l) per valid row in the
-    // workspace (it stays in L2); the CTA that arrives last on the pair's counter combines them and
-    // writes the output.  Nobody waits for anybody: the other CTAs exit at once and free their SMs.
+    // The softmax warpgroups combine the partials a row has inside the CTA.  Not split (C == 1): that
+    // is the result.  Split: every CTA leaves one un-normalised partial row (O, m, l) per query row in
+    // the workspace (it stays in L2), arrives on the block's counter, waits for the others and combines
+    // its own share of the rows.
     const bool has_acc = (warp >= 4) && n_own > 0;     // otherwise the partial is (m = -inf, l = 0, O = 0)
-    const uint32_t o_addr = tmem + lane_base + (warp >= 4 ? my_blk : 0) * G::kOCols;
+    const uint32_t o_addr = tmem + lane_base + (warp >= 4 ? wg : 0) * G::kOCols;
     constexpr int RP = G::kMergePitch;                                         // floats per partial row: O, m, l, pad
-    constexpr int QW = HD / 4;                                                 // columns one thread combines (kDual)
-    const int rows_cap = MODE == kDual ? 64 : n_blocks * kBlockRows;           // partial rows per CTA
-    float* const part_pair = a.partials + static_cast<size_t>(pair) * C * rows_cap * RP;
-    float* const part_mine = part_pair + static_cast<size_t>(rank) * rows_cap * RP;
-    const int wg_threads = G::kWGs * kBlockRows;
-    // row of the partial this thread is responsible for (block-local valid-row number), -1: none
-    const int vi = (warp >= 4 && ri.valid) ? sp.valid_index(rblk * kBlockRows + lrow) : -1;
-    const int pidx = my_blk * 2 + copy;                                        // kDual: partial of the row inside the CTA
-
-    // kDual staging area X: [source][64 rows][RP floats]; sources are the four CTA-local partials of a
-    // row, later the partials of the pair's CTAs.  A thread combines one quarter of its row's columns;
-    // with `carry` the running (m, l, acc) counts as one more source.
-    const uint32_t x_base = merge_base;
     constexpr uint32_t RB = RP * 4;                                            // bytes of a partial row
-    // outgoing partial rows of this CTA, as they lie in the workspace (kDual: after the staging area)
-    const uint32_t y_base = merge_base + (MODE == kDual ? 4u * 64u * RB : 0u);
-    auto combine_x = [&](int n_src, bool carry, float& m_c, float& l_c, float4 (&acc)[QW / 4]) {
-        constexpr uint32_t RBx = RP * 4;
+    constexpr int QW = HD / 4;                                                 // columns one thread combines (kDual)
+    constexpr int rows_cap = G::kRowsCap;                                      // partial rows per CTA
+    constexpr int wg_threads = 2 * kBlockRows;
+    float* const part_group = a.partials + static_cast<size_t>(group) * C * rows_cap * RP;
+    float* const part_mine = part_group + static_cast<size_t>(rank) * rows_cap * RP;
+    const int pidx = wg * 2 + copy;                                            // kDual: partial of the row inside the CTA
+
+    // kDual staging area X: [source][64 rows][RP floats], the four CTA-local partials of a row.  A thread
+    // combines one quarter of its row's columns.
+    const uint32_t x_base = merge_base;
+    // outgoing partial rows of this CTA, as they lie in the workspace (kDual: after the staging area;
+    // kPair: after the 2 KB in which the warpgroups exchange their (m, l))
+    const uint32_t y_base = merge_base + (kIsDual ? 4u * 64u * RB : 2048u);
+    auto combine_x = [&](float& m_c, float& l_c, float4 (&acc)[QW / 4]) {
         float w[4], mp[4], lp[4];
-        float m_new = carry ? m_c : -INFINITY;
+        float m_new = -INFINITY;
         #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            if (k < n_src) {
-                const float2 t = ld_shared_v2(x_base + static_cast<uint32_t>(k * 64 + lrow) * RBx + HD * 4u);
-                mp[k] = t.x; lp[k] = t.y;
-                m_new = fmaxf(m_new, t.x);
-            }
+            const float2 t = ld_shared_v2(x_base + static_cast<uint32_t>(k * 64 + lrow) * RB + HD * 4u);
+            mp[k] = t.x; lp[k] = t.y;
+            m_new = fmaxf(m_new, t.x);
         }
-        const float wc = (carry && m_c != -INFINITY) ? exp2f(m_c - m_new) : 0.f;
-        float l_new = wc * l_c;
+        float l_new = 0.f;
         #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            w[k] = (k < n_src && mp[k] != -INFINITY) ? exp2f(mp[k] - m_new) : 0.f;     // 0: saw no visible key
-            if (k < n_src) l_new += w[k] * lp[k];
+            w[k] = mp[k] != -INFINITY ? exp2f(mp[k] - m_new) : 0.f;     // 0: saw no visible key
+            l_new += w[k] * lp[k];
         }
         #pragma unroll
         for (int i = 0; i < QW / 4; ++i) {
             const uint32_t col = static_cast<uint32_t>(pidx * QW + i * 4) * 4u;
-            float4 r = carry ? make_float4(acc[i].x * wc, acc[i].y * wc, acc[i].z * wc, acc[i].w * wc) : make_float4(0.f, 0.f, 0.f, 0.f);
+            float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
             #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                if (k < n_src) {
-                    const float4 t = ld_shared_v4(x_base + static_cast<uint32_t>(k * 64 + lrow) * RBx + col);
-                    r.x += w[k] * t.x; r.y += w[k] * t.y; r.z += w[k] * t.z; r.w += w[k] * t.w;
-                }
+                const float4 t = ld_shared_v4(x_base + static_cast<uint32_t>(k * 64 + lrow) * RB + col);
+                r.x += w[k] * t.x; r.y += w[k] * t.y; r.z += w[k] * t.z; r.w += w[k] * t.w;
             }
             acc[i] = r;
         }
         m_c = m_new;
         l_c = l_new;
     };
-    if (MODE == kDual) {
-        if (warp >= 4) {
-            // The staging area overlaps the query tile, P and the K/V slots: the query copy must have
-            // landed and every MMA of the CTA must be complete before it is written.
-            mbar_wait_warp(smem_u32(&c.q_full), 0, abort_flag, a.status);
+    if (warp >= 4) {
+        // What is written below overlaps the query tile, P and the K/V slots: the query copy must have
+        // landed and every MMA of the CTA must be complete (each warpgroup has seen its last P V land).
+        mbar_wait_warp(smem_u32(&c.q_full), 0, abort_flag, a.status);
+        const bool any_valid = __any_sync(0xffffffffu, ri.valid);
+        if (kIsDual) {
             named_barrier(2, wg_threads);
             if (tid == kAuxThreads) SS_TR(5, 1);
-            const bool any_valid = __any_sync(0xffffffffu, vi >= 0);
-            constexpr uint32_t RB = RP * 4;
             const uint32_t srow = x_base + static_cast<uint32_t>(pidx * 64 + lrow) * RB;
             if (any_valid) {
                 #pragma unroll
@@ -1029,22 +950,21 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                     uint32_t orr[16];
                     if (has_acc) { tmem_ld16<0>(o_addr + c0, orr); tmem_wait_ld(); }
                     else { for (int i = 0; i < 16; ++i) orr[i] = 0u; }
-                    if (vi >= 0) {
+                    if (ri.valid) {
                         #pragma unroll
                         for (int i = 0; i < 16; i += 4) st_shared_v4(srow + (c0 + i) * 4u, orr[i], orr[i + 1], orr[i + 2], orr[i + 3]);
                     }
                 }
-                if (vi >= 0) st_shared_v4(srow + HD * 4u, __float_as_uint(m_run), __float_as_uint(l_run), 0u, 0u);
+                if (ri.valid) st_shared_v4(srow + HD * 4u, __float_as_uint(m_run), __float_as_uint(l_run), 0u, 0u);
             }
             if (tid == kAuxThreads) SS_TR(5, 2);
             named_barrier(1, wg_threads);
             // each of the row's four threads combines one quarter of the columns
-            if (vi >= 0) {
+            if (ri.valid) {
                 float m_out = -INFINITY, l_out = 0.f;
                 float4 acc[QW / 4];
-                combine_x(4, false, m_out, l_out, acc);
+                combine_x(m_out, l_out, acc);
                 if (C == 1) {
-                    // the pair was not split: this is the result
                     if (!skip) {
                         const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, ri);
                         const float inv = 1.f / l_out;
@@ -1068,72 +988,80 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 }
             }
             if (tid == kAuxThreads) SS_TR(5, 3);
-        }
-    } else if (C == 1) {
-        // the pair was not split: normalise and write this thread's row
-        if (warp >= 4 && __any_sync(0xffffffffu, ri.valid) && !skip) {
-            const float inv = 1.f / l_run;
+        } else {
+            // kPair: both accumulators of a row sit in the row's TMEM lane, so either thread of the row can
+            // read both.  The threads exchange (m, l) through shared memory; then warpgroup 0 finishes
+            // columns [0, kSplitCol) of the row and warpgroup 1 the rest.
+            const uint32_t ml_base = merge_base;                          // [warpgroup][128 rows] (m, l)
+            asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(ml_base + static_cast<uint32_t>(wg * kBlockRows + row_in_blk) * 8u),
+                         "f"(m_run), "f"(l_run) : "memory");
+            tc_fence_before();
+            named_barrier(2, wg_threads);
+            tc_fence_after();
+            if (tid == kAuxThreads) SS_TR(5, 1);
+            const float2 other = ld_shared_v2(ml_base + static_cast<uint32_t>((wg ^ 1) * kBlockRows + row_in_blk) * 8u);
+            const float m_out = fmaxf(m_run, other.x);
+            const float w_me = m_run != -INFINITY ? exp2f(m_run - m_out) : 0.f;      // 0: saw no visible key
+            const float w_ot = other.x != -INFINITY ? exp2f(other.x - m_out) : 0.f;
+            const float l_out = w_me * l_run + w_ot * other.y;
+            const uint32_t o_other = tmem + lane_base + (wg ^ 1) * G::kOCols;
+            constexpr int c_lo_1 = G::kSplitCol;
+            const int c_lo = wg == 0 ? 0 : c_lo_1, c_hi = wg == 0 ? c_lo_1 : HD;
+            const bool write_out = C == 1 && ri.valid && !skip;
             OutPtr dst;
             dst.o = nullptr; dst.lse = nullptr;
-            if (ri.valid) dst = out_ptr<HD>(a, b, h, spec_row0, ri);
-            if (dst.lse) *dst.lse = (m_run + log2f(l_run)) * 0.6931471805599453f;
-            #pragma unroll
-            for (int c0 = 0; c0 < HD; c0 += 16) {
-                uint32_t orr[16];
-                if (has_acc) { tmem_ld16<0>(o_addr + c0, orr); tmem_wait_ld(); }     // all 32 lanes of the warp
-                else { for (int i = 0; i < 16; ++i) orr[i] = 0u; }
-                if (dst.o == nullptr) continue;
-                uint4 lo, hi;
-                lo.x = pack_bf16(__uint_as_float(orr[0]) * inv, __uint_as_float(orr[1]) * inv);
-                lo.y = pack_bf16(__uint_as_float(orr[2]) * inv, __uint_as_float(orr[3]) * inv);
-                lo.z = pack_bf16(__uint_as_float(orr[4]) * inv, __uint_as_float(orr[5]) * inv);
-                lo.w = pack_bf16(__uint_as_float(orr[6]) * inv, __uint_as_float(orr[7]) * inv);
-                hi.x = pack_bf16(__uint_as_float(orr[8]) * inv, __uint_as_float(orr[9]) * inv);
-                hi.y = pack_bf16(__uint_as_float(orr[10]) * inv, __uint_as_float(orr[11]) * inv);
-                hi.z = pack_bf16(__uint_as_float(orr[12]) * inv, __uint_as_float(orr[13]) * inv);
-                hi.w = pack_bf16(__uint_as_float(orr[14]) * inv, __uint_as_float(orr[15]) * inv);
-                *reinterpret_cast<uint4*>(dst.o + c0) = lo;
-                *reinterpret_cast<uint4*>(dst.o + c0 + 8) = hi;
-            }
-        }
-    } else {
-        // kSingle / kMulti, split pair: every thread stores its row's partial straight from TMEM (a
-        // warpgroup that is done does not wait for the others; staging the rows in shared memory first
-        // would, and measured slower)
-        if (warp >= 4 && __any_sync(0xffffffffu, vi >= 0)) {
-            float* dst = part_mine + static_cast<size_t>(rblk * kBlockRows + (vi >= 0 ? vi : 0)) * RP;
-            #pragma unroll
-            for (int c0 = 0; c0 < HD; c0 += 16) {
-                uint32_t orr[16];
-                if (has_acc) { tmem_ld16<0>(o_addr + c0, orr); tmem_wait_ld(); }
-                else { for (int i = 0; i < 16; ++i) orr[i] = 0u; }
-                if (vi >= 0) {
+            if (write_out) dst = out_ptr<HD>(a, b, h, spec_row0, ri);
+            const float inv = C == 1 ? 1.f / l_out : 1.f;
+            const float f_me = w_me * inv, f_ot = w_ot * inv;
+            const uint32_t yrow = y_base + static_cast<uint32_t>(row_in_blk) * RB;
+            if (any_valid) {
+                #pragma unroll
+                for (int cc = 0; cc < G::kSplitCol; cc += 16) {
+                    const int c0 = c_lo + cc;
+                    if (c0 >= c_hi) break;                                // warp-uniform: wg is the same for the whole warp
+                    uint32_t mine[16], theirs[16];
+                    if (has_acc) {
+                        tmem_ld16<0>(o_addr + c0, mine);
+                        tmem_ld16<0>(o_other + c0, theirs);
+                        tmem_wait_ld();
+                    } else {
+                        for (int i = 0; i < 16; ++i) { mine[i] = 0u; theirs[i] = 0u; }
+                    }
+                    float v[16];
                     #pragma unroll
-                    for (int i = 0; i < 16; i += 4)
-                        __stcg(reinterpret_cast<float4*>(dst + c0 + i), make_float4(__uint_as_float(orr[i]), __uint_as_float(orr[i + 1]),
-                                                                                   __uint_as_float(orr[i + 2]), __uint_as_float(orr[i + 3])));
+                    for (int i = 0; i < 16; ++i) v[i] = f_me * __uint_as_float(mine[i]) + f_ot * __uint_as_float(theirs[i]);
+                    if (C == 1) {
+                        if (write_out) store_bf16x16(dst.o + c0, v);
+                    } else {
+                        #pragma unroll
+                        for (int i = 0; i < 16; i += 4)
+                            st_shared_v4(yrow + (c0 + i) * 4u, __float_as_uint(v[i]), __float_as_uint(v[i + 1]), __float_as_uint(v[i + 2]),
+                                         __float_as_uint(v[i + 3]));
+                    }
                 }
             }
-            if (vi >= 0) __stcg(reinterpret_cast<float2*>(dst + HD), make_float2(m_run, l_run));
+            if (C == 1) {
+                if (write_out && dst.lse && wg == 0) *dst.lse = (m_out + log2f(l_out)) * 0.6931471805599453f;
+            } else if (wg == 0) {
+                st_shared_v4(yrow + HD * 4u, __float_as_uint(m_out), __float_as_uint(l_out), 0u, 0u);
+            }
+            if (tid == kAuxThreads) SS_TR(5, 3);
         }
     }
 
     if (C > 1 && warp >= 4) {
-        // Arrive on the pair's counter, then wait (bounded) until the pair's other CTAs have arrived too:
-        // they were launched together and need nothing from this CTA, so the wait is short.  Each CTA then
-        // combines its own share of the rows, so the tail of the kernel is a C-th of a single merger's.
-        // The CTA barrier orders every thread's partial rows before the one thread whose device-scope fence
-        // and arrival publish them.  kDual: the rows wait in Y and that thread ships them to the workspace
-        // in whole lines with one bulk copy.
-        if (MODE == kDual) fence_async_smem();
+        // Ship the partial rows (one bulk copy of whole lines from Y), arrive on the block's counter, then
+        // wait (bounded) until the block's other CTAs have arrived too: they were launched together and
+        // need nothing from this CTA, so the wait is short.  Each CTA then combines its own share of the
+        // rows, so the tail of the kernel is a C-th of a single merger's.  The CTA barrier orders every
+        // thread's rows in Y before the one thread whose copy, device-scope fence and arrival publish them.
+        fence_async_smem();
         named_barrier(3, wg_threads);
         if (tid == kAuxThreads) {
-            unsigned int* cnt = reinterpret_cast<unsigned int*>(a.counters) + pair;
-            if (MODE == kDual) {
-                bulk_store(part_mine, y_base, 64u * RB);
-                bulk_store_wait_all();
-                asm volatile("fence.proxy.async;" ::: "memory");
-            }
+            unsigned int* cnt = reinterpret_cast<unsigned int*>(a.counters) + group;
+            bulk_store(part_mine, y_base, static_cast<uint32_t>(rows_cap) * RB);
+            bulk_store_wait_all();
+            asm volatile("fence.proxy.async;" ::: "memory");
             __threadfence();
             const unsigned int prev = atomicAdd(cnt, 1u);
             const unsigned int target = (prev | static_cast<unsigned int>(C - 1)) + 1u;   // this call's C arrivals end here
@@ -1152,32 +1080,22 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
         named_barrier(3, wg_threads);
         if (tid == kAuxThreads) SS_TR(5, 4);
         if (c.merge_ok && !skip) {
-            // This CTA's share: rows [first, first + share) of the pair's partial rows.  They stream through two
-            // shared-memory buffers, RR rows of every CTA of the pair per round (bulk copies from L2); the copy
+            // This CTA's share: rows [first, first + share) of the block's partial rows.  They stream through two
+            // shared-memory buffers, RR rows of every CTA of the block per round (bulk copies from L2); the copy
             // of round i + 1 runs while round i is combined.
-            constexpr uint32_t RB = RP * 4;
             const int share = rows_cap >> a.cluster_shift;
             const int first = static_cast<int>(rank) * share;
             const int RR = min(share, C == 8 ? 16 : 32);
             const int n_rounds = share / RR;
             const uint32_t buf_bytes = static_cast<uint32_t>(C * RR) * RB;
             const size_t cta_stride = static_cast<size_t>(rows_cap) * RP;
-            mbar_wait_warp(smem_u32(&c.q_full), 0, abort_flag, a.status);      // the query copy may alias the buffers
             auto issue_round = [&](int i) {
                 const uint32_t mbar = smem_u32(&c.merge_full[i & 1]);
                 asm volatile("fence.proxy.async;" ::: "memory");      // generic accesses to the buffer and to the partials come first
                 mbar_expect_tx(mbar, buf_bytes);
                 for (int sidx = 0; sidx < C; ++sidx)
                     bulk_load(merge_base + (i & 1) * buf_bytes + static_cast<uint32_t>(sidx * RR) * RB,
-                              part_pair + sidx * cta_stride + static_cast<size_t>(first + i * RR) * RP, static_cast<uint32_t>(RR) * RB, mbar);
-            };
-            // partial row number -> query row; false for a padding row
-            auto out_row = [&](int idx, RowInfo& r) -> bool {
-                if (MODE == kDual) { r = row_info(sp, idx); return r.valid; }
-                const int blk = idx / kBlockRows, v = idx - blk * kBlockRows;
-                if (v >= sp.n_valid(blk)) return false;
-                r = row_info(sp, sp.row_of(blk, v));
-                return true;
+                              part_group + sidx * cta_stride + static_cast<size_t>(first + i * RR) * RP, static_cast<uint32_t>(RR) * RB, mbar);
             };
             named_barrier(1, wg_threads);                             // every warpgroup is done with the staging area
             if (tid == kAuxThreads) issue_round(0);
@@ -1193,8 +1111,8 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 // work item: (row of the round, group of four columns)
                 for (int w = tid - kAuxThreads; w < RR * (HD / 4); w += wg_threads) {
                     const int rr = w / (HD / 4), g = w - rr * (HD / 4);
-                    RowInfo r;
-                    if (!out_row(first + i * RR + rr, r)) continue;
+                    const RowInfo r = row_info(sp, sp.row0 + first + i * RR + rr);
+                    if (!r.valid) continue;
                     float ms[8], ls[8];
                     float mx = -INFINITY;
                     #pragma unroll
@@ -1226,8 +1144,8 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 }
             }
         }
-        if (tid == kAuxThreads) SS_TR(5, 5);
     }
+    if (tid == kAuxThreads) SS_TR(5, 5);
 
 #ifdef SS_TRACE
     if (tid == 0) atomicMax(&g_wall[s_launch & 7][1], wall_ns());
@@ -1279,7 +1197,8 @@ static bool make_map(CUtensorMap* out, const void* basep, int d, long long n1, l
 }
 
 struct AttnPlan {
-    int tmax8, spec_rows, n_blocks, mode, tile_keys, n_kslots, n_vslots, cluster, threads;
+    int tmax8, spec_rows, s0rows, n_blocks, mode, n_kslots, n_vslots, cluster;
+    long long groups;                          // (sequence, head, row block) triples
     size_t smem;
     size_t counter_bytes, partial_bytes;       // workspace after its header
 };
@@ -1292,49 +1211,43 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     plan->tmax8 = (p.max_nodes + 7) / 8 * 8;
     plan->spec_rows = p.gamma > 0 ? (p.max_nodes * p.gamma + 7) / 8 * 8 : 0;
     const int q_rows = plan->tmax8 + plan->spec_rows;
-    plan->n_blocks = (q_rows + kBlockRows - 1) / kBlockRows;
-    plan->mode = plan->n_blocks > 1 ? kMulti : (q_rows <= 64 ? kDual : kSingle);
-    plan->tile_keys = plan->mode == kMulti ? 64 : 128;
-    plan->threads = kAuxThreads + (plan->mode == kMulti ? kMaxBlocks : (plan->mode == kDual ? 2 : 1)) * kBlockRows;
-    // CTAs per (sequence, head) pair: the largest power of two that still fits the grid on the SMs in one wave
-    const long long pairs = static_cast<long long>(p.batch) * p.n_heads;
+    plan->mode = q_rows <= 64 ? kDual : kPair;
+    plan->n_blocks = plan->mode == kDual ? 1 : (q_rows + kBlockRows - 1) / kBlockRows;
+    // stream rows that share block 0 with the main rows
+    plan->s0rows = plan->spec_rows < kBlockRows - plan->tmax8 ? plan->spec_rows : kBlockRows - plan->tmax8;
+    // CTAs per (sequence, head, row block): the largest power of two that still fits the grid on the SMs in one wave
+    plan->groups = static_cast<long long>(p.batch) * p.n_heads * plan->n_blocks;
     int c = 1;
-    while (c < 8 && pairs * (c * 2) <= sm_count()) c *= 2;
+    while (c < 8 && plan->groups * (c * 2) <= sm_count()) c *= 2;
     plan->cluster = c;
-    const int q_smem_rows = plan->mode == kDual ? kBlockRows : q_rows;
-    const size_t p_total = plan->mode == kDual ? static_cast<size_t>(2) * 3 * 64 * 128                 // two warpgroups
-                         : plan->mode == kSingle ? static_cast<size_t>(2) * q_rows * 128               // two key halves
-                                                 : static_cast<size_t>(plan->n_blocks) * kBlockRows * 128;
-    const size_t qp = static_cast<size_t>(halves) * q_smem_rows * 128 + p_total;
-    const size_t slot = static_cast<size_t>(halves) * plan->tile_keys * 128;
-    // the MMAs of the last block read up to 128 rows past the start of their block: keep that inside the allocation
-    const size_t overhang = static_cast<size_t>(kBlockRows) * 128;
+    const size_t p_total = plan->mode == kDual ? static_cast<size_t>(2) * 3 * 64 * 128 : static_cast<size_t>(2) * kBlockRows * 128;
+    const size_t qp = static_cast<size_t>(halves) * kBlockRows * 128 + p_total;
+    const size_t slot = static_cast<size_t>(halves) * kTileKeys * 128;
     int slots = static_cast<int>((kMaxDynSmem - 1024 - qp) / slot);
     if (slots > 2 * kMaxSlots) slots = 2 * kMaxSlots;
     if (slots < 4) return false;
-    // a K slot is held until every row block has its S queued, a V slot until the last P V: split evenly
-    plan->n_kslots = slots / 2 > kMaxSlots ? kMaxSlots : slots / 2;
+    // a K slot is held until S is queued, a V slot until P V has completed: the odd slot goes to V
+    plan->n_kslots = slots / 2;
     plan->n_vslots = slots - plan->n_kslots > kMaxSlots ? kMaxSlots : slots - plan->n_kslots;
     size_t bytes = qp + static_cast<size_t>(plan->n_kslots + plan->n_vslots) * slot;
-    if (bytes < qp + overhang) bytes = qp + overhang;
-    // kDual stages its four CTA-local partials of every row ((head_dim + 4) floats) once the pipeline is done
-    // after the pipeline kDual stages its four CTA-local partials of every row and the outgoing row (5 x 64 rows)
+    // after the pipeline the same memory stages partial rows ((head_dim + 4) floats each): kDual its four
+    // CTA-local partials of every row and the outgoing rows (5 x 64 rows), kPair 2 KB and 128 outgoing rows
     const size_t row_bytes = static_cast<size_t>(p.head_dim + 4) * 4;
-    const size_t stage = plan->mode == kDual ? 5 * 64 * row_bytes : 0;
+    const size_t stage = plan->mode == kDual ? 5 * 64 * row_bytes : 2048 + kBlockRows * row_bytes;
     if (stage > bytes) bytes = stage;
-    // every CTA of a split pair streams its share of the pair's partial rows through two buffers
-    const size_t merge_bufs = static_cast<size_t>(2) * c * (c == 8 ? 16 : 32) * (p.head_dim + 4) * 4;
+    // every CTA of a split block streams its share of the block's partial rows through two buffers
+    const size_t merge_bufs = static_cast<size_t>(2) * c * (c == 8 ? 16 : 32) * row_bytes;
     if (c > 1 && merge_bufs > bytes) bytes = merge_bufs;
     plan->smem = bytes + 1024;
-    // workspace: one arrival counter per pair; one partial row per (pair, CTA of the pair, query row)
-    const size_t rows_cap = plan->mode == kDual ? 64 : static_cast<size_t>(plan->n_blocks) * kBlockRows;
-    plan->counter_bytes = (static_cast<size_t>(pairs) * sizeof(int32_t) + 255) / 256 * 256;
-    plan->partial_bytes = c > 1 ? static_cast<size_t>(pairs) * c * rows_cap * (p.head_dim + 4) * 4 : 0;
+    // workspace: one arrival counter per group; one partial row per (group, CTA of the group, row)
+    const size_t rows_cap = plan->mode == kDual ? 64 : kBlockRows;
+    plan->counter_bytes = (static_cast<size_t>(plan->groups) * sizeof(int32_t) + 255) / 256 * 256;
+    plan->partial_bytes = c > 1 ? static_cast<size_t>(plan->groups) * c * rows_cap * row_bytes : 0;
     return plan->smem <= static_cast<size_t>(kMaxDynSmem);
 }
 
 template <int HD, int MODE>
-static int32_t launch(const AttnArgs& args, const AttnPlan& plan, long long pairs, cudaStream_t stream) {
+static int32_t launch(const AttnArgs& args, const AttnPlan& plan, cudaStream_t stream) {
     static bool configured[64] = {false};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return SS_ERR_CUDA;
@@ -1345,8 +1258,8 @@ static int32_t launch(const AttnArgs& args, const AttnPlan& plan, long long pair
         configured[dev] = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(pairs * plan.cluster), 1, 1);
-    cfg.blockDim = dim3(static_cast<unsigned>(plan.threads), 1, 1);
+    cfg.gridDim = dim3(static_cast<unsigned>(plan.groups * plan.cluster), 1, 1);
+    cfg.blockDim = dim3(static_cast<unsigned>(Geo<HD, MODE>::kThreads), 1, 1);
     // always more than half of an SM's shared memory: one CTA per SM, so a CTA never queues for TMEM
     cfg.dynamicSmemBytes = plan.smem < 120 * 1024 ? 120 * 1024 : plan.smem;
     cfg.stream = stream;
@@ -1384,6 +1297,7 @@ extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
     if (p->kv_total_slots > 0x7fffffffll) return SS_ERR_UNSUPPORTED;
     const long long rows_main = static_cast<long long>(p->batch) * p->max_nodes;
     if (rows_main * (p->gamma > 0 ? p->gamma : 1) > 0x7fffffffll) return SS_ERR_UNSUPPORTED;
+    if (plan.groups * plan.cluster > 0x7fffffffll) return SS_ERR_UNSUPPORTED;
     const void* ptrs[] = {p->q_main, p->o_main, p->k_cache, p->v_cache, p->workspace,
                           p->gamma ? p->q_spec : nullptr, p->gamma ? p->k_spec : nullptr,
                           p->gamma ? p->v_spec : nullptr, p->gamma ? p->o_spec : nullptr};
@@ -1393,7 +1307,7 @@ extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
     if (p->workspace_bytes < ss_msa_attention_workspace_bytes(p)) return SS_ERR_WORKSPACE;
 
     ss::AttnArgs a;
-    const int d = p->head_dim, H = p->n_heads, tk = plan.tile_keys;
+    const int d = p->head_dim, H = p->n_heads, tk = ss::kTileKeys;
     const bool shared_heads = (p->kv_head_stride == 0);
     const long long kv_heads = shared_heads ? 1 : H;
     const long long kv_hstride = shared_heads ? d : p->kv_head_stride;
@@ -1402,15 +1316,17 @@ extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
               ss::make_map(&a.tm_qm, p->q_main, d, H, d, rows_main, static_cast<long long>(H) * d, plan.tmax8);
     if (ok && p->gamma > 0) {
         const long long rows_spec = rows_main * p->gamma;
-        ok = ss::make_map(&a.tm_qs, p->q_spec, d, H, d, rows_spec, static_cast<long long>(H) * d, plan.spec_rows) &&
-             ss::make_map(&a.tm_ks, p->k_spec, d, H, d, rows_spec, static_cast<long long>(H) * d, tk) &&
-             ss::make_map(&a.tm_vs, p->v_spec, d, H, d, rows_spec, static_cast<long long>(H) * d, tk);
+        const long long hd = static_cast<long long>(H) * d;
+        ok = ss::make_map(&a.tm_qs, p->q_spec, d, H, d, rows_spec, hd, plan.s0rows > 0 ? plan.s0rows : 8) &&
+             ss::make_map(&a.tm_qs1, p->q_spec, d, H, d, rows_spec, hd, ss::kBlockRows) &&
+             ss::make_map(&a.tm_ks, p->k_spec, d, H, d, rows_spec, hd, tk) &&
+             ss::make_map(&a.tm_vs, p->v_spec, d, H, d, rows_spec, hd, tk);
     } else if (ok) {
-        a.tm_qs = a.tm_qm; a.tm_ks = a.tm_k; a.tm_vs = a.tm_v;     // never used when gamma == 0
+        a.tm_qs = a.tm_qm; a.tm_qs1 = a.tm_qm; a.tm_ks = a.tm_k; a.tm_vs = a.tm_v;     // never used when gamma == 0
     }
     if (!ok) return SS_ERR_CUDA;
     a.batch = p->batch; a.n_heads = H; a.gamma = p->gamma; a.max_nodes = p->max_nodes;
-    a.tmax8 = plan.tmax8; a.spec_rows = plan.spec_rows; a.n_blocks = plan.n_blocks;
+    a.tmax8 = plan.tmax8; a.s0rows = plan.s0rows; a.n_blocks = plan.n_blocks;
     a.n_kslots = plan.n_kslots; a.n_vslots = plan.n_vslots;
     a.cluster = plan.cluster;
     a.cluster_shift = 0;
@@ -1426,26 +1342,18 @@ extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
     a.status = reinterpret_cast<int*>(p->workspace);
     a.counters = reinterpret_cast<int*>(static_cast<char*>(p->workspace) + ss::kWsHeaderBytes);
     a.partials = reinterpret_cast<float*>(static_cast<char*>(p->workspace) + ss::kWsHeaderBytes + plan.counter_bytes);
-    const long long pairs = static_cast<long long>(p->batch) * H;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (plan.mode == ss::kDual) {
         switch (d) {
-            case 64: return ss::launch<64, ss::kDual>(a, plan, pairs, s);
-            case 80: return ss::launch<80, ss::kDual>(a, plan, pairs, s);
-            default: return ss::launch<128, ss::kDual>(a, plan, pairs, s);
-        }
-    }
-    if (plan.mode == ss::kSingle) {
-        switch (d) {
-            case 64: return ss::launch<64, ss::kSingle>(a, plan, pairs, s);
-            case 80: return ss::launch<80, ss::kSingle>(a, plan, pairs, s);
-            default: return ss::launch<128, ss::kSingle>(a, plan, pairs, s);
+            case 64: return ss::launch<64, ss::kDual>(a, plan, s);
+            case 80: return ss::launch<80, ss::kDual>(a, plan, s);
+            default: return ss::launch<128, ss::kDual>(a, plan, s);
         }
     }
     switch (d) {
-        case 64: return ss::launch<64, ss::kMulti>(a, plan, pairs, s);
-        case 80: return ss::launch<80, ss::kMulti>(a, plan, pairs, s);
-        default: return ss::launch<128, ss::kMulti>(a, plan, pairs, s);
+        case 64: return ss::launch<64, ss::kPair>(a, plan, s);
+        case 80: return ss::launch<80, ss::kPair>(a, plan, s);
+        default: return ss::launch<128, ss::kPair>(a, plan, s);
     }
 }
 
