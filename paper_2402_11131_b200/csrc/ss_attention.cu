@@ -1063,8 +1063,11 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             bulk_store_wait_all();
             asm volatile("fence.proxy.async;" ::: "memory");
             __threadfence();
-            const unsigned int prev = atomicAdd(cnt, 1u);
-            const unsigned int target = (prev | static_cast<unsigned int>(C - 1)) + 1u;   // this call's C arrivals end here
+            // Every call adds 8 to the counter in total (each CTA 8 / C), so between calls it is a multiple of
+            // 8 whatever split factor earlier calls on this workspace had, and this call's arrivals end at the
+            // next multiple of 8 above the value this CTA found.
+            const unsigned int prev = atomicAdd(cnt, 8u >> a.cluster_shift);
+            const unsigned int target = (prev | 7u) + 1u;
             bool ok = true;
             const long long t0 = clock64();
             for (;;) {

@@ -228,14 +228,17 @@ def test_attention_without_the_prefix_promise_gives_the_same_bits(cuda, oracle):
 
 @pytest.mark.parametrize("n_heads,expect_split", [(1, 8), (3, 8), (20, 4), (40, 2), (100, 1)])
 def test_attention_every_split_factor(cuda, oracle, n_heads, expect_split):
-    """The number of CTAs per (sequence, head) pair follows the head count (8, 4, 2, 1): every merge
-    path, including pairs whose CTAs get no keys at all (8 CTAs, 5 key units)."""
+    """The number of CTAs that share a row block's keys follows the head count (8, 4, 2, 1): every merge
+    path, including CTAs that get no keys at all (8 CTAs, 5 key units).  The layers of a step share one
+    workspace and may have different split factors; the second pass finds the arrival counters as the
+    first one left them."""
     api, DeviceStep = cuda
     for k, (L, T, g) in enumerate([(70, 6, 1), (900, 40, 4)]):
         cfg = W.custom_config("split%d_%d" % (n_heads, k), n_layers=2, n_msa_layers=1, prefix_len=L, n_nodes=T,
                               gamma=g, max_depth=3, n_heads=n_heads, head_dim=64, config_id=660 + k)
         st = W.make_step(cfg)
         dev = DeviceStep(st, with_lse=True)
+        dev.run_attention()
         dev.run_attention()
         assert api.ss_status(dev.attn_ws) == 0
         for i in range(2):
