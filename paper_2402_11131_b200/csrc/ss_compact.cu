@@ -20,6 +20,7 @@ kv_compact_kernel(uint4* __restrict__ k_all, uint4* __restrict__ v_all, int n_he
     const int layer = blockIdx.y, b = blockIdx.z;
     const int cols = n_heads * chunks_per_head;          // 16-byte columns per K (or V) slot
     const int col2 = blockIdx.x * kCompactThreads + threadIdx.x;
+    wait_for_previous_kernel();
     const int L = kv_len_in[b];
     int len = accept_len[b];
     len = max(0, min(len, SS_PATH_STRIDE));
@@ -53,6 +54,7 @@ kv_compact_kernel(uint4* __restrict__ k_all, uint4* __restrict__ v_all, int n_he
 __global__ void kv_len_update_kernel(const int32_t* __restrict__ kv_len_in, const int32_t* __restrict__ accept_len,
                                      int32_t* __restrict__ kv_len_out, int batch) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    wait_for_previous_kernel();      // the gather has read the old lengths
     if (b < batch) kv_len_out[b] = kv_len_in[b] + max(0, min(accept_len[b], SS_PATH_STRIDE));
 }
 
@@ -76,10 +78,12 @@ extern "C" int32_t ss_kv_compact(void* k_cache_all, void* v_cache_all, const ss_
     const int cols2 = 2 * lo.n_heads * chunks_per_head;
     dim3 grid((cols2 + ss::kCompactThreads - 1) / ss::kCompactThreads, lo.n_layers, batch);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    ss::kv_compact_kernel<<<grid, ss::kCompactThreads, 0, s>>>(
-        static_cast<uint4*>(k_cache_all), static_cast<uint4*>(v_cache_all), lo.n_heads, chunks_per_head,
-        lo.layer_stride / 8, lo.slot_stride / 8, lo.head_stride / 8, kv_start, kv_len_in, accept_len, accept_path);
-    if (cudaGetLastError() != cudaSuccess) return SS_ERR_CUDA;
-    ss::kv_len_update_kernel<<<(batch + 127) / 128, 128, 0, s>>>(kv_len_in, accept_len, kv_len_out, batch);
-    return cudaGetLastError() == cudaSuccess ? SS_OK : SS_ERR_CUDA;
+    // both launches may be scheduled while their predecessor drains; each waits for it before touching memory
+    if (ss::launch_after_previous(ss::kv_compact_kernel, grid, dim3(ss::kCompactThreads), s, static_cast<uint4*>(k_cache_all),
+                                  static_cast<uint4*>(v_cache_all), lo.n_heads, chunks_per_head, lo.layer_stride / 8,
+                                  lo.slot_stride / 8, lo.head_stride / 8, kv_start, kv_len_in, accept_len,
+                                  accept_path) != cudaSuccess)
+        return SS_ERR_CUDA;
+    return ss::launch_after_previous(ss::kv_len_update_kernel, dim3((batch + 127) / 128), dim3(128), s, kv_len_in, accept_len,
+                                     kv_len_out, batch) == cudaSuccess ? SS_OK : SS_ERR_CUDA;
 }

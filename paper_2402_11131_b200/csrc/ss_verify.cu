@@ -29,6 +29,7 @@ tree_verify_kernel(const float* __restrict__ logits, const int32_t* __restrict__
                    int32_t* __restrict__ node_argmax, int32_t* __restrict__ counters,
                    Cand* __restrict__ partials) {
     const int chunk = blockIdx.x, t = blockIdx.y, b = blockIdx.z;
+    wait_for_previous_kernel();
     const int T = trees[b].n_nodes;
     __shared__ Cand s_red[kVerifyThreads / 32];
     __shared__ int32_t s_am[SS_MAX_NODES];
@@ -83,6 +84,9 @@ tree_verify_kernel(const float* __restrict__ logits, const int32_t* __restrict__
     if (!s_last) return;
     __threadfence();
 
+    // the tree walk below is one thread's serial loop: its inputs go to shared memory first, loaded by
+    // T threads at once, so that no step of the loop waits for global memory
+    __shared__ int32_t s_parent[SS_MAX_NODES], s_depth[SS_MAX_NODES], s_tok[SS_MAX_NODES];
     if (threadIdx.x < T) {
         const Cand* p = partials + (static_cast<size_t>(b) * max_nodes + threadIdx.x) * n_chunks;
         float bv = -INFINITY;
@@ -97,33 +101,36 @@ tree_verify_kernel(const float* __restrict__ logits, const int32_t* __restrict__
         if (bi == 0x7fffffff) bi = 0;
         s_am[threadIdx.x] = bi;
         if (node_argmax) node_argmax[static_cast<size_t>(b) * max_nodes + threadIdx.x] = bi;
+        s_parent[threadIdx.x] = trees[b].parent[threadIdx.x];
+        s_depth[threadIdx.x] = trees[b].depth[threadIdx.x];
+        s_tok[threadIdx.x] = tokens[static_cast<size_t>(b) * max_nodes + threadIdx.x];
     }
     __syncthreads();
-    {
+    int32_t* const path = accept_path + static_cast<size_t>(b) * SS_PATH_STRIDE;
+    if (threadIdx.x < 32) {
         // validity needs the parent's validity, so sweep in index order (parent[i] < i) with one
         // thread; T <= 64 keeps this trivial
+        int best = 0, len = 1;
         if (threadIdx.x == 0) {
-            const ss_tree_desc& tr = trees[b];
-            const int32_t* tok = tokens + static_cast<size_t>(b) * max_nodes;
             uint64_t valid = 1ull;
-            int best = 0, best_depth = 0;
+            int best_depth = 0;
             for (int c = 1; c < T; ++c) {
-                const int p = tr.parent[c];
-                if (((valid >> p) & 1ull) && tok[c] == s_am[p]) {
+                const int p = s_parent[c];
+                if (p >= 0 && ((valid >> p) & 1ull) && s_tok[c] == s_am[p]) {
                     valid |= 1ull << c;
-                    const int dep = tr.depth[c];
+                    const int dep = s_depth[c];
                     if (dep > best_depth) { best = c; best_depth = dep; }
                 }
             }
-            const int len = best_depth + 1;
-            int32_t* path = accept_path + static_cast<size_t>(b) * SS_PATH_STRIDE;
-            for (int i = len; i < SS_PATH_STRIDE; ++i) path[i] = -1;
-            for (int a = best, i = len - 1; a >= 0 && i >= 0; a = tr.parent[a], --i) path[i] = a;
+            len = best_depth + 1;
+            for (int a = best, i = len - 1; a >= 0 && i >= 0; a = s_parent[a], --i) path[i] = a;
             accept_len[b] = len;
             last_node[b] = best;
             bonus_token[b] = s_am[best];
             counters[b] = 0;   // leave the workspace ready for the next call
         }
+        len = __shfl_sync(0xffffffffu, len, 0);
+        for (int i = len + static_cast<int>(threadIdx.x); i < SS_PATH_STRIDE; i += 32) path[i] = -1;
     }
 }
 
@@ -153,10 +160,11 @@ extern "C" int32_t ss_tree_verify(const float* logits, const int32_t* draft_toke
     const size_t counter_bytes = (static_cast<size_t>(batch) * sizeof(int32_t) + 255) / 256 * 256;
     ss::Cand* partials = reinterpret_cast<ss::Cand*>(ws + ss::kWsHeaderBytes + counter_bytes);
     dim3 grid(n_chunks, max_nodes, batch);
-    ss::tree_verify_kernel<<<grid, ss::kVerifyThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-        logits, draft_tokens, trees, max_nodes, vocab, n_chunks, accept_len, accept_path, last_node,
-        bonus_token, node_argmax, counters, partials);
-    return cudaGetLastError() == cudaSuccess ? SS_OK : SS_ERR_CUDA;
+    const cudaError_t err = ss::launch_after_previous(ss::tree_verify_kernel, grid, dim3(ss::kVerifyThreads),
+                                                      static_cast<cudaStream_t>(stream), logits, draft_tokens, trees, max_nodes,
+                                                      vocab, n_chunks, accept_len, accept_path, last_node, bonus_token,
+                                                      node_argmax, counters, partials);
+    return err == cudaSuccess ? SS_OK : SS_ERR_CUDA;
 }
 
 // ---------------------------------------------------------------------------------------------
