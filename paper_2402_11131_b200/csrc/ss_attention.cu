@@ -106,7 +106,12 @@ struct Ctrl {
     unsigned long long k_full[kMaxSlots], k_empty[kMaxSlots], v_full[kMaxSlots], v_empty[kMaxSlots];
     unsigned long long s_full[2][2];            // per (warpgroup, S buffer): a warpgroup sees every phase of its own
     unsigned long long s_free[2];
-    unsigned long long p_full[2], o_done[2];    // per warpgroup
+    // P of a warpgroup written.  kDual: [w][0], one arrival per thread.  kPair: [w][tile & 1], one arrival per warp: a
+    // warp can only be two tiles ahead of another once the P V between them is complete, so it never arrives twice in a phase
+    unsigned long long p_full[2][2];
+    // P V of a warpgroup complete.  kDual: [w][0].  kPair: [w][tile & 1]: a warpgroup that does not look at every
+    // phase is then never more than one phase behind, which a parity wait needs
+    unsigned long long o_done[2][2];
     unsigned long long anc[SS_MAX_NODES];
     uint32_t tmem_base;
     int abort;
@@ -215,6 +220,12 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_
         "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// D[tmem] (+)= A[tmem] * B[smem]: A is 128 lanes x 16 bf16, two to a 32-bit column (8 columns per step)
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -243,6 +254,12 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[N]
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
         ::SS_W16(r, O), "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31};"
+        ::SS_W16(r, 0), SS_W16(r, 16), "r"(taddr) : "memory");
 }
 // 64 columns starting at taddr
 __device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t (&r)[64]) {
@@ -413,6 +430,27 @@ __device__ __forceinline__ float chunk_exp_store(const uint32_t (&v)[64], float 
     return (sum[0] + sum[1]) + (sum[2] + sum[3]);
 }
 
+// the same exponentials, packed two bf16 to a word (key 2c in the low half of word c); returns the sum
+template <bool MASKED>
+__device__ __forceinline__ float chunk_exp_pack(const uint32_t (&v)[64], float scale, float m_use, unsigned long long vis,
+                                                uint32_t (&pk)[32]) {
+    float sum[4] = {0.f, 0.f, 0.f, 0.f};
+    const uint32_t vlo = static_cast<uint32_t>(vis), vhi = static_cast<uint32_t>(vis >> 32);
+    const float neg_m = -m_use;
+    #pragma unroll
+    for (int k = 0; k < 64; k += 2) {
+        float e0 = exp2f(fmaf(__uint_as_float(v[k]), scale, neg_m));
+        float e1 = exp2f(fmaf(__uint_as_float(v[k + 1]), scale, neg_m));
+        if (MASKED) {
+            e0 = (((k < 32 ? vlo : vhi) >> (k & 31)) & 1u) ? e0 : 0.f;
+            e1 = (((k < 32 ? vlo : vhi) >> ((k + 1) & 31)) & 1u) ? e1 : 0.f;
+        }
+        sum[(k >> 1) & 3] += e0 + e1;
+        pk[k >> 1] = pack_bf16(e0, e1);
+    }
+    return (sum[0] + sum[1]) + (sum[2] + sum[3]);
+}
+
 // Kernel variants.  kPair: a block of up to 128 rows; warpgroup w takes keys 64w .. 64w+63 of every
 // tile, with its own P tile (64 keys wide), running maximum and accumulator.  kDual: at most 64 rows:
 // the block holds the rows twice, copy 0 takes keys 0..63 of a tile and copy 1 keys 64..127 (P is zero
@@ -436,7 +474,7 @@ struct Geo {
     // P of one warpgroup, 128 B rows of 64 keys (swizzled).  kPair: 128 rows.  kDual: [copy-0 rows 0..63 |
     // 64 zero rows | copy-1 rows 0..63]; the MMA reads keys 0..63 from the first 128 rows and keys 64..127
     // from the last 128 rows, so each copy's other half is zero.
-    static constexpr uint32_t kPBytes = MODE == kDual ? 3u * 64u * 128u : 128u * 128u;
+    static constexpr uint32_t kPBytes = MODE == kDual ? 3u * 64u * 128u : 0u;
     static constexpr int kRowsCap = MODE == kDual ? 64 : kBlockRows;   // partial rows a CTA ships
     static constexpr int kSplitCol = ((HD / 16 + 1) / 2) * 16;    // kPair: warpgroup 0 finishes columns [0, kSplitCol)
 };
@@ -534,11 +572,13 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     } else if (tid == 64) {                               // every other barrier (first used after the CTA-wide sync)
         for (int s = 0; s < kMaxSlots; ++s) { mbar_init(smem_u32(&c.k_empty[s]), 1); mbar_init(smem_u32(&c.v_empty[s]), 1); }
         for (int s = 0; s < 2; ++s) {
-            mbar_init(smem_u32(&c.s_free[s]), kIsDual ? 4 : 8);          // warps that read an S buffer
+            mbar_init(smem_u32(&c.s_free[s]), kIsDual ? 4 : 1);          // kDual: warps that read an S buffer; kPair: the P V commit
             mbar_init(smem_u32(&c.s_full[0][s]), 1);
             mbar_init(smem_u32(&c.s_full[1][s]), 1);
-            mbar_init(smem_u32(&c.p_full[s]), kBlockRows);
-            mbar_init(smem_u32(&c.o_done[s]), 1);
+            mbar_init(smem_u32(&c.p_full[s][0]), kIsDual ? kBlockRows : 4);   // kDual: threads; kPair: warps
+            mbar_init(smem_u32(&c.p_full[s][1]), 4);
+            mbar_init(smem_u32(&c.o_done[s][0]), 1);
+            mbar_init(smem_u32(&c.o_done[s][1]), 1);
             mbar_init(smem_u32(&c.merge_full[s]), 1);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -748,7 +788,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 if (kIsDual) {
                     // the whole tile for warpgroup j & 1: keys 0..63 from copy 0's rows, 64..127 from copy 1's
                     const int w = j & 1;
-                    if (!mbar_wait(smem_u32(&c.p_full[w]), (j >> 1) & 1, abort_flag, a.status)) break;
+                    if (!mbar_wait(smem_u32(&c.p_full[w][0]), (j >> 1) & 1, abort_flag, a.status)) break;
                     SS_TR(2, 9 + 4 * j);
                     tc_fence_after();
                     const uint32_t pa = p_base + w * G::kPBytes;
@@ -756,22 +796,25 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                     for (int ks = 0; ks < TK / 16; ++ks)
                         tc_mma(tmem + w * G::kOCols, desc_k_major(pa + (ks >> 2) * (64u * 128u) + (ks & 3) * 32u),
                                desc_mn_major(va + ks * 2048u, G::kBoxBytes), G::kIdescPV, (j >= 2 || ks > 0) ? 1u : 0u);
-                    tc_commit(smem_u32(&c.o_done[w]));
+                    tc_commit(smem_u32(&c.o_done[w][0]));
                 } else {
-                    // keys 64w .. 64w+63 into the accumulator of warpgroup w
+                    // keys 64w .. 64w+63 into the accumulator of warpgroup w; P is read from TMEM, where the
+                    // warpgroup left it over the first 32 columns of its half of the S buffer
+                    const int buf = j & 1;
                     #pragma unroll
                     for (int w = 0; w < 2; ++w) {
-                        if (!mbar_wait(smem_u32(&c.p_full[w]), j & 1, abort_flag, a.status)) { ok = false; break; }
+                        if (!mbar_wait(smem_u32(&c.p_full[w][buf]), (j >> 1) & 1, abort_flag, a.status)) { ok = false; break; }
                         if (w == 0) SS_TR(2, 9 + 4 * j);
                         tc_fence_after();
-                        const uint32_t pa = p_base + w * G::kPBytes;
+                        const uint32_t pa = tmem_s + buf * TK + w * 64;
                         #pragma unroll
                         for (int ks = 0; ks < 4; ++ks)
-                            tc_mma(tmem + w * G::kOCols, desc_k_major(pa + ks * 32u),
-                                   desc_mn_major(va + (w * 4 + ks) * 2048u, G::kBoxBytes), G::kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
-                        tc_commit(smem_u32(&c.o_done[w]));
+                            tc_mma_ts(tmem + w * G::kOCols, pa + ks * 8u, desc_mn_major(va + (w * 4 + ks) * 2048u, G::kBoxBytes),
+                                      G::kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
+                        tc_commit(smem_u32(&c.o_done[w][buf]));
                     }
                     if (!ok) break;
+                    tc_commit(smem_u32(&c.s_free[buf]));                 // both halves of P have been read: S may be overwritten
                 }
                 SS_TR(2, 10 + 4 * j);
                 tc_commit(smem_u32(&c.v_empty[rv.slot]));                // P V of tile j is queued: V may go when it completes
@@ -822,19 +865,28 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 }
             }
             if (tr_on) SS_TR(trole, 9 + 6 * n_own);
-            // the scores stay in registers: S can be overwritten
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&c.s_free[buf]));
-            // the previous PV of this warpgroup must be complete: it read the P tile that is about to
-            // be overwritten, and it wrote the accumulator that a raised maximum rescales
-            if (n_own > 0) {
-                if (!mbar_wait_warp(smem_u32(&c.o_done[wg]), (n_own - 1) & 1, abort_flag, a.status)) break;
+            const bool rescale = n_own > 0 && __any_sync(0xffffffffu, need);
+            if (kIsDual) {
+                // the scores stay in registers: S can be overwritten
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&c.s_free[buf]));
+                // the previous PV of this warpgroup must be complete: it read the P tile that is about to
+                // be overwritten, and it wrote the accumulator that a raised maximum rescales
+                if (n_own > 0) {
+                    if (!mbar_wait_warp(smem_u32(&c.o_done[wg][0]), (n_own - 1) & 1, abort_flag, a.status)) break;
+                    tc_fence_after();
+                }
+            } else if (rescale) {
+                // kPair: P goes to the S buffer itself (handed back by the P V that reads it), so only a raised
+                // maximum waits for the previous P V: it rescales the accumulator that P V wrote
+                // (S of this tile exists, so the P V two tiles back is complete: the barrier is at most one phase behind)
+                if (!mbar_wait_warp(smem_u32(&c.o_done[wg][(j - 1) & 1]), ((j - 1) >> 1) & 1, abort_flag, a.status)) break;
                 tc_fence_after();
             }
             if (tr_on) SS_TR(trole, 10 + 6 * n_own);
             if (warp_active) {
-                if (n_own > 0 && __any_sync(0xffffffffu, need)) {
+                if (rescale) {
                     #pragma unroll
                     for (int c0 = 0; c0 < HD; c0 += 16) {
                         uint32_t orr[16];
@@ -848,8 +900,16 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 }
                 // ---- pass 2: P = exp2(S - m) as bf16, row sum -------------------------------------------
                 const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
-                l_run += masked ? chunk_exp_store<true>(sr, a.scale_log2, m_use, vis, p_row, row_in_blk)
-                                : chunk_exp_store<false>(sr, a.scale_log2, m_use, 0ull, p_row, row_in_blk);
+                if (kIsDual) {
+                    l_run += masked ? chunk_exp_store<true>(sr, a.scale_log2, m_use, vis, p_row, row_in_blk)
+                                    : chunk_exp_store<false>(sr, a.scale_log2, m_use, 0ull, p_row, row_in_blk);
+                } else {
+                    // two bf16 to a column, over the first 32 of the 64 score columns this thread has read
+                    uint32_t pk[32];
+                    l_run += masked ? chunk_exp_pack<true>(sr, a.scale_log2, m_use, vis, pk) : chunk_exp_pack<false>(sr, a.scale_log2, m_use, 0ull, pk);
+                    tmem_st32(s_addr, pk);
+                    tmem_wait_st();
+                }
             }
             if (tr_on) SS_TR(trole, 11 + 6 * n_own);
             // V rows past the end of the sequence's keys may hold anything (even NaN patterns): P is 0
@@ -871,13 +931,24 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             if (tr_on) SS_TR(trole, 12 + 6 * n_own);
             fence_async_smem();
             tc_fence_before();
-            mbar_arrive(smem_u32(&c.p_full[wg]));
+            if (kIsDual) {
+                mbar_arrive(smem_u32(&c.p_full[wg][0]));
+            } else {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&c.p_full[wg][buf]));
+            }
             if (tr_on) SS_TR(trole, 13 + 6 * n_own);
             ++n_own;
         }
         // the warpgroup's last PV must have landed in TMEM before the accumulator is read
         if (n_own > 0) {
-            mbar_wait_warp(smem_u32(&c.o_done[wg]), (n_own - 1) & 1, abort_flag, a.status);
+            if (kIsDual) {
+                mbar_wait_warp(smem_u32(&c.o_done[wg][0]), (n_own - 1) & 1, abort_flag, a.status);
+            } else {
+                // the last two P V may both be outstanding: one barrier each
+                if (n_own > 1) mbar_wait_warp(smem_u32(&c.o_done[wg][(n_own - 2) & 1]), ((n_own - 2) >> 1) & 1, abort_flag, a.status);
+                mbar_wait_warp(smem_u32(&c.o_done[wg][(n_own - 1) & 1]), ((n_own - 1) >> 1) & 1, abort_flag, a.status);
+            }
             tc_fence_after();
         }
     }
@@ -1223,7 +1294,7 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     int c = 1;
     while (c < 8 && plan->groups * (c * 2) <= sm_count()) c *= 2;
     plan->cluster = c;
-    const size_t p_total = plan->mode == kDual ? static_cast<size_t>(2) * 3 * 64 * 128 : static_cast<size_t>(2) * kBlockRows * 128;
+    const size_t p_total = plan->mode == kDual ? static_cast<size_t>(2) * 3 * 64 * 128 : 0;      // kPair keeps P in TMEM
     const size_t qp = static_cast<size_t>(halves) * kBlockRows * 128 + p_total;
     const size_t slot = static_cast<size_t>(halves) * kTileKeys * 128;
     int slots = static_cast<int>((kMaxDynSmem - 1024 - qp) / slot);
