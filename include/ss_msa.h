@@ -98,8 +98,11 @@ int32_t ss_tree_build(const int32_t* parent, int32_t n_nodes, int32_t gamma, ss_
  *   lse_main float[batch][max_nodes][n_heads], lse_spec float[batch][max_nodes][gamma][n_heads]:
  *                                  optional natural-log sum-exp of the scaled scores (NULL to skip).
  * Scores are sm_scale * <q, k>; softmax statistics and both products accumulate in fp32.
- * The workspace holds, besides the status word, one arrival counter per (sequence, head) pair and the
- * partial rows of pairs whose keys are split over several CTAs (ss_msa_attention_workspace_bytes).
+ * The workspace holds, besides the status word, one arrival counter per (sequence, head, block of 128
+ * query rows) and the partial rows of blocks whose keys are split over several CTAs
+ * (ss_msa_attention_workspace_bytes).  Calls of different shapes may share one workspace as long as they
+ * are ordered on one stream and it is large enough for each: a call leaves every counter at a multiple
+ * of 8.
  * Reads no K/V row past slot kv_start[b]+L_b+T_b-1 whose value can reach an output (a tile may touch
  * later slots of the slab; what it finds there is masked or cleared); writes only o_*, lse_* and the
  * workspace.
