@@ -749,6 +749,10 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             SS_TR(1, 0);
             Ring rk;
             rk.start();
+            // A descriptor's low word is (address >> 4): a step inside the tile is an addition to the descriptor
+            // (shared memory ends below 2^18, so nothing carries out of the field), and the issuing thread
+            // spends its cycles on the MMAs, not on rebuilding descriptors
+            const uint64_t dq = desc_k_major(q_base);
             for (int j = 0; ok && j < sp.n_tiles; ++j, rk.advance(nk)) {
                 const int buf = j & 1;
                 if (!mbar_wait(smem_u32(&c.k_full[rk.slot]), rk.round & 1, abort_flag, a.status)) break;
@@ -756,12 +760,11 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 if (j >= 2 && !mbar_wait(smem_u32(&c.s_free[buf]), ((j >> 1) - 1) & 1, abort_flag, a.status)) break;
                 SS_TR(1, 9 + 4 * j);
                 tc_fence_after();
-                const uint32_t ka = k_base + rk.slot * G::kSlotBytes;
+                const uint64_t dk = desc_k_major(k_base + rk.slot * G::kSlotBytes);
                 #pragma unroll
                 for (int ks = 0; ks < G::kKSteps; ++ks) {
                     const uint32_t hh = ks >> 2, off = (ks & 3) * 32u;
-                    tc_mma(tmem_s + buf * TK, desc_k_major(q_base + hh * kQHalfBytes + off),
-                           desc_k_major(ka + hh * G::kBoxBytes + off), G::kIdescS, ks > 0);
+                    tc_mma(tmem_s + buf * TK, dq + ((hh * kQHalfBytes + off) >> 4), dk + ((hh * G::kBoxBytes + off) >> 4), G::kIdescS, ks > 0);
                 }
                 SS_TR(1, 10 + 4 * j);
                 if (kIsDual) {
@@ -791,16 +794,17 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                     if (!mbar_wait(smem_u32(&c.p_full[w][0]), (j >> 1) & 1, abort_flag, a.status)) break;
                     SS_TR(2, 9 + 4 * j);
                     tc_fence_after();
-                    const uint32_t pa = p_base + w * G::kPBytes;
+                    const uint64_t dp = desc_k_major(p_base + w * G::kPBytes), dv = desc_mn_major(va, G::kBoxBytes);
                     #pragma unroll
                     for (int ks = 0; ks < TK / 16; ++ks)
-                        tc_mma(tmem + w * G::kOCols, desc_k_major(pa + (ks >> 2) * (64u * 128u) + (ks & 3) * 32u),
-                               desc_mn_major(va + ks * 2048u, G::kBoxBytes), G::kIdescPV, (j >= 2 || ks > 0) ? 1u : 0u);
+                        tc_mma(tmem + w * G::kOCols, dp + (((ks >> 2) * (64u * 128u) + (ks & 3) * 32u) >> 4), dv + ((ks * 2048u) >> 4),
+                               G::kIdescPV, (j >= 2 || ks > 0) ? 1u : 0u);
                     tc_commit(smem_u32(&c.o_done[w][0]));
                 } else {
                     // keys 64w .. 64w+63 into the accumulator of warpgroup w; P is read from TMEM, where the
                     // warpgroup left it over the first 32 columns of its half of the S buffer
                     const int buf = j & 1;
+                    const uint64_t dv = desc_mn_major(va, G::kBoxBytes);
                     #pragma unroll
                     for (int w = 0; w < 2; ++w) {
                         if (!mbar_wait(smem_u32(&c.p_full[w][buf]), (j >> 1) & 1, abort_flag, a.status)) { ok = false; break; }
@@ -809,8 +813,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                         const uint32_t pa = tmem_s + buf * TK + w * 64;
                         #pragma unroll
                         for (int ks = 0; ks < 4; ++ks)
-                            tc_mma_ts(tmem + w * G::kOCols, pa + ks * 8u, desc_mn_major(va + (w * 4 + ks) * 2048u, G::kBoxBytes),
-                                      G::kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
+                            tc_mma_ts(tmem + w * G::kOCols, pa + ks * 8u, dv + (((w * 4 + ks) * 2048u) >> 4), G::kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
                         tc_commit(smem_u32(&c.o_done[w][buf]));
                     }
                     if (!ok) break;
