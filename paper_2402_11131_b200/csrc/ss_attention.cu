@@ -555,6 +555,18 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     const long long spec_row0 = static_cast<long long>(b) * a.max_nodes * a.gamma;   // first stream row of the sequence
 
     // ---- prologue ---------------------------------------------------------------------------------
+    // Per-sequence scalars (every thread reads them; through L2: under an early launch the SM's L1 may predate
+    // the previous kernel's last writes).  Under the caller's promise they are requested first of all, so that
+    // their latency passes while the barriers are set up (volatile: the loads stay where they are written).
+    int L = 0, T = 0, cap = 0x7fffffff;
+    long long slot0 = 0;
+    auto load_scalars = [&]() {
+        asm volatile("ld.global.cg.s32 %0, [%1];" : "=r"(L) : "l"(a.kv_len + b) : "memory");
+        asm volatile("ld.global.cg.s32 %0, [%1];" : "=r"(T) : "l"(&a.trees[b].n_nodes) : "memory");
+        asm volatile("ld.global.cg.s64 %0, [%1];" : "=l"(slot0) : "l"(a.kv_start + b) : "memory");
+        if (a.kv_capacity != nullptr) asm volatile("ld.global.cg.s32 %0, [%1];" : "=r"(cap) : "l"(a.kv_capacity + b) : "memory");
+    };
+    if (a.prefix_stable) load_scalars();
     // Everything up to the dependency wait touches no global memory, so under programmatic dependent
     // launch it overlaps the tail of the previous kernel in the stream.
     if (tid == 0) {                                       // Q / K producer: the barriers its copies complete on
@@ -598,19 +610,17 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     // Without the caller's promise nothing is read before the wait.  With it (prefix_stable: nothing
     // still in flight writes the cached prefix, the lengths or the trees) the lengths are read and the
     // first prefix tiles requested right away, so HBM streams while the previous kernel drains.
-    if (!a.prefix_stable) dependency_wait();
+    if (!a.prefix_stable) {
+        dependency_wait();
+        load_scalars();
+    }
     if (tid == 0) SS_TR(0, 2);
     constexpr uint32_t kTmemCols = 512;                   // two accumulators and two S buffers of 128 columns
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&c.tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // per-sequence scalars (every thread reads them)
-    // (read through L2: under an early launch the SM's L1 may predate the previous kernel's last writes)
-    int L = __ldcg(a.kv_len + b);
-    int T = min(max(__ldcg(&a.trees[b].n_nodes), 0), a.max_nodes);
-    const long long slot0 = __ldcg(a.kv_start + b);
-    const int cap = a.kv_capacity != nullptr ? __ldcg(a.kv_capacity + b) : 0x7fffffff;
+    T = min(max(T, 0), a.max_nodes);
     bool skip = false;                                    // sequence over its slot capacity: nothing read or written
     if (L < 0 || L + T > cap) {
         skip = true;
@@ -1124,32 +1134,32 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     }
 
     if (C > 1 && warp >= 4) {
-        // Ship the partial rows (one bulk copy of whole lines from Y), arrive on the block's counter, then
-        // wait (bounded) until the block's other CTAs have arrived too: they were launched together and
-        // need nothing from this CTA, so the wait is short.  Each CTA then combines its own share of the
-        // rows, so the tail of the kernel is a C-th of a single merger's.  The CTA barrier orders every
-        // thread's rows in Y before the one thread whose copy, device-scope fence and arrival publish them.
-        fence_async_smem();
-        named_barrier(3, wg_threads);
+        // Publication.  The partial rows wait in Y; every thread copies its 16-byte pieces to the workspace
+        // (whole lines, they stay in L2) and then arrives on the block's counter with release semantics, which
+        // orders its own pieces before its arrival: no barrier, fence or returned value lies between the rows
+        // and their publication.  A call adds 2048 to the counter in total (each of the 256 threads of each of
+        // the C CTAs 8 / C), so between calls it is a multiple of 2048 whatever split factor earlier calls on the
+        // workspace had, and after this CTA's own arrivals it is one again exactly when all C CTAs have arrived.
+        // One thread then waits (bounded) for that: the other CTAs were launched together with this one and need
+        // nothing from it, so the wait is short.
+        named_barrier(3, wg_threads);                                 // Y is complete
+        const int t = tid - kAuxThreads;
+        unsigned int* cnt = reinterpret_cast<unsigned int*>(a.counters) + group;
+        {
+            constexpr int kPieces = rows_cap * static_cast<int>(RB / 16);
+            float4* dstp = reinterpret_cast<float4*>(part_mine);
+            #pragma unroll 4
+            for (int i = t; i < kPieces; i += wg_threads) __stcg(dstp + i, ld_shared_v4(y_base + static_cast<uint32_t>(i) * 16u));
+            asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(cnt), "r"(8u >> a.cluster_shift) : "memory");
+        }
         if (tid == kAuxThreads) {
-            unsigned int* cnt = reinterpret_cast<unsigned int*>(a.counters) + group;
-            bulk_store(part_mine, y_base, static_cast<uint32_t>(rows_cap) * RB);
-            bulk_store_wait_all();
-            asm volatile("fence.proxy.async;" ::: "memory");
-            __threadfence();
-            // Every call adds 8 to the counter in total (each CTA 8 / C), so between calls it is a multiple of
-            // 8 whatever split factor earlier calls on this workspace had, and this call's arrivals end at the
-            // next multiple of 8 above the value this CTA found.
-            const unsigned int prev = atomicAdd(cnt, 8u >> a.cluster_shift);
-            const unsigned int target = (prev | 7u) + 1u;
             bool ok = true;
             const long long t0 = clock64();
             for (;;) {
-                unsigned int now;
+                unsigned int now;       // this thread's own arrival precedes the load (same address, program order)
                 asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(now) : "l"(cnt) : "memory");
-                if (static_cast<int>(now - target) >= 0) break;
+                if ((now & 2047u) == 0u) break;
                 if (*abort_flag || clock64() - t0 > kWaitCycles) { ok = false; break; }
-                __nanosleep(32);
             }
             if (!ok) { c.abort = 1; set_status(a.status, SS_ERR_DEVICE_TIMEOUT); }
             c.merge_ok = ok ? 1 : 0;
@@ -1157,68 +1167,47 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
         named_barrier(3, wg_threads);
         if (tid == kAuxThreads) SS_TR(5, 4);
         if (c.merge_ok && !skip) {
-            // This CTA's share: rows [first, first + share) of the block's partial rows.  They stream through two
-            // shared-memory buffers, RR rows of every CTA of the block per round (bulk copies from L2); the copy
-            // of round i + 1 runs while round i is combined.
+            // This CTA's share: rows [first, first + share) of the block's partial rows, read straight from L2
+            // (past L1, which may hold lines of an earlier call).  Work item: (row, group of four columns); a
+            // thread has the loads of all C sources of its item in flight at once.
             const int share = rows_cap >> a.cluster_shift;
             const int first = static_cast<int>(rank) * share;
-            const int RR = min(share, C == 8 ? 16 : 32);
-            const int n_rounds = share / RR;
-            const uint32_t buf_bytes = static_cast<uint32_t>(C * RR) * RB;
             const size_t cta_stride = static_cast<size_t>(rows_cap) * RP;
-            auto issue_round = [&](int i) {
-                const uint32_t mbar = smem_u32(&c.merge_full[i & 1]);
-                asm volatile("fence.proxy.async;" ::: "memory");      // generic accesses to the buffer and to the partials come first
-                mbar_expect_tx(mbar, buf_bytes);
-                for (int sidx = 0; sidx < C; ++sidx)
-                    bulk_load(merge_base + (i & 1) * buf_bytes + static_cast<uint32_t>(sidx * RR) * RB,
-                              part_group + sidx * cta_stride + static_cast<size_t>(first + i * RR) * RP, static_cast<uint32_t>(RR) * RB, mbar);
-            };
-            named_barrier(1, wg_threads);                             // every warpgroup is done with the staging area
-            if (tid == kAuxThreads) issue_round(0);
-            bool ok = true;
-            for (int i = 0; i < n_rounds; ++i) {                      // every thread runs every round: the barriers stay matched
-                if (i + 1 < n_rounds) {
-                    named_barrier(1, wg_threads);                     // everyone has read buffer (i + 1) & 1
-                    if (tid == kAuxThreads) issue_round(i + 1);
-                }
-                ok = ok && mbar_wait_warp(smem_u32(&c.merge_full[i & 1]), (i >> 1) & 1, abort_flag, a.status);
-                if (!ok) continue;
-                const uint32_t xb = merge_base + (i & 1) * buf_bytes;
-                // work item: (row of the round, group of four columns)
-                for (int w = tid - kAuxThreads; w < RR * (HD / 4); w += wg_threads) {
-                    const int rr = w / (HD / 4), g = w - rr * (HD / 4);
-                    const RowInfo r = row_info(sp, sp.row0 + first + i * RR + rr);
-                    if (!r.valid) continue;
-                    float ms[8], ls[8];
-                    float mx = -INFINITY;
-                    #pragma unroll
-                    for (int sidx = 0; sidx < 8; ++sidx) {
-                        if (sidx < C) {
-                            const float2 t = ld_shared_v2(xb + static_cast<uint32_t>(sidx * RR + rr) * RB + HD * 4u);
-                            ms[sidx] = t.x; ls[sidx] = t.y;
-                            mx = fmaxf(mx, t.x);
-                        }
+            for (int w = t; w < share * (HD / 4); w += wg_threads) {
+                const int rr = w / (HD / 4), g = w - rr * (HD / 4);
+                const RowInfo r = row_info(sp, sp.row0 + first + rr);
+                if (!r.valid) continue;
+                const float* src = part_group + static_cast<size_t>(first + rr) * RP;
+                float4 v[8];
+                float2 ml[8];
+                #pragma unroll
+                for (int sidx = 0; sidx < 8; ++sidx) {
+                    if (sidx < C) {
+                        v[sidx] = __ldcg(reinterpret_cast<const float4*>(src + sidx * cta_stride + g * 4));
+                        ml[sidx] = __ldcg(reinterpret_cast<const float2*>(src + sidx * cta_stride + HD));
                     }
-                    float l = 0.f;
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                    #pragma unroll
-                    for (int sidx = 0; sidx < 8; ++sidx) {
-                        if (sidx < C) {
-                            const float wgt = ms[sidx] == -INFINITY ? 0.f : exp2f(ms[sidx] - mx);   // 0: saw no visible key
-                            l += wgt * ls[sidx];
-                            const float4 t = ld_shared_v4(xb + static_cast<uint32_t>(sidx * RR + rr) * RB + g * 16u);
-                            acc.x += wgt * t.x; acc.y += wgt * t.y; acc.z += wgt * t.z; acc.w += wgt * t.w;
-                        }
-                    }
-                    const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, r);
-                    const float inv = 1.f / l;
-                    uint2 o;
-                    o.x = pack_bf16(acc.x * inv, acc.y * inv);
-                    o.y = pack_bf16(acc.z * inv, acc.w * inv);
-                    *reinterpret_cast<uint2*>(dst.o + g * 4) = o;
-                    if (dst.lse && g == 0) *dst.lse = (mx + log2f(l)) * 0.6931471805599453f;
                 }
+                float mx = -INFINITY;
+                #pragma unroll
+                for (int sidx = 0; sidx < 8; ++sidx)
+                    if (sidx < C) mx = fmaxf(mx, ml[sidx].x);
+                float l = 0.f;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                #pragma unroll
+                for (int sidx = 0; sidx < 8; ++sidx) {
+                    if (sidx < C) {
+                        const float wgt = ml[sidx].x == -INFINITY ? 0.f : exp2f(ml[sidx].x - mx);   // 0: saw no visible key
+                        l += wgt * ml[sidx].y;
+                        acc.x += wgt * v[sidx].x; acc.y += wgt * v[sidx].y; acc.z += wgt * v[sidx].z; acc.w += wgt * v[sidx].w;
+                    }
+                }
+                const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, r);
+                const float inv = 1.f / l;
+                uint2 o;
+                o.x = pack_bf16(acc.x * inv, acc.y * inv);
+                o.y = pack_bf16(acc.z * inv, acc.w * inv);
+                *reinterpret_cast<uint2*>(dst.o + g * 4) = o;
+                if (dst.lse && g == 0) *dst.lse = (mx + log2f(l)) * 0.6931471805599453f;
             }
         }
     }
