@@ -29,9 +29,9 @@
 //
 // Split-KV merge.  Each CTA ends with un-normalised (m, l, O) per row, combines what it holds for a
 // row locally, and -- when the keys were split -- leaves one partial row in the workspace (it stays in
-// L2).  It then arrives on the block's counter and waits, bounded, for the other CTAs of the block
-// (launched with it, needing nothing from it); each CTA combines its own share of the rows and writes
-// bf16 output.
+// L2): every thread stores its pieces and arrives on the block's counter with release semantics.  One
+// thread waits, bounded, for the other CTAs of the block (launched with it, needing nothing from it);
+// each CTA then combines its own share of the rows, read straight from L2, and writes bf16 output.
 //
 // Launch.  Programmatic dependent launch: one thread of each CTA waits for the previous kernel of
 // the stream; before that wait the kernel touches global memory only under the caller's
@@ -116,7 +116,6 @@ struct Ctrl {
     uint32_t tmem_base;
     int abort;
     int merge_ok;                // the block's other CTAs arrived in time
-    unsigned long long merge_full[2];   // a batch of the block's partials has been copied into shared memory
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -190,19 +189,6 @@ __device__ __forceinline__ float2 ld_shared_v2(uint32_t addr) {
     float2 v;
     asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
     return v;
-}
-// contiguous global memory -> shared memory, completing on an mbarrier of this CTA
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-// shared memory -> contiguous global memory; the calling thread commits and waits for the whole group
-__device__ __forceinline__ void bulk_store(void* dst, uint32_t src, uint32_t bytes) {
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void bulk_store_wait_all() {
-    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -591,7 +577,6 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             mbar_init(smem_u32(&c.p_full[s][1]), 4);
             mbar_init(smem_u32(&c.o_done[s][0]), 1);
             mbar_init(smem_u32(&c.o_done[s][1]), 1);
-            mbar_init(smem_u32(&c.merge_full[s]), 1);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -1301,9 +1286,6 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     const size_t row_bytes = static_cast<size_t>(p.head_dim + 4) * 4;
     const size_t stage = plan->mode == kDual ? 5 * 64 * row_bytes : 2048 + kBlockRows * row_bytes;
     if (stage > bytes) bytes = stage;
-    // every CTA of a split block streams its share of the block's partial rows through two buffers
-    const size_t merge_bufs = static_cast<size_t>(2) * c * (c == 8 ? 16 : 32) * row_bytes;
-    if (c > 1 && merge_bufs > bytes) bytes = merge_bufs;
     plan->smem = bytes + 1024;
     // workspace: one arrival counter per group; one partial row per (group, CTA of the group, row)
     const size_t rows_cap = plan->mode == kDual ? 64 : kBlockRows;
