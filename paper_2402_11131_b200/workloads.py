@@ -69,6 +69,8 @@ class StepConfig:
     p_accept_range: Optional[tuple]
     tree_kind: str              # "uniform_parent" (tiny) | "topk_growth"
     max_children: int = 4
+    k_ramp: float = 0.0         # test inputs only: K of cache slot s is scaled by (1 + k_ramp * s), so the
+                                # largest score of a row keeps growing along the keys
 
     @property
     def seed(self) -> int:
@@ -189,7 +191,12 @@ class StepInputs:
         s = layer if slab_seed is None else slab_seed
         kc = vc = None
         if with_slab:
-            kc = _normal_bf16(_rng(c.seed, _TID_K, s), (self.total_slots, H, d))
+            if c.k_ramp:
+                x = _rng(c.seed, _TID_K, s).standard_normal(size=(self.total_slots, H, d), dtype=np.float32)
+                x *= (1.0 + np.float32(c.k_ramp) * np.arange(self.total_slots, dtype=np.float32))[:, None, None]
+                kc = f32_to_bf16_bits(x)
+            else:
+                kc = _normal_bf16(_rng(c.seed, _TID_K, s), (self.total_slots, H, d))
             vc = _normal_bf16(_rng(c.seed, _TID_V, s), (self.total_slots, H, d))
         return LayerInputs(layer, msa and g > 0, qm, qs, ks, vs, kc, vc)
 
@@ -229,8 +236,8 @@ def make_step(cfg: StepConfig, *, q_unit_variance: bool = False) -> StepInputs:
 def custom_config(name: str, *, batch=1, n_layers=1, n_msa_layers=1, n_heads=2, head_dim=64,
                   prefix_len=64, prefix_len_range=None, n_nodes=6, max_depth=2, gamma=3, vocab=512,
                   p_accept=0.6, p_accept_range=None, tree_kind="uniform_parent", max_children=4,
-                  config_id=100) -> StepConfig:
+                  config_id=100, k_ramp=0.0) -> StepConfig:
     """A free-form configuration for tests (edge cases, ragged tails, odd sizes)."""
     return StepConfig(name, config_id, batch, n_layers, n_msa_layers, n_heads, head_dim, prefix_len,
                       prefix_len_range, n_nodes, max_depth, gamma, vocab, p_accept, p_accept_range,
-                      tree_kind, max_children)
+                      tree_kind, max_children, k_ramp)

@@ -94,6 +94,14 @@ EDGE_CASES = {
     "batch_ragged_small": dict(batch=5, prefix_len_range=(0, 300), n_nodes=13, gamma=3, max_depth=3, n_heads=4),
     "many_pairs_short": dict(batch=24, prefix_len_range=(1, 40), n_nodes=8, gamma=2, max_depth=3, n_heads=8),
     "long_prefix_two_heads": dict(prefix_len=9000, n_nodes=16, gamma=3, max_depth=3, n_heads=2, head_dim=128),
+    # the largest score of every row grows by far more than 2^8 from tile to tile: the running maximum is raised,
+    # and the accumulator rescaled, on every tile (<= 64 rows per head, and three row blocks of 128)
+    "growing_scores_small_head": dict(prefix_len=1500, n_nodes=12, gamma=0, max_depth=3, n_heads=40, head_dim=128,
+                                      k_ramp=0.05),
+    "growing_scores_row_blocks": dict(prefix_len=1500, n_nodes=64, gamma=4, max_depth=5, n_heads=40, head_dim=128,
+                                      tree_kind="topk_growth", k_ramp=0.05),
+    "growing_scores_split_keys": dict(prefix_len=3000, n_nodes=40, gamma=2, max_depth=4, n_heads=3, head_dim=64,
+                                      k_ramp=0.03),
 }
 
 
