@@ -45,6 +45,8 @@ class DeviceStep:
 
         self.k_all = torch.empty((nl, st.total_slots, H, d), dtype=torch.bfloat16, device=dev)
         self.v_all = torch.empty_like(self.k_all)
+        # the main-stream queries of all layers lie in one allocation, so that a host copy can fill several layers at once
+        self.q_main_all = torch.empty((nl, B, T, H, d), dtype=torch.bfloat16, device=dev)
         self.q_main, self.o_main, self.q_spec, self.k_spec, self.v_spec, self.o_spec = [], [], [], [], [], []
         self.lse_main, self.lse_spec = [], []
         self.is_msa: List[bool] = []
@@ -62,7 +64,8 @@ class DeviceStep:
                 if distinct_slabs is not None:
                     slab_cache[seed] = (self.k_all[i], self.v_all[i])
             self.is_msa.append(ly.is_msa)
-            self.q_main.append(api.bf16_to_device(ly.q_main, dev))
+            self.q_main_all[i].copy_(api.bf16_to_device(ly.q_main, dev))
+            self.q_main.append(self.q_main_all[i])
             self.o_main.append(torch.zeros((B, T, H, d), dtype=torch.bfloat16, device=dev))
             self.lse_main.append(torch.zeros((B, T, H), dtype=torch.float32, device=dev) if with_lse else None)
             if ly.is_msa:
@@ -75,11 +78,16 @@ class DeviceStep:
                 for lst in (self.q_spec, self.k_spec, self.v_spec, self.o_spec, self.lse_spec):
                     lst.append(None)
             if pinned_host:
-                h = {"q_main": self.q_main[i].cpu().pin_memory()}
+                h = {}
                 if ly.is_msa:
                     h.update(q_spec=self.q_spec[i].cpu().pin_memory(), k_spec=self.k_spec[i].cpu().pin_memory(),
                              v_spec=self.v_spec[i].cpu().pin_memory())
                 self.host_inputs.append(h)
+
+        self.host_q_main_all = self.q_main_all.cpu().pin_memory() if pinned_host else None
+        if pinned_host:
+            for i in range(nl):
+                self.host_inputs[i]["q_main"] = self.host_q_main_all[i]
 
         # attention workspace: sized for the largest layer, shared by all (calls are stream-ordered)
         ws_bytes = 0
