@@ -381,12 +381,25 @@ __device__ __forceinline__ unsigned long long visible_mask(bool cache, int x, in
 // max over 64 scores of (visible ? s * scale : -inf), four independent chains
 template <bool MASKED>
 __device__ __forceinline__ float chunk_max(const uint32_t (&v)[64], float scale, unsigned long long vis) {
-    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
     const uint32_t vlo = static_cast<uint32_t>(vis), vhi = static_cast<uint32_t>(vis >> 32);
+    if (!MASKED) {
+        // every score counts: the extreme of the raw scores, scaled once (the minimum if the scale is negative)
+        float hi[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        if (scale >= 0.f) {
+            #pragma unroll
+            for (int i = 0; i < 64; ++i) hi[i & 3] = fmaxf(hi[i & 3], __uint_as_float(v[i]));
+            return fmaxf(fmaxf(hi[0], hi[1]), fmaxf(hi[2], hi[3])) * scale;
+        }
+        float lo[4] = {INFINITY, INFINITY, INFINITY, INFINITY};
+        #pragma unroll
+        for (int i = 0; i < 64; ++i) lo[i & 3] = fminf(lo[i & 3], __uint_as_float(v[i]));
+        return fminf(fminf(lo[0], lo[1]), fminf(lo[2], lo[3])) * scale;
+    }
+    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
     #pragma unroll
     for (int i = 0; i < 64; ++i) {
         float s = __uint_as_float(v[i]) * scale;
-        if (MASKED) s = (((i < 32 ? vlo : vhi) >> (i & 31)) & 1u) ? s : -INFINITY;
+        s = (((i < 32 ? vlo : vhi) >> (i & 31)) & 1u) ? s : -INFINITY;
         mx[i & 3] = fmaxf(mx[i & 3], s);
     }
     return fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
