@@ -975,160 +975,115 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     const uint32_t o_addr = tmem + lane_base + (warp >= 4 ? wg : 0) * G::kOCols;
     constexpr int RP = G::kMergePitch;                                         // floats per partial row: O, m, l, pad
     constexpr uint32_t RB = RP * 4;                                            // bytes of a partial row
-    constexpr int QW = HD / 4;                                                 // columns one thread combines (kDual)
     constexpr int rows_cap = G::kRowsCap;                                      // partial rows per CTA
     constexpr int wg_threads = 2 * kBlockRows;
     float* const part_group = a.partials + static_cast<size_t>(group) * C * rows_cap * RP;
     float* const part_mine = part_group + static_cast<size_t>(rank) * rows_cap * RP;
-    const int pidx = wg * 2 + copy;                                            // kDual: partial of the row inside the CTA
 
-    // kDual staging area X: [source][64 rows][RP floats], the four CTA-local partials of a row.  A thread
-    // combines one quarter of its row's columns.
-    const uint32_t x_base = merge_base;
-    // outgoing partial rows of this CTA, as they lie in the workspace (kDual: after the staging area;
-    // kPair: after the 2 KB in which the warpgroups exchange their (m, l))
-    const uint32_t y_base = merge_base + (kIsDual ? 4u * 64u * RB : 2048u);
-    auto combine_x = [&](float& m_c, float& l_c, float4 (&acc)[QW / 4]) {
-        float w[4], mp[4], lp[4];
-        float m_new = -INFINITY;
-        #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const float2 t = ld_shared_v2(x_base + static_cast<uint32_t>(k * 64 + lrow) * RB + HD * 4u);
-            mp[k] = t.x; lp[k] = t.y;
-            m_new = fmaxf(m_new, t.x);
-        }
-        float l_new = 0.f;
-        #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            w[k] = mp[k] != -INFINITY ? exp2f(mp[k] - m_new) : 0.f;     // 0: saw no visible key
-            l_new += w[k] * lp[k];
-        }
-        #pragma unroll
-        for (int i = 0; i < QW / 4; ++i) {
-            const uint32_t col = static_cast<uint32_t>(pidx * QW + i * 4) * 4u;
-            float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
-            #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const float4 t = ld_shared_v4(x_base + static_cast<uint32_t>(k * 64 + lrow) * RB + col);
-                r.x += w[k] * t.x; r.y += w[k] * t.y; r.z += w[k] * t.z; r.w += w[k] * t.w;
-            }
-            acc[i] = r;
-        }
-        m_c = m_new;
-        l_c = l_new;
-    };
+    // Shared memory after the main loop: 2 KB in which the warpgroups exchange their (m, l) (the first thing
+    // a finished warpgroup writes); once both warpgroups are done, kDual: Z, the rows of copy 1 on their way
+    // to copy 0; then Y, the outgoing partial rows of this CTA as they lie in the workspace.
+    // kPair: a warpgroup that is done has seen the last S land, so the query tile under merge_base is free.
+    // kDual: the other warpgroup may still have a tile to go, so the (m, l) get 2 KB of their own after the rings.
+    const uint32_t ml_base = kIsDual ? v_base + nv_slots * G::kSlotBytes : merge_base;   // [warpgroup][128 lanes] (m, l)
+    const uint32_t z_base = merge_base + 2048u;                                // kDual: [64 rows][RP floats]
+    const uint32_t y_base = z_base + (kIsDual ? 64u * RB : 0u);                // [rows_cap][RP floats]
     if (warp >= 4) {
-        // What is written below overlaps the query tile, P and the K/V slots: the query copy must have
-        // landed and every MMA of the CTA must be complete (each warpgroup has seen its last P V land).
+        // What is written below (except the (m, l)) overlaps the query tile, P and the K/V slots: the query copy
+        // must have landed and every MMA of the CTA must be complete (each warpgroup has seen its last P V land).
         mbar_wait_warp(smem_u32(&c.q_full), 0, abort_flag, a.status);
         const bool any_valid = __any_sync(0xffffffffu, ri.valid);
+        // Both accumulators of a TMEM lane can be read by either of the lane's two threads (one per
+        // warpgroup).  The two exchange (m, l) through shared memory; then warpgroup 0 combines columns
+        // [0, kSplitCol) of the lane's two partials and warpgroup 1 the rest.
+        asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(ml_base + static_cast<uint32_t>(wg * kBlockRows + row_in_blk) * 8u),
+                     "f"(m_run), "f"(l_run) : "memory");
+        tc_fence_before();
+        named_barrier(2, wg_threads);
+        tc_fence_after();
+        if (tid == kAuxThreads) SS_TR(5, 1);
+        const float2 other = ld_shared_v2(ml_base + static_cast<uint32_t>((wg ^ 1) * kBlockRows + row_in_blk) * 8u);
+        float m_out = fmaxf(m_run, other.x);
+        const float w_me = m_run != -INFINITY ? exp2f(m_run - m_out) : 0.f;      // 0: saw no visible key
+        const float w_ot = other.x != -INFINITY ? exp2f(other.x - m_out) : 0.f;
+        float l_out = w_me * l_run + w_ot * other.y;
+        // an accumulator that no MMA has written holds anything: it is not read (kDual: warpgroup w has tiles w, w+2, ..)
+        const bool has_ot = kIsDual ? sp.n_tiles > (wg ^ 1) : has_acc;
+        const uint32_t o_other = tmem + lane_base + (wg ^ 1) * G::kOCols;
+        const int c_lo = wg == 0 ? 0 : G::kSplitCol, c_hi = wg == 0 ? G::kSplitCol : HD;
+        float v[G::kSplitCol];                                                   // this thread's columns of the lane's combined partial
+        #pragma unroll
+        for (int cc = 0; cc < G::kSplitCol; cc += 16) {
+            const int c0 = c_lo + cc;
+            uint32_t mine[16], theirs[16];
+            #pragma unroll
+            for (int i = 0; i < 16; ++i) { mine[i] = 0u; theirs[i] = 0u; }
+            if (any_valid && c0 < c_hi) {                                        // warp-uniform
+                if (has_acc) tmem_ld16<0>(o_addr + c0, mine);
+                if (has_ot) tmem_ld16<0>(o_other + c0, theirs);
+                tmem_wait_ld();
+            }
+            #pragma unroll
+            for (int i = 0; i < 16; ++i) v[cc + i] = w_me * __uint_as_float(mine[i]) + w_ot * __uint_as_float(theirs[i]);
+        }
         if (kIsDual) {
-            named_barrier(2, wg_threads);
-            if (tid == kAuxThreads) SS_TR(5, 1);
-            const uint32_t srow = x_base + static_cast<uint32_t>(pidx * 64 + lrow) * RB;
-            if (any_valid) {
+            // the lane's partial covers the keys of its copy; copy 1 hands its rows to copy 0 through Z
+            const uint32_t zrow = z_base + static_cast<uint32_t>(lrow) * RB;
+            if (copy == 1) {
                 #pragma unroll
-                for (int c0 = 0; c0 < HD; c0 += 16) {
-                    uint32_t orr[16];
-                    if (has_acc) { tmem_ld16<0>(o_addr + c0, orr); tmem_wait_ld(); }
-                    else { for (int i = 0; i < 16; ++i) orr[i] = 0u; }
-                    if (ri.valid) {
-                        #pragma unroll
-                        for (int i = 0; i < 16; i += 4) st_shared_v4(srow + (c0 + i) * 4u, orr[i], orr[i + 1], orr[i + 2], orr[i + 3]);
-                    }
-                }
-                if (ri.valid) st_shared_v4(srow + HD * 4u, __float_as_uint(m_run), __float_as_uint(l_run), 0u, 0u);
+                for (int cc = 0; cc < G::kSplitCol; cc += 4)
+                    if (c_lo + cc < c_hi)
+                        st_shared_v4(zrow + (c_lo + cc) * 4u, __float_as_uint(v[cc]), __float_as_uint(v[cc + 1]), __float_as_uint(v[cc + 2]),
+                                     __float_as_uint(v[cc + 3]));
+                if (wg == 0) st_shared_v4(zrow + HD * 4u, __float_as_uint(m_out), __float_as_uint(l_out), 0u, 0u);
             }
             if (tid == kAuxThreads) SS_TR(5, 2);
             named_barrier(1, wg_threads);
-            // each of the row's four threads combines one quarter of the columns
-            if (ri.valid) {
-                float m_out = -INFINITY, l_out = 0.f;
-                float4 acc[QW / 4];
-                combine_x(m_out, l_out, acc);
-                if (C == 1) {
-                    if (!skip) {
-                        const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, ri);
-                        const float inv = 1.f / l_out;
-                        #pragma unroll
-                        for (int i = 0; i < QW / 4; ++i) {
-                            uint2 o;
-                            o.x = pack_bf16(acc[i].x * inv, acc[i].y * inv);
-                            o.y = pack_bf16(acc[i].z * inv, acc[i].w * inv);
-                            *reinterpret_cast<uint2*>(dst.o + pidx * QW + i * 4) = o;
-                        }
-                        if (dst.lse && pidx == 0) *dst.lse = (m_out + log2f(l_out)) * 0.6931471805599453f;
-                    }
-                } else {
-                    // the partial row goes to the outgoing area Y, in the staging area's row order
-                    const uint32_t yrow = y_base + static_cast<uint32_t>(lrow) * RB;
-                    #pragma unroll
-                    for (int i = 0; i < QW / 4; ++i)
-                        st_shared_v4(yrow + static_cast<uint32_t>(pidx * QW + i * 4) * 4u, __float_as_uint(acc[i].x), __float_as_uint(acc[i].y),
-                                     __float_as_uint(acc[i].z), __float_as_uint(acc[i].w));
-                    if (pidx == 0) st_shared_v4(yrow + HD * 4u, __float_as_uint(m_out), __float_as_uint(l_out), 0u, 0u);
-                }
-            }
-            if (tid == kAuxThreads) SS_TR(5, 3);
-        } else {
-            // kPair: both accumulators of a row sit in the row's TMEM lane, so either thread of the row can
-            // read both.  The threads exchange (m, l) through shared memory; then warpgroup 0 finishes
-            // columns [0, kSplitCol) of the row and warpgroup 1 the rest.
-            const uint32_t ml_base = merge_base;                          // [warpgroup][128 rows] (m, l)
-            asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(ml_base + static_cast<uint32_t>(wg * kBlockRows + row_in_blk) * 8u),
-                         "f"(m_run), "f"(l_run) : "memory");
-            tc_fence_before();
-            named_barrier(2, wg_threads);
-            tc_fence_after();
-            if (tid == kAuxThreads) SS_TR(5, 1);
-            const float2 other = ld_shared_v2(ml_base + static_cast<uint32_t>((wg ^ 1) * kBlockRows + row_in_blk) * 8u);
-            const float m_out = fmaxf(m_run, other.x);
-            const float w_me = m_run != -INFINITY ? exp2f(m_run - m_out) : 0.f;      // 0: saw no visible key
-            const float w_ot = other.x != -INFINITY ? exp2f(other.x - m_out) : 0.f;
-            const float l_out = w_me * l_run + w_ot * other.y;
-            const uint32_t o_other = tmem + lane_base + (wg ^ 1) * G::kOCols;
-            constexpr int c_lo_1 = G::kSplitCol;
-            const int c_lo = wg == 0 ? 0 : c_lo_1, c_hi = wg == 0 ? c_lo_1 : HD;
-            const bool write_out = C == 1 && ri.valid && !skip;
-            OutPtr dst;
-            dst.o = nullptr; dst.lse = nullptr;
-            if (write_out) dst = out_ptr<HD>(a, b, h, spec_row0, ri);
-            const float inv = C == 1 ? 1.f / l_out : 1.f;
-            const float f_me = w_me * inv, f_ot = w_ot * inv;
-            const uint32_t yrow = y_base + static_cast<uint32_t>(row_in_blk) * RB;
-            if (any_valid) {
+            if (copy == 0) {
+                const float2 z = ld_shared_v2(zrow + HD * 4u);
+                const float m_f = fmaxf(m_out, z.x);
+                const float w_a = m_out != -INFINITY ? exp2f(m_out - m_f) : 0.f;
+                const float w_b = z.x != -INFINITY ? exp2f(z.x - m_f) : 0.f;
+                l_out = w_a * l_out + w_b * z.y;
+                m_out = m_f;
                 #pragma unroll
-                for (int cc = 0; cc < G::kSplitCol; cc += 16) {
-                    const int c0 = c_lo + cc;
-                    if (c0 >= c_hi) break;                                // warp-uniform: wg is the same for the whole warp
-                    uint32_t mine[16], theirs[16];
-                    if (has_acc) {
-                        tmem_ld16<0>(o_addr + c0, mine);
-                        tmem_ld16<0>(o_other + c0, theirs);
-                        tmem_wait_ld();
-                    } else {
-                        for (int i = 0; i < 16; ++i) { mine[i] = 0u; theirs[i] = 0u; }
-                    }
-                    float v[16];
-                    #pragma unroll
-                    for (int i = 0; i < 16; ++i) v[i] = f_me * __uint_as_float(mine[i]) + f_ot * __uint_as_float(theirs[i]);
-                    if (C == 1) {
-                        if (write_out) store_bf16x16(dst.o + c0, v);
-                    } else {
-                        #pragma unroll
-                        for (int i = 0; i < 16; i += 4)
-                            st_shared_v4(yrow + (c0 + i) * 4u, __float_as_uint(v[i]), __float_as_uint(v[i + 1]), __float_as_uint(v[i + 2]),
-                                         __float_as_uint(v[i + 3]));
+                for (int cc = 0; cc < G::kSplitCol; cc += 4) {
+                    if (c_lo + cc < c_hi) {
+                        const float4 t = ld_shared_v4(zrow + (c_lo + cc) * 4u);
+                        v[cc] = w_a * v[cc] + w_b * t.x; v[cc + 1] = w_a * v[cc + 1] + w_b * t.y;
+                        v[cc + 2] = w_a * v[cc + 2] + w_b * t.z; v[cc + 3] = w_a * v[cc + 3] + w_b * t.w;
                     }
                 }
             }
-            if (C == 1) {
-                if (write_out && dst.lse && wg == 0) *dst.lse = (m_out + log2f(l_out)) * 0.6931471805599453f;
-            } else if (wg == 0) {
-                st_shared_v4(yrow + HD * 4u, __float_as_uint(m_out), __float_as_uint(l_out), 0u, 0u);
-            }
-            if (tid == kAuxThreads) SS_TR(5, 3);
         }
+        // the thread now holds its columns of the row's partial over all keys of this CTA (kDual: copy 0 only)
+        if (!kIsDual || copy == 0) {
+            if (C == 1) {
+                if (ri.valid && !skip) {
+                    const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, ri);
+                    const float inv = 1.f / l_out;
+                    #pragma unroll
+                    for (int cc = 0; cc < G::kSplitCol; cc += 16) {
+                        if (c_lo + cc < c_hi) {
+                            float o[16];
+                            #pragma unroll
+                            for (int i = 0; i < 16; ++i) o[i] = v[cc + i] * inv;
+                            store_bf16x16(dst.o + c_lo + cc, o);
+                        }
+                    }
+                    if (dst.lse && wg == 0) *dst.lse = (m_out + log2f(l_out)) * 0.6931471805599453f;
+                }
+            } else {
+                const uint32_t yrow = y_base + static_cast<uint32_t>(lrow) * RB;
+                #pragma unroll
+                for (int cc = 0; cc < G::kSplitCol; cc += 4)
+                    if (c_lo + cc < c_hi)
+                        st_shared_v4(yrow + (c_lo + cc) * 4u, __float_as_uint(v[cc]), __float_as_uint(v[cc + 1]), __float_as_uint(v[cc + 2]),
+                                     __float_as_uint(v[cc + 3]));
+                if (wg == 0) st_shared_v4(yrow + HD * 4u, __float_as_uint(m_out), __float_as_uint(l_out), 0u, 0u);
+            }
+        }
+        if (tid == kAuxThreads) SS_TR(5, 3);
     }
 
     if (C > 1 && warp >= 4) {
@@ -1287,17 +1242,18 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     const size_t p_total = plan->mode == kDual ? static_cast<size_t>(2) * 3 * 64 * 128 : 0;      // kPair keeps P in TMEM
     const size_t qp = static_cast<size_t>(halves) * kBlockRows * 128 + p_total;
     const size_t slot = static_cast<size_t>(halves) * kTileKeys * 128;
-    int slots = static_cast<int>((kMaxDynSmem - 1024 - qp) / slot);
+    const size_t ml_own = plan->mode == kDual ? 2048 : 0;    // kDual: the warpgroups' (m, l) exchange is not aliased
+    int slots = static_cast<int>((kMaxDynSmem - 1024 - ml_own - qp) / slot);
     if (slots > 2 * kMaxSlots) slots = 2 * kMaxSlots;
     if (slots < 4) return false;
     // a K slot is held until S is queued, a V slot until P V has completed: the odd slot goes to V
     plan->n_kslots = slots / 2;
     plan->n_vslots = slots - plan->n_kslots > kMaxSlots ? kMaxSlots : slots - plan->n_kslots;
-    size_t bytes = qp + static_cast<size_t>(plan->n_kslots + plan->n_vslots) * slot;
-    // after the pipeline the same memory stages partial rows ((head_dim + 4) floats each): kDual its four
-    // CTA-local partials of every row and the outgoing rows (5 x 64 rows), kPair 2 KB and 128 outgoing rows
+    size_t bytes = qp + static_cast<size_t>(plan->n_kslots + plan->n_vslots) * slot + ml_own;
+    // after the pipeline the same memory stages partial rows ((head_dim + 4) floats each): 2 KB, then kDual 64
+    // rows in transit between the copies and 64 outgoing rows, kPair 128 outgoing rows
     const size_t row_bytes = static_cast<size_t>(p.head_dim + 4) * 4;
-    const size_t stage = plan->mode == kDual ? 5 * 64 * row_bytes : 2048 + kBlockRows * row_bytes;
+    const size_t stage = 2048 + (plan->mode == kDual ? 2 * 64 : kBlockRows) * row_bytes;
     if (stage > bytes) bytes = stage;
     plan->smem = bytes + 1024;
     // workspace: one arrival counter per group; one partial row per (group, CTA of the group, row)
