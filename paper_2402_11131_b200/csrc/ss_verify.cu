@@ -30,7 +30,7 @@ tree_verify_kernel(const float* __restrict__ logits, const int32_t* __restrict__
                    Cand* __restrict__ partials) {
     const int chunk = blockIdx.x, t = blockIdx.y, b = blockIdx.z;
     wait_for_previous_kernel();
-    const int T = trees[b].n_nodes;
+    const int T = min(max(trees[b].n_nodes, 0), max_nodes);     // a descriptor is never trusted beyond the arrays' extent
     __shared__ Cand s_red[kVerifyThreads / 32];
     __shared__ int32_t s_am[SS_MAX_NODES];
     __shared__ bool s_last;
