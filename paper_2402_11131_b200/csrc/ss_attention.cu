@@ -8,6 +8,7 @@
 // block's transient stream keys (node-major) are cut into 16-key units and CTA r takes units
 // [U*r/C, U*(r+1)/C), so every CTA of a block streams the same number of bytes.  The CTAs of a pair
 // run in the same wave, so a K/V tile crosses HBM once and is served from L2 to the other row blocks.
+// A batch (up to 32 sequences, no key split) is dispatched longest prefix first.
 //
 // Inside a CTA.
 //   threads 0, 96  TMA producers of the K ring and of the V ring (mbarrier complete_tx); swizzle-128B
@@ -522,7 +523,8 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     const int group = blockIdx.x >> a.cluster_shift;       // (pair, row block): the CTAs that share its keys
     const int rb = kIsDual ? 0 : group % a.n_blocks;
     const int pair = kIsDual ? group : group / a.n_blocks;
-    const int b = pair / a.n_heads, h = pair - b * a.n_heads;
+    int b = pair / a.n_heads;                              // the sequence (for a batch: its place in the dispatch order, see below)
+    const int h = pair - b * a.n_heads;
     const int nk = a.n_kslots, nv_slots = a.n_vslots;
     volatile int* abort_flag = &c.abort;
 
@@ -551,7 +553,6 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     const uint32_t k_base = p_base + 2u * G::kPBytes;                   // [slot][half][128 keys][128 B]
     const uint32_t v_base = k_base + nk * G::kSlotBytes;                // [slot][half][128 keys][128 B]
     const uint32_t merge_base = base;                                   // aliases everything above, after the main loop
-    const long long spec_row0 = static_cast<long long>(b) * a.max_nodes * a.gamma;   // first stream row of the sequence
 
     // ---- prologue ---------------------------------------------------------------------------------
     // Per-sequence scalars (every thread reads them; through L2: under an early launch the SM's L1 may predate
@@ -559,7 +560,21 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     // their latency passes while the barriers are set up (volatile: the loads stay where they are written).
     int L = 0, T = 0, cap = 0x7fffffff;
     long long slot0 = 0;
+    // A batch whose grid takes several waves is dispatched longest sequence first (CTAs start in the order of
+    // their index), so that the last wave holds the short ones: place s of the order goes to the sequence with
+    // the s-th longest prefix.  Every warp ranks the (at most 32) lengths for itself.
+    const bool by_length = a.batch > 1 && a.batch <= 32 && C == 1;
     auto load_scalars = [&]() {
+        if (by_length) {
+            int len = -1;
+            if (lane < a.batch) asm volatile("ld.global.cg.s32 %0, [%1];" : "=r"(len) : "l"(a.kv_len + lane) : "memory");
+            int longer = 0;                                // sequences that come before this lane's in the order
+            for (int o = 0; o < a.batch; ++o) {
+                const int other = __shfl_sync(0xffffffffu, len, o);
+                longer += (other > len || (other == len && o < lane)) ? 1 : 0;
+            }
+            b = __ffs(__ballot_sync(0xffffffffu, lane < a.batch && longer == b)) - 1;
+        }
         asm volatile("ld.global.cg.s32 %0, [%1];" : "=r"(L) : "l"(a.kv_len + b) : "memory");
         asm volatile("ld.global.cg.s32 %0, [%1];" : "=r"(T) : "l"(&a.trees[b].n_nodes) : "memory");
         asm volatile("ld.global.cg.s64 %0, [%1];" : "=l"(slot0) : "l"(a.kv_start + b) : "memory");
@@ -612,6 +627,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
         dependency_wait();
         load_scalars();
     }
+    const long long spec_row0 = static_cast<long long>(b) * a.max_nodes * a.gamma;   // first stream row of the sequence
     if (tid == 0) SS_TR(0, 2);
     constexpr uint32_t kTmemCols = 512;                   // two accumulators and two S buffers of 128 columns
     if (warp == 1) {
