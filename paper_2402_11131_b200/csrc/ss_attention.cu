@@ -87,6 +87,10 @@ struct alignas(64) AttnArgs {
     int cluster, cluster_shift;      // CTAs that share a block's keys; cluster = 1 << cluster_shift
     int n_kslots, n_vslots;          // ring depths
     int head_coord;                  // 1, or 0 when all heads share one K/V (head stride 0)
+    int gamma_magic;                 // ceil(65536 / gamma): x / gamma == (x * gamma_magic) >> 16 for x < 256
+    int n_prefetch;                  // leading CTAs of the grid that only ask the L2 for the call's tiles
+    const char *k_ptr, *v_ptr, *q_ptr, *qs_ptr, *ks_ptr, *vs_ptr;    // the same tensors as plain pointers (prefetch CTAs)
+    long long kv_slot_stride, kv_head_stride;                        // elements
     int prefix_stable;               // the caller's SS_ATTN_PREFIX_STABLE promise
     float scale_log2;                // sm_scale * log2(e)
     __nv_bfloat16* o_main;
@@ -272,8 +276,9 @@ __device__ __forceinline__ uint64_t desc_mn_major(uint32_t addr, uint32_t lbo) {
            (static_cast<uint64_t>(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 // Instruction descriptor: fp32 accumulator, bf16 A and B, M = 128
-__host__ __device__ constexpr uint32_t idesc_bf16(int n, bool b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | (static_cast<uint32_t>(n >> 3) << 17) |
+__host__ __device__ constexpr uint32_t idesc_bf16(int n, bool a_mn_major, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (a_mn_major ? (1u << 15) : 0u) | (b_mn_major ? (1u << 16) : 0u) |
+           (static_cast<uint32_t>(n >> 3) << 17) |
            (static_cast<uint32_t>(kBlockRows >> 4) << 24);
 }
 
@@ -307,7 +312,7 @@ struct Ring {
     }
 };
 
-__device__ __forceinline__ Span make_span(const AttnArgs& a, int L, int T, int rank, int rb) {
+__device__ __forceinline__ Span make_span(const AttnArgs& a, int L, int T, int rank, int rb, int unit) {
     Span s;
     s.L = L; s.T = T; s.gamma = a.gamma; s.tmax8 = a.tmax8;
     s.n_stream = T * a.gamma;
@@ -320,15 +325,15 @@ __device__ __forceinline__ Span make_span(const AttnArgs& a, int L, int T, int r
     if (x1 > x0) { slo = x0 / a.gamma * a.gamma; shi = x1; }
     const bool any_row = s.row0 < T || x1 > x0;           // a block without a valid row streams nothing
     const int ec = any_row ? L + T : 0;
-    const int uc = (ec + kUnit - 1) / kUnit, us = (shi - slo + kUnit - 1) / kUnit;
+    const int uc = (ec + unit - 1) / unit, us = (shi - slo + unit - 1) / unit;
     const int u = uc + us;
     // u < 2^28 and rank < 8: the products fit 32 bits; the split factor is a power of two
     const int u0 = static_cast<int>((static_cast<unsigned>(u) * static_cast<unsigned>(rank)) >> a.cluster_shift);
     const int u1 = static_cast<int>((static_cast<unsigned>(u) * static_cast<unsigned>(rank + 1)) >> a.cluster_shift);
-    s.kc0 = min(u0, uc) * kUnit;
-    s.kc1 = min(min(u1, uc) * kUnit, ec);
-    s.ks0 = slo + (max(u0, uc) - uc) * kUnit;
-    s.ks1 = min(slo + (max(u1, uc) - uc) * kUnit, shi);
+    s.kc0 = min(u0, uc) * unit;
+    s.kc1 = min(min(u1, uc) * unit, ec);
+    s.ks0 = slo + (max(u0, uc) - uc) * unit;
+    s.ks1 = min(slo + (max(u1, uc) - uc) * unit, shi);
     s.n_cache_tiles = s.kc1 > s.kc0 ? (s.kc1 - s.kc0 + kTileKeys - 1) / kTileKeys : 0;
     const int nst = s.ks1 > s.ks0 ? (s.ks1 - s.ks0 + kTileKeys - 1) / kTileKeys : 0;
     s.n_tiles = s.n_cache_tiles + nst;
@@ -457,7 +462,7 @@ __device__ __forceinline__ float chunk_exp_pack(const uint32_t (&v)[64], float s
 // in the other half), and the two warpgroups, each with its own accumulator, take alternate tiles, so
 // one tile's softmax overlaps the other's MMAs.  The partials a row then has inside the CTA (two, four)
 // are combined before the merge across CTAs.
-enum Mode { kPair = 0, kDual = 2 };
+enum Mode { kPair = 0, kCols = 1, kDual = 2 };
 
 template <int HD, int MODE>
 struct Geo {
@@ -466,8 +471,8 @@ struct Geo {
     static constexpr int kSlotBytes = kHalves * kBoxBytes;        // one K tile (or one V tile)
     static constexpr int kKSteps = HD / 16;                       // MMA K steps of S = Q K^T
     static constexpr int kMergePitch = HD + 4;                    // floats per partial row: O, m, l, pad
-    static constexpr uint32_t kIdescS = idesc_bf16(kTileKeys, false);
-    static constexpr uint32_t kIdescPV = idesc_bf16(HD, true);
+    static constexpr uint32_t kIdescS = idesc_bf16(kTileKeys, false, false);
+    static constexpr uint32_t kIdescPV = idesc_bf16(HD, false, true);
     static constexpr int kOCols = 128;                            // TMEM columns reserved per accumulator
     static constexpr int kThreads = kAuxThreads + 2 * kBlockRows; // two softmax warpgroups
     static constexpr int kCopies = MODE == kDual ? 2 : 1;
@@ -642,7 +647,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     }
     if (tid == 0) SS_TR(0, 3);
 
-    const Span sp = make_span(a, L, T, static_cast<int>(rank), rb);
+    const Span sp = make_span(a, L, T, static_cast<int>(rank), rb, kUnit);
 
     // K tile j / V tile j of the span -> ring slot st (K: thread 0, V: thread 96)
     auto load_k = [&](int j, int st) {
@@ -1197,6 +1202,12 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     }
 }
 
+}  // namespace ss
+
+#include "ss_attention_cols.cuh"
+
+namespace ss {
+
 // ---------------------------------------------------------------------------------------------
 // host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -1232,7 +1243,7 @@ static bool make_map(CUtensorMap* out, const void* basep, int d, long long n1, l
 }
 
 struct AttnPlan {
-    int tmax8, spec_rows, s0rows, n_blocks, mode, n_kslots, n_vslots, cluster;
+    int tmax8, spec_rows, s0rows, n_blocks, mode, n_kslots, n_vslots, cluster, n_prefetch;
     long long groups;                          // (sequence, head, row block) triples
     size_t smem;
     size_t counter_bytes, partial_bytes;       // workspace after its header
@@ -1246,8 +1257,8 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     plan->tmax8 = (p.max_nodes + 7) / 8 * 8;
     plan->spec_rows = p.gamma > 0 ? (p.max_nodes * p.gamma + 7) / 8 * 8 : 0;
     const int q_rows = plan->tmax8 + plan->spec_rows;
-    plan->mode = q_rows <= 64 ? kDual : kPair;
-    plan->n_blocks = plan->mode == kDual ? 1 : (q_rows + kBlockRows - 1) / kBlockRows;
+    plan->mode = q_rows <= kColsRows ? kCols : kPair;
+    plan->n_blocks = plan->mode != kPair ? 1 : (q_rows + kBlockRows - 1) / kBlockRows;
     // stream rows that share block 0 with the main rows
     plan->s0rows = plan->spec_rows < kBlockRows - plan->tmax8 ? plan->spec_rows : kBlockRows - plan->tmax8;
     // CTAs per (sequence, head, row block): the largest power of two that still fits the grid on the SMs in one wave
@@ -1255,6 +1266,25 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     int c = 1;
     while (c < 8 && plan->groups * (c * 2) <= sm_count()) c *= 2;
     plan->cluster = c;
+    plan->n_prefetch = 0;
+    if (plan->mode == kCols) {
+        // SMs that the worker CTAs leave free run prefetch CTAs (only with the caller's promise about the lengths)
+        const long long workers = plan->groups * c;
+        if ((p.flags & SS_ATTN_PREFIX_STABLE) && workers < sm_count()) plan->n_prefetch = static_cast<int>(sm_count() - workers);
+        // the query tile, then a ring of K/V tiles; sized so that two CTAs share an SM
+        const size_t q_bytes = static_cast<size_t>(halves) * kColsRows * 128, slot = static_cast<size_t>(halves) * kTileKeys * 128;
+        const size_t pad = halves == 1 ? static_cast<size_t>(kTileKeys) * 128 : 0;
+        int slots = static_cast<int>((kColsSmemLimit - 1024 - q_bytes - pad) / slot);
+        if (slots > kColsMaxSlots) slots = kColsMaxSlots;
+        if (slots < 3) return false;
+        plan->n_kslots = slots;
+        plan->n_vslots = 0;
+        plan->smem = q_bytes + static_cast<size_t>(slots) * slot + pad;
+        const size_t row_bytes = static_cast<size_t>(p.head_dim + 4) * 4;
+        plan->counter_bytes = (static_cast<size_t>(plan->groups) * sizeof(int32_t) + 255) / 256 * 256;
+        plan->partial_bytes = c > 1 ? static_cast<size_t>(plan->groups) * c * kColsRows * row_bytes : 0;
+        return true;
+    }
     const size_t p_total = plan->mode == kDual ? static_cast<size_t>(2) * 3 * 64 * 128 : 0;      // kPair keeps P in TMEM
     const size_t qp = static_cast<size_t>(halves) * kBlockRows * 128 + p_total;
     const size_t slot = static_cast<size_t>(halves) * kTileKeys * 128;
@@ -1304,6 +1334,32 @@ static int32_t launch(const AttnArgs& args, const AttnPlan& plan, cudaStream_t s
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, msa_attention_kernel<HD, MODE>, args) == cudaSuccess ? SS_OK : SS_ERR_CUDA;
+}
+
+template <int HD>
+static int32_t launch_cols(const AttnArgs& args, const AttnPlan& plan, cudaStream_t stream) {
+    static bool configured[64] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SS_ERR_CUDA;
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        if (cudaFuncSetAttribute(msa_attention_cols_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kColsSmemLimit - 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(msa_attention_cols_kernel<HD>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 cudaSharedmemCarveoutMaxShared) != cudaSuccess)
+            return SS_ERR_CUDA;
+        configured[dev] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(plan.groups * plan.cluster + plan.n_prefetch), 1, 1);
+    cfg.blockDim = dim3(static_cast<unsigned>(kColsThreads), 1, 1);
+    cfg.dynamicSmemBytes = plan.smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, msa_attention_cols_kernel<HD>, args) == cudaSuccess ? SS_OK : SS_ERR_CUDA;
 }
 
 }  // namespace ss
@@ -1365,6 +1421,12 @@ extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
     a.cluster_shift = 0;
     while ((1 << a.cluster_shift) < plan.cluster) ++a.cluster_shift;
     a.head_coord = shared_heads ? 0 : 1;
+    a.gamma_magic = p->gamma > 0 ? (65536 + p->gamma - 1) / p->gamma : 0;
+    a.n_prefetch = plan.n_prefetch;
+    a.k_ptr = static_cast<const char*>(p->k_cache); a.v_ptr = static_cast<const char*>(p->v_cache);
+    a.q_ptr = static_cast<const char*>(p->q_main); a.qs_ptr = static_cast<const char*>(p->q_spec);
+    a.ks_ptr = static_cast<const char*>(p->k_spec); a.vs_ptr = static_cast<const char*>(p->v_spec);
+    a.kv_slot_stride = p->kv_slot_stride; a.kv_head_stride = p->kv_head_stride;
     a.prefix_stable = (p->flags & SS_ATTN_PREFIX_STABLE) ? 1 : 0;
     a.scale_log2 = p->sm_scale * 1.4426950408889634f;
     a.o_main = static_cast<__nv_bfloat16*>(p->o_main);
@@ -1376,11 +1438,11 @@ extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
     a.counters = reinterpret_cast<int*>(static_cast<char*>(p->workspace) + ss::kWsHeaderBytes);
     a.partials = reinterpret_cast<float*>(static_cast<char*>(p->workspace) + ss::kWsHeaderBytes + plan.counter_bytes);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (plan.mode == ss::kDual) {
+    if (plan.mode == ss::kCols) {
         switch (d) {
-            case 64: return ss::launch<64, ss::kDual>(a, plan, s);
-            case 80: return ss::launch<80, ss::kDual>(a, plan, s);
-            default: return ss::launch<128, ss::kDual>(a, plan, s);
+            case 64: return ss::launch_cols<64>(a, plan, s);
+            case 80: return ss::launch_cols<80>(a, plan, s);
+            default: return ss::launch_cols<128>(a, plan, s);
         }
     }
     switch (d) {
@@ -1400,7 +1462,7 @@ extern "C" int32_t ss_trace_clear() {
     if (cudaGetSymbolAddress(&p, ss::g_trace) != cudaSuccess) return -1;
     if (cudaMemset(p, 0, sizeof(ss::g_trace)) != cudaSuccess) return -1;
     unsigned long long wall[8][6];
-    for (int i = 0; i < 8; ++i) { wall[i][0] = ~0ull; wall[i][1] = 0ull; wall[i][2] = 0ull; wall[i][3] = 0ull; wall[i][4] = 0ull; wall[i][5] = ~0ull; }
+    for (int i = 0; i < 8; ++i) { wall[i][0] = ~0ull; wall[i][1] = 0ull; wall[i][2] = 0ull; wall[i][3] = ~0ull; wall[i][4] = 0ull; wall[i][5] = ~0ull; }
     unsigned long long keys[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     if (cudaMemcpyToSymbol(ss::g_wall, wall, sizeof(wall)) != cudaSuccess) return -1;
     return cudaMemcpyToSymbol(ss::g_key, keys, sizeof(keys)) == cudaSuccess ? 0 : -1;
