@@ -102,7 +102,7 @@ int32_t ss_tree_build(const int32_t* parent, int32_t n_nodes, int32_t gamma, ss_
  * query rows) and the partial rows of blocks whose keys are split over several CTAs
  * (ss_msa_attention_workspace_bytes).  Calls of different shapes may share one workspace as long as they
  * are ordered on one stream and it is large enough for each: a call leaves every counter at a multiple
- * of 2048.
+ * of 4096.
  * Reads no K/V row past slot kv_start[b]+L_b+T_b-1 whose value can reach an output (a tile may touch
  * later slots of the slab; what it finds there is masked or cleared); writes only o_*, lse_* and the
  * workspace.

@@ -140,3 +140,111 @@ def kv_compact(k_all, v_all, L, accept_len, path):
                                  C.byref(new_len))
     _check(rc, "kv_compact")
     return k_dst, v_dst, int(new_len.value)
+
+
+def next_draft(stream_logits, k: int, bonus_token: int, max_nodes: int):
+    """Next tree draft from the stream logits [gamma][V] of the last accepted node.
+    Returns (tokens int32[n], parent int32[n])."""
+    lg = np.ascontiguousarray(stream_logits, dtype=np.float32)
+    gamma, V = lg.shape
+    tokens = np.zeros(max_nodes, dtype=np.int32)
+    parent = np.zeros(max_nodes, dtype=np.int32)
+    n = C.c_int32(0)
+    rc = _load().ssor_next_draft(_p(lg), C.c_int32(gamma), C.c_int32(V), C.c_int32(int(k)), C.c_int32(int(bonus_token)),
+                                 C.c_int32(int(max_nodes)), C.byref(n), _p(tokens), _p(parent))
+    _check(rc, "next_draft")
+    return tokens[:n.value].copy(), parent[:n.value].copy()
+
+
+def tree_prune(logits, tokens, parent, threshold: float, decide=None):
+    """Prunes sub-trees below edges whose early-exit transition probability is under the threshold.
+    logits f32 [T][V].  Returns dict(edge_prob f64[T], keep u8[T], new_index i32[T], kept_nodes i32[n],
+    new_parent i32[n])."""
+    logits = np.ascontiguousarray(logits, dtype=np.float32)
+    tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+    parent = np.ascontiguousarray(parent, dtype=np.int32)
+    T, V = logits.shape
+    prob = np.zeros(T, dtype=np.float64)
+    keep = np.zeros(T, dtype=np.uint8)
+    new_index = np.zeros(T, dtype=np.int32)
+    kept = np.zeros(T, dtype=np.int32)
+    new_parent = np.zeros(T, dtype=np.int32)
+    n = C.c_int32(0)
+    dec = None if decide is None else np.ascontiguousarray(decide, dtype=np.uint8)
+    rc = _load().ssor_tree_prune(_p(logits), _p(tokens), _p(parent), C.c_int32(T), C.c_int32(V), C.c_double(float(threshold)),
+                                 _p(dec), _p(prob), _p(keep), _p(new_index), C.byref(n), _p(kept), _p(new_parent))
+    _check(rc, "tree_prune")
+    return dict(edge_prob=prob, keep=keep, new_index=new_index, kept_nodes=kept[:n.value].copy(),
+                new_parent=new_parent[:n.value].copy())
+
+
+def tree_verify_soft(logits, tokens, parent, eps: float, delta: float, decide=None, path_cap: Optional[int] = None):
+    """Verification with the soft (typical-acceptance) criterion.  Returns the dict of tree_verify plus
+    edge_prob and node_entropy."""
+    logits = np.ascontiguousarray(logits, dtype=np.float32)
+    tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+    parent = np.ascontiguousarray(parent, dtype=np.int32)
+    T, V = logits.shape
+    cap = T if path_cap is None else int(path_cap)
+    path = np.zeros(cap, dtype=np.int32)
+    prob = np.zeros(T, dtype=np.float64)
+    ent = np.zeros(T, dtype=np.float64)
+    ln, last, bonus = C.c_int32(0), C.c_int32(0), C.c_int32(0)
+    dec = None if decide is None else np.ascontiguousarray(decide, dtype=np.uint8)
+    rc = _load().ssor_tree_verify_soft(_p(logits), _p(tokens), _p(parent), C.c_int32(T), C.c_int32(V), C.c_double(float(eps)),
+                                       C.c_double(float(delta)), _p(dec), C.byref(ln), _p(path), C.c_int32(cap),
+                                       C.byref(last), C.byref(bonus), _p(prob), _p(ent))
+    _check(rc, "tree_verify_soft")
+    return dict(accept_len=int(ln.value), path=path, last_node=int(last.value), bonus_token=int(bonus.value),
+                edge_prob=prob, node_entropy=ent)
+
+
+def tree_verify_sampled(logits, tokens, parent, k: int, u, drawn=None, path_cap: Optional[int] = None):
+    """Verification against tokens drawn from the top-k softmax (temperature 1) with the uniforms u[T]."""
+    logits = np.ascontiguousarray(logits, dtype=np.float32)
+    tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+    parent = np.ascontiguousarray(parent, dtype=np.int32)
+    u = np.ascontiguousarray(u, dtype=np.float32)
+    T, V = logits.shape
+    cap = T if path_cap is None else int(path_cap)
+    path = np.zeros(cap, dtype=np.int32)
+    node_token = np.zeros(T, dtype=np.int32)
+    ln, last, bonus = C.c_int32(0), C.c_int32(0), C.c_int32(0)
+    dr = None if drawn is None else np.ascontiguousarray(drawn, dtype=np.int32)
+    rc = _load().ssor_tree_verify_sampled(_p(logits), _p(tokens), _p(parent), C.c_int32(T), C.c_int32(V), C.c_int32(int(k)),
+                                          _p(u), _p(dr), C.byref(ln), _p(path), C.c_int32(cap), C.byref(last),
+                                          C.byref(bonus), _p(node_token))
+    _check(rc, "tree_verify_sampled")
+    return dict(accept_len=int(ln.value), path=path, last_node=int(last.value), bonus_token=int(bonus.value),
+                node_token=node_token)
+
+
+def stream_insert(m, p):
+    """S[t][j] = M[t] + P[j] (Eq. 3 with the identity transformation).  m uint16 [rows][hidden],
+    p uint16 [gamma][hidden] (bf16 bit patterns).  Returns uint16 [rows][gamma][hidden]."""
+    m = np.ascontiguousarray(m, dtype=np.uint16)
+    p = np.ascontiguousarray(p, dtype=np.uint16)
+    rows, hidden = m.shape
+    gamma = p.shape[0]
+    out = np.zeros((rows, gamma, hidden), dtype=np.uint16)
+    _check(_load().ssor_stream_insert(_p(m), _p(p), _p(out), C.c_int64(rows), C.c_int32(gamma), C.c_int32(hidden)),
+           "stream_insert")
+    return out
+
+
+def rotation_table(epsilon: float, gamma: int) -> np.ndarray:
+    """cos / sin of epsilon * n, n = 1..gamma, evaluated in fp64 and rounded to fp32: [gamma][2]."""
+    n = np.arange(1, gamma + 1, dtype=np.float64)
+    return np.stack([np.cos(epsilon * n), np.sin(epsilon * n)], axis=1).astype(np.float32)
+
+
+def value_rotate(v, gamma: int, epsilon: float):
+    """V[t][n] = V[t] * exp(i * epsilon * n) on consecutive (re, im) pairs (Eq. 7).  v uint16 [rows][width].
+    Returns uint16 [rows][gamma][width]."""
+    v = np.ascontiguousarray(v, dtype=np.uint16)
+    rows, width = v.shape
+    out = np.zeros((rows, gamma, width), dtype=np.uint16)
+    cs = np.ascontiguousarray(rotation_table(epsilon, gamma))
+    _check(_load().ssor_value_rotate(_p(v), _p(out), C.c_int64(rows), C.c_int32(gamma), C.c_int32(width), _p(cs)),
+           "value_rotate")
+    return out

@@ -73,6 +73,7 @@ constexpr int kAuxThreads = 128;     // warps 0..3: producers and MMA issuers
 constexpr int kMaxDynSmem = 232448 - 1024;  // 227 KB per CTA less the static control block
 constexpr float kRescaleStep = 8.f;  // raise the running maximum only when it grows by more than 2^8
 constexpr long long kWaitCycles = 2000000000ll;   // bound of every mbarrier wait (~1 s)
+constexpr unsigned int kArrivalsPerCall = 4096u;  // what the CTAs of a split block add to its arrival counter in one call
 
 struct alignas(64) AttnArgs {
     CUtensorMap tm_k, tm_v;          // cache slab    dims (d, H, slots)        box (64, 1, 128)
@@ -88,9 +89,6 @@ struct alignas(64) AttnArgs {
     int n_kslots, n_vslots;          // ring depths
     int head_coord;                  // 1, or 0 when all heads share one K/V (head stride 0)
     int gamma_magic;                 // ceil(65536 / gamma): x / gamma == (x * gamma_magic) >> 16 for x < 256
-    int n_prefetch;                  // leading CTAs of the grid that only ask the L2 for the call's tiles
-    const char *k_ptr, *v_ptr, *q_ptr, *qs_ptr, *ks_ptr, *vs_ptr;    // the same tensors as plain pointers (prefetch CTAs)
-    long long kv_slot_stride, kv_head_stride;                        // elements
     int prefix_stable;               // the caller's SS_ATTN_PREFIX_STABLE promise
     float scale_log2;                // sm_scale * log2(e)
     __nv_bfloat16* o_main;
@@ -312,7 +310,7 @@ struct Ring {
     }
 };
 
-__device__ __forceinline__ Span make_span(const AttnArgs& a, int L, int T, int rank, int rb, int unit) {
+__device__ __forceinline__ Span make_span(const AttnArgs& a, int L, int T, int rank, int rb, int unit, bool front_heavy = false) {
     Span s;
     s.L = L; s.T = T; s.gamma = a.gamma; s.tmax8 = a.tmax8;
     s.n_stream = T * a.gamma;
@@ -328,8 +326,10 @@ __device__ __forceinline__ Span make_span(const AttnArgs& a, int L, int T, int r
     const int uc = (ec + unit - 1) / unit, us = (shi - slo + unit - 1) / unit;
     const int u = uc + us;
     // u < 2^28 and rank < 8: the products fit 32 bits; the split factor is a power of two
-    const int u0 = static_cast<int>((static_cast<unsigned>(u) * static_cast<unsigned>(rank)) >> a.cluster_shift);
-    const int u1 = static_cast<int>((static_cast<unsigned>(u) * static_cast<unsigned>(rank + 1)) >> a.cluster_shift);
+    // front_heavy: the odd units go to the first CTAs (rounding up instead of down)
+    const unsigned round_up = front_heavy ? static_cast<unsigned>(a.cluster - 1) : 0u;
+    const int u0 = static_cast<int>((static_cast<unsigned>(u) * static_cast<unsigned>(rank) + round_up) >> a.cluster_shift);
+    const int u1 = static_cast<int>((static_cast<unsigned>(u) * static_cast<unsigned>(rank + 1) + round_up) >> a.cluster_shift);
     s.kc0 = min(u0, uc) * unit;
     s.kc1 = min(min(u1, uc) * unit, ec);
     s.ks0 = slo + (max(u0, uc) - uc) * unit;
@@ -1111,8 +1111,8 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
         // Publication.  The partial rows wait in Y; every thread copies its 16-byte pieces to the workspace
         // (whole lines, they stay in L2) and then arrives on the block's counter with release semantics, which
         // orders its own pieces before its arrival: no barrier, fence or returned value lies between the rows
-        // and their publication.  A call adds 2048 to the counter in total (each of the 256 threads of each of
-        // the C CTAs 8 / C), so between calls it is a multiple of 2048 whatever split factor earlier calls on the
+        // and their publication.  A call adds 4096 to the counter in total (each of the 256 threads of each of
+        // the C CTAs 16 / C), so between calls it is a multiple of 4096 whatever split factor earlier calls on the
         // workspace had, and after this CTA's own arrivals it is one again exactly when all C CTAs have arrived.
         // One thread then waits (bounded) for that: the other CTAs were launched together with this one and need
         // nothing from it, so the wait is short.
@@ -1124,7 +1124,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             float4* dstp = reinterpret_cast<float4*>(part_mine);
             #pragma unroll 4
             for (int i = t; i < kPieces; i += wg_threads) __stcg(dstp + i, ld_shared_v4(y_base + static_cast<uint32_t>(i) * 16u));
-            asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(cnt), "r"(8u >> a.cluster_shift) : "memory");
+            asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(cnt), "r"(16u >> a.cluster_shift) : "memory");
         }
         if (tid == kAuxThreads) {
             bool ok = true;
@@ -1132,7 +1132,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             for (;;) {
                 unsigned int now;       // this thread's own arrival precedes the load (same address, program order)
                 asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(now) : "l"(cnt) : "memory");
-                if ((now & 2047u) == 0u) break;
+                if ((now & (kArrivalsPerCall - 1u)) == 0u) break;
                 if (*abort_flag || clock64() - t0 > kWaitCycles) { ok = false; break; }
             }
             if (!ok) { c.abort = 1; set_status(a.status, SS_ERR_DEVICE_TIMEOUT); }
@@ -1204,7 +1204,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
 
 }  // namespace ss
 
-#include "ss_attention_cols.cuh"
+#include "ss_attention_small.cuh"
 
 namespace ss {
 
@@ -1243,7 +1243,7 @@ static bool make_map(CUtensorMap* out, const void* basep, int d, long long n1, l
 }
 
 struct AttnPlan {
-    int tmax8, spec_rows, s0rows, n_blocks, mode, n_kslots, n_vslots, cluster, n_prefetch;
+    int tmax8, spec_rows, s0rows, n_blocks, mode, n_kslots, n_vslots, cluster;
     long long groups;                          // (sequence, head, row block) triples
     size_t smem;
     size_t counter_bytes, partial_bytes;       // workspace after its header
@@ -1257,7 +1257,7 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     plan->tmax8 = (p.max_nodes + 7) / 8 * 8;
     plan->spec_rows = p.gamma > 0 ? (p.max_nodes * p.gamma + 7) / 8 * 8 : 0;
     const int q_rows = plan->tmax8 + plan->spec_rows;
-    plan->mode = q_rows <= kColsRows ? kCols : kPair;
+    plan->mode = q_rows <= kSmRows ? kCols : kPair;
     plan->n_blocks = plan->mode != kPair ? 1 : (q_rows + kBlockRows - 1) / kBlockRows;
     // stream rows that share block 0 with the main rows
     plan->s0rows = plan->spec_rows < kBlockRows - plan->tmax8 ? plan->spec_rows : kBlockRows - plan->tmax8;
@@ -1266,23 +1266,18 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     int c = 1;
     while (c < 8 && plan->groups * (c * 2) <= sm_count()) c *= 2;
     plan->cluster = c;
-    plan->n_prefetch = 0;
     if (plan->mode == kCols) {
-        // SMs that the worker CTAs leave free run prefetch CTAs (only with the caller's promise about the lengths)
-        const long long workers = plan->groups * c;
-        if ((p.flags & SS_ATTN_PREFIX_STABLE) && workers < sm_count()) plan->n_prefetch = static_cast<int>(sm_count() - workers);
-        // the query tile, then a ring of K/V tiles; sized so that two CTAs share an SM
-        const size_t q_bytes = static_cast<size_t>(halves) * kColsRows * 128, slot = static_cast<size_t>(halves) * kTileKeys * 128;
-        const size_t pad = halves == 1 ? static_cast<size_t>(kTileKeys) * 128 : 0;
-        int slots = static_cast<int>((kColsSmemLimit - 1024 - q_bytes - pad) / slot);
-        if (slots > kColsMaxSlots) slots = kColsMaxSlots;
+        // the query tile on its way to TMEM, then one ring of K/V tiles (at the end it stages 64 partial rows)
+        const size_t q_bytes = static_cast<size_t>(halves) * kSmRows * 128, slot = static_cast<size_t>(halves) * kTileKeys * 128;
+        int slots = static_cast<int>((kSmDynSmem - q_bytes) / slot);
+        if (slots > kSmMaxSlots) slots = kSmMaxSlots;
         if (slots < 3) return false;
         plan->n_kslots = slots;
         plan->n_vslots = 0;
-        plan->smem = q_bytes + static_cast<size_t>(slots) * slot + pad;
-        const size_t row_bytes = static_cast<size_t>(p.head_dim + 4) * 4;
+        plan->smem = q_bytes + static_cast<size_t>(slots) * slot;
         plan->counter_bytes = (static_cast<size_t>(plan->groups) * sizeof(int32_t) + 255) / 256 * 256;
-        plan->partial_bytes = c > 1 ? static_cast<size_t>(plan->groups) * c * kColsRows * row_bytes : 0;
+        // a split head leaves the partial rows (O, m, l) of each of its CTAs in the workspace
+        plan->partial_bytes = c > 1 ? static_cast<size_t>(plan->groups) * c * kSmRows * (p.head_dim + 4) * 4 : 0;
         return true;
     }
     const size_t p_total = plan->mode == kDual ? static_cast<size_t>(2) * 3 * 64 * 128 : 0;      // kPair keeps P in TMEM
@@ -1342,16 +1337,16 @@ static int32_t launch_cols(const AttnArgs& args, const AttnPlan& plan, cudaStrea
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return SS_ERR_CUDA;
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        if (cudaFuncSetAttribute(msa_attention_cols_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 kColsSmemLimit - 1024) != cudaSuccess ||
-            cudaFuncSetAttribute(msa_attention_cols_kernel<HD>, cudaFuncAttributePreferredSharedMemoryCarveout,
+        if (cudaFuncSetAttribute(msa_attention_small_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmDynSmem) != cudaSuccess ||
+            cudaFuncSetAttribute(msa_attention_small_kernel<HD>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                  cudaSharedmemCarveoutMaxShared) != cudaSuccess)
             return SS_ERR_CUDA;
         configured[dev] = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(plan.groups * plan.cluster + plan.n_prefetch), 1, 1);
-    cfg.blockDim = dim3(static_cast<unsigned>(kColsThreads), 1, 1);
+    cfg.gridDim = dim3(static_cast<unsigned>(plan.groups * plan.cluster), 1, 1);
+    cfg.blockDim = dim3(static_cast<unsigned>(kSmThreads), 1, 1);
     cfg.dynamicSmemBytes = plan.smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -1359,7 +1354,7 @@ static int32_t launch_cols(const AttnArgs& args, const AttnPlan& plan, cudaStrea
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, msa_attention_cols_kernel<HD>, args) == cudaSuccess ? SS_OK : SS_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, msa_attention_small_kernel<HD>, args) == cudaSuccess ? SS_OK : SS_ERR_CUDA;
 }
 
 }  // namespace ss
@@ -1422,11 +1417,6 @@ extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
     while ((1 << a.cluster_shift) < plan.cluster) ++a.cluster_shift;
     a.head_coord = shared_heads ? 0 : 1;
     a.gamma_magic = p->gamma > 0 ? (65536 + p->gamma - 1) / p->gamma : 0;
-    a.n_prefetch = plan.n_prefetch;
-    a.k_ptr = static_cast<const char*>(p->k_cache); a.v_ptr = static_cast<const char*>(p->v_cache);
-    a.q_ptr = static_cast<const char*>(p->q_main); a.qs_ptr = static_cast<const char*>(p->q_spec);
-    a.ks_ptr = static_cast<const char*>(p->k_spec); a.vs_ptr = static_cast<const char*>(p->v_spec);
-    a.kv_slot_stride = p->kv_slot_stride; a.kv_head_stride = p->kv_head_stride;
     a.prefix_stable = (p->flags & SS_ATTN_PREFIX_STABLE) ? 1 : 0;
     a.scale_log2 = p->sm_scale * 1.4426950408889634f;
     a.o_main = static_cast<__nv_bfloat16*>(p->o_main);

@@ -1,0 +1,715 @@
+// Tree-masked multi-stream attention for heads of at most 64 query rows (Eq. 1, Eq. 2).  Included by
+// ss_attention.cu after its helpers.
+//
+// What bounds a tile of 128 keys on one SM is shared-memory bandwidth (128 B per cycle): the 64 KB of the K and
+// V tile are written once by TMA and must be read once by the two MMAs, which is about 1000 cycles -- as long
+// as nothing else goes through shared memory.  So both small operands live in TMEM and are the A operand of
+// their MMA (tcgen05.mma with A in TMEM), and only K and V are read from shared memory:
+//
+//   S = Q K^T     A = the query tile in TMEM (written there once), B = a K tile (K-major), N = 128 keys
+//   O += P V      A = P in TMEM (bf16, written by the softmax threads over the scores they have just read),
+//                 B = the V tile (MN-major), N = head_dim
+//
+// The 64 rows fill half of the 128 TMEM lanes; the other half holds the rows a second time (copy 1).  The
+// copies take alternate tiles: copy c exponentiates tiles c, c + 2, .. into a P buffer of its own, in which the
+// other copy's lanes stay zero, so one tile's exponentials overlap the other tile's MMAs, and each copy
+// accumulates its own partial row, over its own tiles.  There is one score buffer: a copy moves its scores
+// to registers (four softmax threads share a lane, 32 scores each) and hands the buffer back at once.
+//
+// Softmax with a shared reference.  The four threads of a lane exponentiate against one reference m_ref (any
+// value at or above the lane's scores, and not absurdly far above, gives the same result after
+// normalisation): the lane's maximum over the first tile.  A later score that exceeds it by more than 2^8
+// raises it: the copy's softmax threads agree on that through one reducing barrier per tile, exchange their
+// maxima through shared memory, rescale the lane's accumulator and their row sums, and redo the tile's P.
+//
+// Roles (640 threads): warp 0 lane 0 requests tiles (TMA) into one ring, K and V tiles alternating; warp 1
+// lane 0 issues S and hands K slots back; warp 2 lane 0 issues P V and hands V slots back; warps 4..19 are the
+// softmax threads, four to a TMEM lane.
+//
+// End of a CTA.  Copy 1 hands its partial rows (O, m, l) to copy 0 through shared memory.  C = 1: copy 0
+// normalises and writes bf16.  Split heads (C > 1): the combined rows go to the workspace in whole lines, the
+// CTAs of the head meet on its arrival counter, and each combines its share of the rows from all C partials.
+#pragma once
+
+namespace ss {
+
+// developer trace of this kernel
+#ifdef SS_TRACE
+#define SS_TRC(role, slot)                                                                                       \
+    do {                                                                                                         \
+        const int tr_cta_ = static_cast<int>(blockIdx.x);                                                        \
+        if (tr_cta_ >= 0 && tr_cta_ < ss::kTraceCtas && (slot) < ss::kTraceSlots) ss::g_trace[tr_cta_][role][slot] = clock64(); \
+    } while (0)
+#else
+#define SS_TRC(role, slot) do { } while (0)
+#endif
+
+constexpr int kSmRows = 64;                       // query rows of the variant
+constexpr int kSmThreads = 640;
+constexpr int kSmSoftmax = 512;                   // four threads per TMEM lane
+constexpr int kSmMaxSlots = 6;
+constexpr int kSmDynSmem = 216 * 1024;            // one CTA per SM
+
+template <int HD>
+struct GeoS {
+    static constexpr int kHalves = HD > 64 ? 2 : 1;               // 64-element boxes along head_dim
+    static constexpr int kBoxBytes = kTileKeys * 128;             // one TMA box: 128 keys x 128 B
+    static constexpr int kSlotBytes = kHalves * kBoxBytes;        // a K tile or a V tile
+    static constexpr int kQHalfBytes = kSmRows * 128;
+    static constexpr int kQBytes = kHalves * kQHalfBytes;         // staging of the query tile on its way to TMEM
+    static constexpr int kKSteps = HD / 16;
+    static constexpr int kCpt = HD / 4;                           // accumulator columns a thread finishes
+    static constexpr uint32_t kTmemCols = 512;                    // Q (64), O (128), two score buffers (128 each)
+    static constexpr int kPitch = HD + 4;                         // floats of a partial row: O, m, l, pad
+    static constexpr size_t kCtaFloats = static_cast<size_t>(kSmRows) * kPitch;         // workspace of one CTA of a split head
+};
+
+struct CtrlS {
+    unsigned long long q_full, q_ready;        // query tile in shared memory / in TMEM (16 warps)
+    // A slot's K fills and V fills complete on barriers of their own: each is awaited by one thread, which then
+    // sees every phase of its barrier (K and V tiles alternate in a slot when the ring has an odd number of
+    // slots, and a parity wait that is two phases behind would pass at once).
+    unsigned long long slot_full[2][kSmMaxSlots], slot_empty[kSmMaxSlots];
+    // by tile parity = copy that consumes the tile; each barrier is then looked at in every phase by its waiters
+    unsigned long long s_full[2];              // S of a tile complete
+    unsigned long long s_free[2];              // its scores are in registers (the copy's 8 warps): the one score buffer is free
+    unsigned long long p_full[2];              // P of a tile written to the copy's P buffer (8 warps)
+    unsigned long long pv_done[2];             // P V of a tile complete: the copy's P buffer is free
+    unsigned long long anc[SS_MAX_NODES];
+    alignas(16) float xch[4][2 * kSmRows];     // exchange between the four threads of a lane (maxima, row sums)
+    uint32_t tmem_base;
+    int abort;
+    int merge_ok;
+    int wait_limit;                            // bound of every wait, in units of 1024 cycles
+};
+
+__device__ __forceinline__ uint32_t bar_red_or(int id, int threads, bool pred) {
+    uint32_t out;
+    asm volatile("{\n .reg .pred p, q;\n setp.ne.u32 q, %1, 0;\n bar.red.or.pred p, %2, %3, q;\n selp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(out) : "r"(pred ? 1u : 0u), "r"(id), "r"(threads) : "memory");
+    return out;
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};"
+                 ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(taddr) : "memory");
+}
+// waits whose limit comes from the control block (the caller may shorten it through the workspace header)
+__device__ __noinline__ bool mbar_wait_slow_s(uint32_t bar, uint32_t parity, CtrlS* c, int* status) {
+    const long long t0 = clock64();
+    volatile int* abort = &c->abort;
+    const long long limit = static_cast<long long>(*reinterpret_cast<volatile int*>(&c->wait_limit)) << 10;
+    for (;;) {
+        for (int i = 0; i < 256; ++i) {
+            if (mbar_try(bar, parity)) return true;
+            if (*abort) return false;
+        }
+        if (clock64() - t0 > limit) {
+            *abort = 1;
+            set_status(status, SS_ERR_DEVICE_TIMEOUT);
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ bool mbar_wait_s(uint32_t bar, uint32_t parity, CtrlS* c, int* status) {
+    if (mbar_try(bar, parity)) return true;
+    return mbar_wait_slow_s(bar, parity, c, status);
+}
+__device__ __forceinline__ bool mbar_wait_warp_s(uint32_t bar, uint32_t parity, CtrlS* c, int* status) {
+    return __all_sync(0xffffffffu, mbar_wait_s(bar, parity, c, status));
+}
+
+template <int HD>
+__global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(const __grid_constant__ AttnArgs a) {
+    using G = GeoS<HD>;
+    constexpr int TK = kTileKeys;
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    __shared__ __align__(16) CtrlS c;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int C = a.cluster;
+    const int blk = static_cast<int>(blockIdx.x);
+    const uint32_t rank = blk & (C - 1);
+    const int group = blk >> a.cluster_shift;              // (sequence, head)
+    int b = group / a.n_heads;
+    const int h = group - b * a.n_heads;
+    const int n_slots = a.n_kslots;
+    if (tid == 0) SS_TRC(0, 0);
+#ifdef SS_TRACE
+    __shared__ unsigned int s_launch;
+    if (tid == 0) {
+        const unsigned long long key = reinterpret_cast<unsigned long long>(a.o_main);
+        s_launch = 0;
+        for (unsigned int i = 0; i < 8; ++i) {
+            const unsigned long long old = atomicCAS(&g_key[i], 0ull, key);
+            if (old == 0ull || old == key) { s_launch = i; break; }
+        }
+        atomicMin(&g_wall[s_launch & 7][0], wall_ns());
+        atomicMax(&g_wall[s_launch & 7][2], wall_ns());
+        if (blk < kTraceCtas) g_trace[blk][0][150] = static_cast<long long>(wall_ns());
+    }
+#endif
+
+    const uint32_t base = smem_u32(smem_raw);              // 1024-byte aligned (checked below): swizzle atoms
+    const uint32_t q_base = base;                          // [half][64 rows][128 B]: the query tile on its way to TMEM
+    const uint32_t ring_base = q_base + G::kQBytes;        // [slot][half][128 keys][128 B]
+    auto slot_addr = [&](int s) { return ring_base + static_cast<uint32_t>(s) * G::kSlotBytes; };
+
+    // ---- prologue (see msa_attention_kernel: the same launch protocol) ------------------------------
+    int L = 0, T = 0, cap = 0x7fffffff;
+    long long slot0 = 0;
+    const bool by_length = a.batch > 1 && a.batch <= 32 && C == 1;
+    auto load_scalars = [&]() {
+        if (by_length) {
+            int len = -1;
+            if (lane < a.batch) asm volatile("ld.global.cg.s32 %0, [%1];" : "=r"(len) : "l"(a.kv_len + lane) : "memory");
+            int longer = 0;
+            for (int o = 0; o < a.batch; ++o) {
+                const int other = __shfl_sync(0xffffffffu, len, o);
+                longer += (other > len || (other == len && o < lane)) ? 1 : 0;
+            }
+            b = __ffs(__ballot_sync(0xffffffffu, lane < a.batch && longer == b)) - 1;
+        }
+        asm volatile("ld.global.cg.s32 %0, [%1];" : "=r"(L) : "l"(a.kv_len + b) : "memory");
+        asm volatile("ld.global.cg.s32 %0, [%1];" : "=r"(T) : "l"(&a.trees[b].n_nodes) : "memory");
+        asm volatile("ld.global.cg.s64 %0, [%1];" : "=l"(slot0) : "l"(a.kv_start + b) : "memory");
+        if (a.kv_capacity != nullptr) asm volatile("ld.global.cg.s32 %0, [%1];" : "=r"(cap) : "l"(a.kv_capacity + b) : "memory");
+    };
+    if (a.prefix_stable) load_scalars();
+    if (tid == 0) {
+        mbar_init(smem_u32(&c.q_full), 1);
+        for (int s = 0; s < kSmMaxSlots; ++s) { mbar_init(smem_u32(&c.slot_full[0][s]), 1); mbar_init(smem_u32(&c.slot_full[1][s]), 1); }
+        c.abort = 0;
+        c.wait_limit = static_cast<int>(kWaitCycles >> 10);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        tma_prefetch_desc(&a.tm_qm); tma_prefetch_desc(&a.tm_k); tma_prefetch_desc(&a.tm_v);
+        if (a.gamma > 0) { tma_prefetch_desc(&a.tm_qs); tma_prefetch_desc(&a.tm_ks); tma_prefetch_desc(&a.tm_vs); }
+    } else if (tid == 64) {
+        mbar_init(smem_u32(&c.q_ready), 16);
+        for (int s = 0; s < kSmMaxSlots; ++s) mbar_init(smem_u32(&c.slot_empty[s]), 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(smem_u32(&c.s_full[s]), 1);
+            mbar_init(smem_u32(&c.s_free[s]), 8);
+            mbar_init(smem_u32(&c.p_full[s]), 8);
+            mbar_init(smem_u32(&c.pv_done[s]), 1);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    auto dependency_wait = [&]() {
+        if (tid == 0) {
+            SS_TRC(0, 2);
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            SS_TRC(0, 3);
+#ifdef SS_TRACE
+            atomicMin(&g_wall[s_launch & 7][3], wall_ns());
+            atomicMax(&g_wall[s_launch & 7][4], wall_ns());
+            if (blk < kTraceCtas) g_trace[blk][0][151] = static_cast<long long>(wall_ns());
+#endif
+            asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+        }
+        __syncthreads();
+    };
+    if (!a.prefix_stable) {
+        dependency_wait();
+        load_scalars();
+    }
+    const long long spec_row0 = static_cast<long long>(b) * a.max_nodes * a.gamma;
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&c.tmem_base)), "r"(G::kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    T = min(max(T, 0), a.max_nodes);
+    bool skip = false;
+    const bool bad_smem = (base & 1023u) != 0u;           // never expected: nothing is copied to shared memory then
+    if (L < 0 || L + T > cap || bad_smem) {
+        skip = true;
+        L = 0; T = 0;
+    }
+    // whole tiles are dealt out, the first CTAs of a head taking the odd ones: the last CTA has the masked tiles
+    const Span sp = make_span(a, L, T, static_cast<int>(rank), 0, kTileKeys, true);
+
+    // ring entry i: K tile i/2 (even) or V tile i/2 (odd)
+    auto load_entry = [&](int i, int st) {
+        const int j = i >> 1;
+        const bool is_v = (i & 1) != 0;
+        const uint32_t bar = smem_u32(&c.slot_full[i & 1][st]);
+        mbar_expect_tx(bar, G::kSlotBytes);
+        const uint32_t dst = slot_addr(st);
+        const int x = sp.first_key(j);
+        #pragma unroll
+        for (int hh = 0; hh < G::kHalves; ++hh) {
+            if (sp.is_cache(j)) tma_load_3d(dst + hh * G::kBoxBytes, is_v ? &a.tm_v : &a.tm_k, hh * 64, h * a.head_coord, static_cast<int>(slot0 + x), bar);
+            else tma_load_3d(dst + hh * G::kBoxBytes, is_v ? &a.tm_vs : &a.tm_ks, hh * 64, h, static_cast<int>(spec_row0 + x), bar);
+        }
+    };
+    const int n_entries = 2 * sp.n_tiles;
+    // Two tiles are requested right away (before the dependency wait, under the caller's promise); the rest of
+    // the ring follows once the query rows have arrived, which would otherwise queue behind the tiles on their
+    // way into this SM
+    const int n_early = min(n_entries, min(n_slots, 4));
+    auto prefix_only = [&](int j) { return sp.is_cache(j) && sp.first_key(j) + TK <= sp.L; };
+    int n_pre = 0;
+    if (a.prefix_stable) {
+        if (tid == 0) {
+            // the first tiles that lie wholly inside the cached prefix
+            while (n_pre < n_early && prefix_only(n_pre >> 1)) { load_entry(n_pre, n_pre); ++n_pre; }
+        }
+        dependency_wait();
+    }
+    if (tid == 0) {
+        if (skip) set_status(a.status, bad_smem ? SS_ERR_CUDA : SS_ERR_CAPACITY);
+        // the query tile first: nothing can be computed before it is there
+        const uint32_t qbar = smem_u32(&c.q_full);
+        const bool with_spec = a.gamma > 0 && a.s0rows > 0;
+        const uint32_t rows = a.tmax8 + (with_spec ? a.s0rows : 0);
+        mbar_expect_tx(qbar, bad_smem ? 0u : G::kHalves * rows * 128u);
+        #pragma unroll
+        for (int hh = 0; hh < G::kHalves; ++hh) {
+            if (bad_smem) break;
+            const uint32_t dst = q_base + hh * G::kQHalfBytes;
+            tma_load_3d(dst, &a.tm_qm, hh * 64, h, b * a.max_nodes, qbar);
+            if (with_spec) tma_load_3d(dst + a.tmax8 * 128u, &a.tm_qs, hh * 64, h, static_cast<int>(spec_row0), qbar);
+        }
+        for (int i = n_pre; i < n_early; ++i) load_entry(i, i);
+        // the caller may shorten the bound of the device-side waits (workspace word 1, units of 1024 cycles)
+        int lim;
+        asm volatile("ld.global.cg.s32 %0, [%1];" : "=r"(lim) : "l"(a.status + 1) : "memory");
+        if (lim > 0) c.wait_limit = lim;
+        SS_TRC(0, 5);
+    }
+    if (tid >= kAuxThreads && tid < kAuxThreads + SS_MAX_NODES) c.anc[tid - kAuxThreads] = __ldcg(&a.trees[b].anc_mask[tid - kAuxThreads]);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (tid == 0) SS_TRC(0, 6);
+    const uint32_t tmem = c.tmem_base;
+    const uint32_t tmem_q = tmem;                          // 64 columns: the query rows, two bf16 to a column
+    const uint32_t tmem_o = tmem + 64;                     // 128 columns
+    const uint32_t tmem_s = tmem + 192;                    // one score buffer of 128 columns
+    const uint32_t tmem_p = tmem + 320;                    // two P buffers of 64 columns (128 keys as bf16), one per copy
+    int* const status = a.status;
+    // fill number of a slot's barrier of one kind: with an odd number of slots the kinds alternate in a slot
+    const bool odd_ring = (n_slots & 1) != 0;
+    auto fill_parity = [&](const Ring& r) { return static_cast<uint32_t>((odd_ring ? r.round >> 1 : r.round) & 1); };
+    auto wait_slot_full = [&](int kind, const Ring& r) {
+        return mbar_wait_s(smem_u32(&c.slot_full[kind][r.slot]), fill_parity(r), &c, status);
+    };
+
+    // =============================== warp 0: tile requests =======================================
+    if (warp == 0) {
+        if (lane == 0 && n_entries > n_early) {
+            Ring r;
+            r.start();
+            for (int i = 0; i < n_early; ++i) r.advance(n_slots);
+            bool ok = mbar_wait_s(smem_u32(&c.q_ready), 0, &c, status);
+            for (int i = n_early; ok && i < n_entries; ++i) {
+                if (r.round > 0) ok = mbar_wait_s(smem_u32(&c.slot_empty[r.slot]), (r.round - 1) & 1, &c, status);
+                SS_TRC(0, 8 + i);
+                if (ok) { load_entry(i, r.slot); r.advance(n_slots); }
+            }
+            if (!ok) {                 // gave up: let the copies already in flight land before the CTA leaves
+                const int issued = r.slot + r.round * n_slots;
+                Ring d;
+                d.start();
+                for (int i = 0; i < issued; ++i, d.advance(n_slots))
+                    if (i >= issued - n_slots) mbar_drain(smem_u32(&c.slot_full[i & 1][d.slot]), fill_parity(d));
+            }
+        }
+    }
+    // =============================== warp 1: S = Q K^T, A from TMEM ================================
+    else if (warp == 1) {
+        if (lane == 0) {
+            bool ok = mbar_wait_s(smem_u32(&c.q_ready), 0, &c, status);
+            SS_TRC(1, 0);
+            Ring r;
+            r.start();
+            for (int j = 0; ok && j < sp.n_tiles; ++j) {
+                const int buf = j & 1;
+                if (!wait_slot_full(0, r)) break;
+                SS_TRC(1, 8 + 4 * j);
+                // the scores of the tile before must be in registers
+                if (j >= 1 && !mbar_wait_s(smem_u32(&c.s_free[buf ^ 1]), ((j - 1) >> 1) & 1, &c, status)) break;
+                SS_TRC(1, 9 + 4 * j);
+                tc_fence_after();
+                const uint64_t dk = desc_k_major(slot_addr(r.slot));
+                #pragma unroll
+                for (int ks = 0; ks < G::kKSteps; ++ks) {
+                    const uint32_t hh = ks >> 2, off = (ks & 3) * 32u;
+                    tc_mma_ts(tmem_s, tmem_q + ks * 8u, dk + ((hh * G::kBoxBytes + off) >> 4), idesc_bf16(TK, false, false), ks > 0);
+                }
+                tc_commit(smem_u32(&c.s_full[buf]));
+                tc_commit(smem_u32(&c.slot_empty[r.slot]));                   // K may go when S is complete
+                SS_TRC(1, 10 + 4 * j);
+                r.advance(n_slots); r.advance(n_slots);
+            }
+        }
+    }
+    // =============================== warp 2: O += P V, A from TMEM ================================
+    else if (warp == 2) {
+        if (lane == 0) {
+            Ring rv;
+            rv.start();
+            rv.advance(n_slots);
+            bool okq = mbar_wait_s(smem_u32(&c.q_ready), 0, &c, status);     // the P buffers' constant zeros are in place
+            for (int j = 0; okq && j < sp.n_tiles; ++j) {
+                const int buf = j & 1;
+                if (!wait_slot_full(1, rv)) break;
+                SS_TRC(2, 8 + 4 * j);
+                if (!mbar_wait_s(smem_u32(&c.p_full[buf]), (j >> 1) & 1, &c, status)) break;
+                SS_TRC(2, 9 + 4 * j);
+                tc_fence_after();
+                const uint64_t dv = desc_mn_major(slot_addr(rv.slot), G::kBoxBytes);
+                // P of the tile: the copy's buffer, keys 16 ks .. 16 ks + 15 in columns 8 ks .. 8 ks + 7 (zero in the
+                // other copy's lanes)
+                #pragma unroll
+                for (int ks = 0; ks < TK / 16; ++ks)
+                    tc_mma_ts(tmem_o, tmem_p + buf * 64u + 8u * ks, dv + ((ks * 2048u) >> 4), idesc_bf16(HD, false, true),
+                              (j > 0 || ks > 0) ? 1u : 0u);
+                tc_commit(smem_u32(&c.pv_done[buf]));
+                tc_commit(smem_u32(&c.slot_empty[rv.slot]));
+                SS_TRC(2, 10 + 4 * j);
+                rv.advance(n_slots); rv.advance(n_slots);
+            }
+        }
+    }
+    // =============================== warps 4..19: softmax =========================================
+    const int w4 = warp >= 4 ? (warp - 4) >> 2 : 0;                           // which 32 keys of a tile (and which quarter of a row)
+    const int tl = ((warp & 3) << 5) | lane;                                  // TMEM lane = (copy, row)
+    const int copy = tl >> 6, row = tl & 63;
+    const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    float m_ref = -INFINITY, l_part = 0.f;
+    RowInfo ri;
+    ri.valid = false; ri.node = 0; ri.stream = 0;
+    if (warp >= 4) {
+        ri = row_info(sp, row);
+        const unsigned long long anc = ri.valid ? c.anc[ri.node] : 0ull;
+        // ---- the query row of this lane, from shared memory into TMEM: 32 of its elements per thread (two bf16
+        // to a column, as they lie in memory); a lane without a row holds zeros.  The lane's part of the other
+        // copy's P buffer is zero for the whole kernel.
+        {
+            const bool have_q = mbar_wait_warp_s(smem_u32(&c.q_full), 0, &c, status);
+            uint32_t qv[16];
+            #pragma unroll
+            for (int i = 0; i < 16; ++i) qv[i] = 0u;
+            tmem_st16<0>(tmem_p + lane_base + static_cast<uint32_t>((1 - copy) * 64 + 16 * w4), qv);
+            const int hh = w4 >> 1;
+            if (have_q && ri.valid && hh < G::kHalves && !bad_smem) {
+                #pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t piece = static_cast<uint32_t>((w4 & 1) * 4 + i);
+                    const float4 f = ld_shared_v4(q_base + hh * G::kQHalfBytes + row * 128u + ((piece ^ (row & 7)) << 4));
+                    qv[4 * i + 0] = __float_as_uint(f.x); qv[4 * i + 1] = __float_as_uint(f.y);
+                    qv[4 * i + 2] = __float_as_uint(f.z); qv[4 * i + 3] = __float_as_uint(f.w);
+                }
+            }
+            tmem_st16<0>(tmem_q + lane_base + 16u * w4, qv);
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&c.q_ready));
+        }
+        if (tid == kAuxThreads) SS_TRC(5, 6);
+        const bool leader = (tid == kAuxThreads) || (tid == kAuxThreads + 64);      // lane 0 of each copy's first warp
+        const uint32_t p_addr = tmem_p + lane_base + static_cast<uint32_t>(copy * 64 + 16 * w4);   // my 32 keys of a tile as bf16
+        const uint32_t o_addr = tmem_o + lane_base + 32u * w4;
+        int other_seen = 0;                                                    // phases of the other copy's completion barrier seen
+        bool failed = false;
+        // copy c takes the tiles j = c, c + 2, ..: all 128 keys of the tile for its 64 rows
+        for (int j = copy; j < sp.n_tiles; j += 2) {
+            bool ok = true;
+            // every phase of both completion barriers is looked at, in order: a parity wait is then never more than
+            // one phase behind.  P V of tile j - 3 (the other copy's) completed before that of tile j - 2 (this
+            // copy's), which is awaited below before P is overwritten.
+            while (ok && j >= 3 && other_seen <= ((j - 3) >> 1)) {
+                ok = mbar_wait_warp_s(smem_u32(&c.pv_done[1 - copy]), other_seen & 1, &c, status);
+                ++other_seen;
+            }
+            ok = mbar_wait_warp_s(smem_u32(&c.s_full[copy]), (j >> 1) & 1, &c, status) && ok;
+            if (leader) SS_TRC(3, 8 + 6 * j);
+            tc_fence_after();
+            const int x0 = sp.first_key(j), nvk = sp.valid_keys(j);
+            const bool cache = sp.is_cache(j);
+            const bool masked = !cache || x0 + TK > sp.L || nvk < TK;
+            const uint32_t vis = masked ? static_cast<uint32_t>(visible_mask(cache, x0 + 32 * w4, nvk - 32 * w4, sp.L, sp.gamma, ri, anc) & 0xffffffffull)
+                                        : 0xffffffffu;
+            uint32_t sr[32];
+            if (ok) {
+                tmem_ld32<0>(tmem_s + lane_base + 32u * w4, sr);
+                tmem_wait_ld();
+            }
+            // the scores are in registers: S of the next tile (the other copy's) may overwrite the buffer
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&c.s_free[copy]));
+
+            // Raises the lane's reference to its maximum over this tile and rescales what it has accumulated.  The
+            // P V of the tile before this one is the last that can have been issued (they are issued in tile order
+            // and this tile's P is not published yet): once it is complete the accumulator is at rest.
+            auto raise = [&]() {
+                float mx = -INFINITY;
+                #pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const float v = __uint_as_float(sr[i]) * a.scale_log2;
+                    mx = fmaxf(mx, ((vis >> i) & 1u) ? v : -INFINITY);
+                }
+                c.xch[w4][tl] = mx;
+                named_barrier(6 + copy, 256);
+                const float m_new = ri.valid ? fmaxf(fmaxf(m_ref, fmaxf(c.xch[0][tl], c.xch[1][tl])), fmaxf(c.xch[2][tl], c.xch[3][tl]))
+                                             : INFINITY;       // a lane without a row never asks for a raise again
+                const float corr = m_new == m_ref ? 1.f : exp2f(m_ref - m_new);          // 0 when nothing was visible so far
+                m_ref = m_new;
+                l_part *= corr;
+                bool ok2 = true;
+                if (j >= 2) {
+                    while (ok2 && other_seen <= ((j - 1) >> 1)) {
+                        ok2 = mbar_wait_warp_s(smem_u32(&c.pv_done[1 - copy]), other_seen & 1, &c, status);
+                        ++other_seen;
+                    }
+                    tc_fence_after();
+                    if (ok2) {
+                        uint32_t orr[32];
+                        tmem_ld32<0>(o_addr, orr);
+                        tmem_wait_ld();
+                        #pragma unroll
+                        for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * corr);
+                        tmem_st32(o_addr, orr);
+                        tmem_wait_st();
+                    }
+                }
+                named_barrier(6 + copy, 256);                // the exchange buffer may be written again
+                return ok2;
+            };
+
+            if (j < 2) raise();                                               // every thread of the copy, so the barriers inside match
+            // P of this copy's previous tile must have been read before it is overwritten
+            if (j >= 2) ok = mbar_wait_warp_s(smem_u32(&c.pv_done[copy]), ((j - 2) >> 1) & 1, &c, status) && ok;
+            bool leave = false;
+            for (int attempt = 0; attempt < 3; ++attempt) {
+                float tmax = -INFINITY, lsum = 0.f;
+                if (ok) {
+                    uint32_t pk[16];
+                    #pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float t0 = fmaf(__uint_as_float(sr[i]), a.scale_log2, -m_ref);
+                        float t1 = fmaf(__uint_as_float(sr[i + 1]), a.scale_log2, -m_ref);
+                        float e0 = exp2f(t0), e1 = exp2f(t1);
+                        if (masked) {
+                            const bool v0 = (vis >> i) & 1u, v1 = (vis >> (i + 1)) & 1u;
+                            t0 = v0 ? t0 : -INFINITY; t1 = v1 ? t1 : -INFINITY;
+                            e0 = v0 ? e0 : 0.f; e1 = v1 ? e1 : 0.f;
+                        }
+                        tmax = fmaxf(tmax, fmaxf(t0, t1));
+                        lsum += e0 + e1;
+                        pk[i >> 1] = pack_bf16(e0, e1);
+                    }
+                    tmem_st16<0>(p_addr, pk);
+                }
+                if (leader) SS_TRC(3, 9 + 6 * j + (attempt > 0 ? 3 : 0));
+                // one reducing barrier per tile: did a score outgrow its reference, or did a wait run out
+                const uint32_t any = bar_red_or(4 + copy, 256, !ok || tmax > kRescaleStep);
+                if (leader) SS_TRC(3, 10 + 6 * j);
+                if (!any) { l_part += lsum; break; }
+                if (*reinterpret_cast<volatile int*>(&c.abort)) { leave = true; break; }
+                ok = raise() && ok;
+                if (attempt == 2) l_part += lsum;
+            }
+            if (leave) { failed = true; break; }
+            // V rows past the end of the sequence's keys may hold anything (even NaN patterns): P is 0 there,
+            // but 0 * NaN is NaN, so they are cleared: a thread looks after rows (row, row + 64) of the tile
+            const int region_left = (cache ? sp.L + sp.T : sp.n_stream) - x0;
+            if (region_left < TK) {
+                Ring rv;
+                rv.start();
+                for (int i = 0; i < 2 * j + 1; ++i) rv.advance(n_slots);
+                if (mbar_wait_warp_s(smem_u32(&c.slot_full[1][rv.slot]), fill_parity(rv), &c, status)) {
+                    #pragma unroll
+                    for (int up = 0; up < 2; ++up) {
+                        const int vr = row + 64 * up;
+                        if (vr >= region_left && (w4 >> 1) < G::kHalves) {
+                            const uint32_t dst = slot_addr(rv.slot) + (w4 >> 1) * G::kBoxBytes + vr * 128u + (w4 & 1) * 64u;
+                            #pragma unroll
+                            for (int i = 0; i < 4; ++i) st_shared_v4(dst + i * 16, 0u, 0u, 0u, 0u);
+                        }
+                    }
+                    fence_async_smem();
+                }
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&c.p_full[copy]));
+            if (leader) SS_TRC(3, 11 + 6 * j);
+        }
+        // every P V must be complete before the accumulator is read: this copy's last one, and the other copy's
+        if (!failed) {
+            const int n_mine = sp.n_tiles > copy ? (sp.n_tiles - copy + 1) >> 1 : 0;
+            const int n_other = sp.n_tiles > 1 - copy ? (sp.n_tiles - (1 - copy) + 1) >> 1 : 0;
+            bool ok = true;
+            if (n_mine > 0) ok = mbar_wait_warp_s(smem_u32(&c.pv_done[copy]), (n_mine - 1) & 1, &c, status);
+            while (ok && other_seen < n_other) {
+                ok = mbar_wait_warp_s(smem_u32(&c.pv_done[1 - copy]), other_seen & 1, &c, status);
+                ++other_seen;
+            }
+            tc_fence_after();
+        }
+    }
+    __syncwarp();
+    if (tid == kAuxThreads) SS_TRC(5, 0);
+
+    // ======================================== epilogue ==========================================
+    // A lane's partial over the keys of its copy: O in TMEM, the reference, and the sum of its four threads' row
+    // sums.  Copy 1 hands its rows to copy 0 through shared memory (the ring is idle: every copy has landed and
+    // every MMA is complete).  C = 1: copy 0 normalises and writes bf16.  Split head: the combined rows go back
+    // to shared memory and from there, in whole lines, to the workspace (they stay in L2); every thread's pieces
+    // precede its release arrival on the head's counter (a call adds 4096 to it in total), one thread waits
+    // (bounded) for the other CTAs of the head, which were launched with this one and need nothing from it, and
+    // each CTA combines its share of the rows.
+    constexpr int CPT = G::kCpt;
+    constexpr uint32_t YB = G::kPitch * 4;                                    // bytes of a staged row
+    const uint32_t y_base = ring_base;                                        // [64 rows][kPitch floats]
+    float* const part_group = a.partials + static_cast<size_t>(group) * C * G::kCtaFloats;
+    float* const part_mine = part_group + static_cast<size_t>(rank) * G::kCtaFloats;
+    const bool has_acc = sp.n_tiles > 0;
+    if (warp >= 4) {
+        c.xch[w4][tl] = l_part;
+        named_barrier(8, kSmSoftmax);
+        float l_lane = (c.xch[0][tl] + c.xch[1][tl]) + (c.xch[2][tl] + c.xch[3][tl]);
+        const bool aborted = *reinterpret_cast<volatile int*>(&c.abort) != 0;
+        uint32_t orr[32];
+        #pragma unroll
+        for (int i = 0; i < 32; ++i) orr[i] = 0u;
+        if (has_acc && !aborted) {
+            tmem_ld32<0>(tmem_o + lane_base + static_cast<uint32_t>(CPT * w4), orr);
+            tmem_wait_ld();
+        }
+        if (!has_acc || !ri.valid) { m_ref = -INFINITY; l_lane = 0.f; }
+        if (tid == kAuxThreads) SS_TRC(5, 1);
+        const uint32_t yrow = y_base + static_cast<uint32_t>(row) * YB;
+        if (copy == 1) {
+            #pragma unroll
+            for (int i = 0; i < CPT; i += 4) st_shared_v4(yrow + static_cast<uint32_t>(CPT * w4 + i) * 4u, orr[i], orr[i + 1], orr[i + 2], orr[i + 3]);
+            if (w4 == 0) st_shared_v4(yrow + HD * 4u, __float_as_uint(m_ref), __float_as_uint(l_lane), 0u, 0u);
+        }
+        named_barrier(8, kSmSoftmax);
+        float m_out = m_ref, l_out = l_lane;
+        if (copy == 0) {
+            const float2 z = ld_shared_v2(yrow + HD * 4u);
+            m_out = fmaxf(m_ref, z.x);
+            const float wa = m_ref == -INFINITY ? 0.f : exp2f(m_ref - m_out), wb = z.x == -INFINITY ? 0.f : exp2f(z.x - m_out);
+            l_out = wa * l_lane + wb * z.y;
+            #pragma unroll
+            for (int i = 0; i < CPT; i += 4) {
+                const float4 t4 = ld_shared_v4(yrow + static_cast<uint32_t>(CPT * w4 + i) * 4u);
+                orr[i] = __float_as_uint(wa * __uint_as_float(orr[i]) + wb * t4.x);
+                orr[i + 1] = __float_as_uint(wa * __uint_as_float(orr[i + 1]) + wb * t4.y);
+                orr[i + 2] = __float_as_uint(wa * __uint_as_float(orr[i + 2]) + wb * t4.z);
+                orr[i + 3] = __float_as_uint(wa * __uint_as_float(orr[i + 3]) + wb * t4.w);
+            }
+            if (C == 1) {
+                if (ri.valid && !skip && !aborted) {
+                    const float inv = 1.f / l_out;
+                    const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, ri);
+                    #pragma unroll
+                    for (int i = 0; i < CPT; i += 4) {
+                        uint2 o;
+                        o.x = pack_bf16(__uint_as_float(orr[i]) * inv, __uint_as_float(orr[i + 1]) * inv);
+                        o.y = pack_bf16(__uint_as_float(orr[i + 2]) * inv, __uint_as_float(orr[i + 3]) * inv);
+                        *reinterpret_cast<uint2*>(dst.o + CPT * w4 + i) = o;
+                    }
+                    if (dst.lse && w4 == 0) *dst.lse = (m_out + log2f(l_out)) * 0.6931471805599453f;
+                }
+            } else {
+                // same addresses this thread has just read: the combined row replaces copy 1's
+                #pragma unroll
+                for (int i = 0; i < CPT; i += 4) st_shared_v4(yrow + static_cast<uint32_t>(CPT * w4 + i) * 4u, orr[i], orr[i + 1], orr[i + 2], orr[i + 3]);
+                if (w4 == 0) st_shared_v4(yrow + HD * 4u, __float_as_uint(m_out), __float_as_uint(l_out), 0u, 0u);
+            }
+        }
+        if (C > 1) {
+            named_barrier(8, kSmSoftmax);                                     // the staged rows are complete
+            const int t = tid - kAuxThreads;
+            if (!skip && !aborted) {
+                constexpr int kPieces = kSmRows * G::kPitch / 4;
+                float4* dstp = reinterpret_cast<float4*>(part_mine);
+                #pragma unroll 5
+                for (int i = t; i < kPieces; i += kSmSoftmax) __stcg(dstp + i, ld_shared_v4(y_base + static_cast<uint32_t>(i) * 16u));
+            }
+            if (tid == kAuxThreads) SS_TRC(5, 2);
+            // one arrival per warp: the warp barrier orders the lanes' pieces before lane 0's release
+            unsigned int* cnt = reinterpret_cast<unsigned int*>(a.counters) + group;
+            __syncwarp();
+            if (lane == 0) asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(cnt), "r"(256u >> a.cluster_shift) : "memory");
+            if (tid == kAuxThreads) {
+                bool ok = !aborted;
+                const long long t0 = clock64();
+                const long long limit = static_cast<long long>(c.wait_limit) << 10;
+                while (ok) {
+                    unsigned int now;
+                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(now) : "l"(cnt) : "memory");
+                    if ((now & (kArrivalsPerCall - 1u)) == 0u) break;
+                    if (clock64() - t0 > limit) ok = false;
+                }
+                if (!ok) { c.abort = 1; set_status(a.status, SS_ERR_DEVICE_TIMEOUT); }
+                c.merge_ok = ok ? 1 : 0;
+            }
+            named_barrier(3, kSmSoftmax);
+            if (tid == kAuxThreads) SS_TRC(5, 4);
+            if (c.merge_ok && !skip) {
+                // this CTA's share of the rows, read straight from L2 (past L1, which may hold lines of an earlier
+                // call): work item (row, four columns), the loads of all C sources in flight at once
+                const int share = kSmRows >> a.cluster_shift;
+                const int first = static_cast<int>(rank) * share;
+                for (int w = t; w < share * (HD / 4); w += kSmSoftmax) {
+                    const int rr = w / (HD / 4), g4 = w - rr * (HD / 4);
+                    const RowInfo r = row_info(sp, first + rr);
+                    if (!r.valid) continue;
+                    const float* src = part_group + static_cast<size_t>(first + rr) * G::kPitch;
+                    float4 v[8];
+                    float2 ml[8];
+                    #pragma unroll
+                    for (int sidx = 0; sidx < 8; ++sidx) {
+                        if (sidx < C) {
+                            v[sidx] = __ldcg(reinterpret_cast<const float4*>(src + sidx * G::kCtaFloats + g4 * 4));
+                            ml[sidx] = __ldcg(reinterpret_cast<const float2*>(src + sidx * G::kCtaFloats + HD));
+                        }
+                    }
+                    float mx = -INFINITY;
+                    #pragma unroll
+                    for (int sidx = 0; sidx < 8; ++sidx)
+                        if (sidx < C) mx = fmaxf(mx, ml[sidx].x);
+                    float l = 0.f;
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    #pragma unroll
+                    for (int sidx = 0; sidx < 8; ++sidx) {
+                        if (sidx < C) {
+                            const float wgt = ml[sidx].x == -INFINITY ? 0.f : exp2f(ml[sidx].x - mx);   // 0: saw no visible key
+                            l += wgt * ml[sidx].y;
+                            acc.x += wgt * v[sidx].x; acc.y += wgt * v[sidx].y; acc.z += wgt * v[sidx].z; acc.w += wgt * v[sidx].w;
+                        }
+                    }
+                    const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, r);
+                    const float inv = 1.f / l;
+                    uint2 o;
+                    o.x = pack_bf16(acc.x * inv, acc.y * inv);
+                    o.y = pack_bf16(acc.z * inv, acc.w * inv);
+                    *reinterpret_cast<uint2*>(dst.o + g4 * 4) = o;
+                    if (dst.lse && g4 == 0) *dst.lse = (mx + log2f(l)) * 0.6931471805599453f;
+                }
+            }
+        }
+    }
+    if (tid == kAuxThreads) SS_TRC(5, 5);
+#ifdef SS_TRACE
+    if (tid == 0) atomicMax(&g_wall[s_launch & 7][1], wall_ns());
+    if (tid == 0) atomicMin(&g_wall[s_launch & 7][5], wall_ns());
+    if (tid == 0 && blk < kTraceCtas) g_trace[blk][0][152] = static_cast<long long>(wall_ns());
+#endif
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(G::kTmemCols) : "memory");
+    }
+}
+
+}  // namespace ss
