@@ -9,6 +9,11 @@
  *   ss_msa_attention   one layer of tree-masked multi-stream attention           (Eq. 1, Eq. 2)
  *   ss_tree_verify     greedy verification of the tree draft                     (Sec. 3.2.2, App. A.1)
  *   ss_kv_compact      lazy KV-cache backtracking of the accepted path           (App. A.1)
+ *   ss_next_draft      next tree draft from the stream logits of the last accepted node (Sec. 3.2.2, App. A.1)
+ *   ss_tree_prune      parallel tree pruning by early-exit transition probabilities  (Sec. 3.2.3)
+ *   ss_tree_verify_soft / ss_tree_verify_sampled   soft matching, top-k sampling at T = 1  (App. A.2, App. B)
+ *   ss_stream_insert   stream initialisation S = M + P_j                            (Eq. 3)
+ *   ss_value_rotate    value-rotation stream variant                                (Eq. 7)
  *   ss_status          read back the device status word
  *
  * Conventions
@@ -40,6 +45,7 @@ extern "C" {
 #define SS_MAX_NODES 64      /* tree nodes per sequence (one 64-bit ancestor word per node) */
 #define SS_MAX_GAMMA 4       /* speculative streams per node */
 #define SS_PATH_STRIDE SS_MAX_NODES /* entries per sequence in accept_path */
+#define SS_MAX_TOPK 8        /* tokens taken per stream / per node by the top-k entry points */
 
 enum {
     SS_OK = 0,
@@ -185,6 +191,85 @@ int32_t ss_tree_verify_static(const float* logits, const int32_t* draft_tokens, 
                               int32_t batch, int32_t max_nodes, int32_t vocab, int32_t* accept_len,
                               int32_t* accept_path, int32_t* last_node, int32_t* bonus_token,
                               int32_t* node_argmax, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Order of logits used by every arg-max / top-k below and by ss_tree_verify: IEEE fp32 order with
+ * -0 == +0, equal values by ascending index; a NaN ranks below every comparable value (inputs are
+ * meant to be finite; a row without any comparable value reports index 0 first). */
+
+/* Next tree draft (Sec. 3.2.2 "Parallel speculation and verification", App. A.1).  The correction token
+ * is the root; the top_k best tokens of stream g's logits are the children of every node of level g - 1,
+ * so that tokens drawn from stream n are the predecessors of those drawn from stream n + 1.  Nodes are
+ * numbered level by level, the children of a node in rank order (parent[i] < i); the full tree has
+ * 1 + sum_{g=1..gamma} top_k^g nodes (Sec. 3.2.3) and is cut after max_nodes nodes in that order.
+ *   stream_logits float [batch][n_rows][gamma][vocab]   logits of the speculative streams
+ *   row_index     int32 [batch] or NULL   which of the n_rows of each sequence to use: the last accepted
+ *                                         node written by a verification call (NULL: row 0)
+ *   bonus_token   int32 [batch]           the correction token (root of the new draft)
+ *   draft_tokens  int32 [batch][max_nodes]  out: tokens of the new tree, -1 past its nodes
+ *   trees         [batch]                 out: descriptors of the new trees, as ss_tree_build would give
+ * All pointers are device pointers: a decode loop needs no host round trip between the verification of one
+ * draft and the attention over the next.  Errors: SS_ERR_INVALID_ARG, SS_ERR_UNSUPPORTED (gamma >
+ * SS_MAX_GAMMA, top_k > SS_MAX_TOPK or > vocab, max_nodes > SS_MAX_NODES), SS_ERR_WORKSPACE, SS_ERR_CUDA. */
+size_t ss_next_draft_workspace_bytes(int32_t batch, int32_t gamma, int32_t vocab);
+int32_t ss_next_draft(const float* stream_logits, int32_t n_rows, const int32_t* row_index, const int32_t* bonus_token,
+                      int32_t batch, int32_t gamma, int32_t vocab, int32_t top_k, int32_t max_nodes,
+                      int32_t* draft_tokens, ss_tree_desc* trees, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Parallel tree pruning (Sec. 3.2.3; pruning paragraph and figure of App. A.1).  The transition probability
+ * of the edge parent -> child is the early-exit probability of the child's token at the parent,
+ * softmax(exit_logits[parent])[draft_tokens[child]]; an edge below `threshold` drops the child's whole
+ * sub-tree; the survivors keep their order and are re-indexed.  The root always survives.  The cache of
+ * the layers below is not touched (backtracking is lazy: ss_kv_compact gathers by original node index, so
+ * map a path of the pruned tree through kept_nodes first).
+ *   exit_logits  float [batch][max_nodes][vocab]   early-exit logits of every node (the caller's H(o(M^l)))
+ *   edge_prob    float [batch][max_nodes]  out: transition probability of each node's edge (root: 1)
+ *   new_index    int32 [batch][max_nodes]  out: index in the pruned tree, -1 if dropped
+ *   kept_nodes   int32 [batch][max_nodes]  out: original index of each surviving node, -1 past them
+ *   kept_tokens  int32 [batch][max_nodes]  out: their draft tokens
+ *   pruned_trees [batch]                   out: descriptors of the pruned trees
+ * Probabilities are computed in fp32 (log-sum-exp of the row); a transition within rounding of the
+ * threshold may fall on either side. */
+size_t ss_tree_prune_workspace_bytes(int32_t batch, int32_t max_nodes, int32_t vocab);
+int32_t ss_tree_prune(const float* exit_logits, const int32_t* draft_tokens, const ss_tree_desc* trees, int32_t batch,
+                      int32_t max_nodes, int32_t vocab, float threshold, float* edge_prob, int32_t* new_index,
+                      int32_t* kept_nodes, int32_t* kept_tokens, ss_tree_desc* pruned_trees, void* workspace,
+                      size_t workspace_bytes, void* stream);
+
+/* Verification with "soft" matching (App. A.2 names it as the relaxation of the hard criterion; the rule is
+ * the typical acceptance of the work it cites): a draft token is accepted when the main stream gives it a
+ * probability of at least min(eps, delta * exp(-H)), H the entropy of the main stream's distribution at the
+ * parent.  Outputs as ss_tree_verify (bonus_token is the arg-max at the last accepted node), plus
+ * edge_prob and node_entropy (float [batch][max_nodes], node_entropy may be NULL).  Workspace:
+ * ss_tree_prune_workspace_bytes. */
+int32_t ss_tree_verify_soft(const float* logits, const int32_t* draft_tokens, const ss_tree_desc* trees, int32_t batch,
+                            int32_t max_nodes, int32_t vocab, float eps, float delta, int32_t* accept_len,
+                            int32_t* accept_path, int32_t* last_node, int32_t* bonus_token, float* edge_prob,
+                            float* node_entropy, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Verification under top-k sampling at temperature 1 (App. B "Top-k Sampling"): the main stream's token at
+ * node t is drawn from the softmax over its top_k largest logits by inversion with uniforms[b][t] in [0, 1)
+ * (the first rank whose cumulative probability exceeds it); a draft token is accepted when it equals the
+ * token drawn at its parent; bonus_token is the token drawn at the last accepted node.  The caller owns
+ * the random numbers.  node_token int32 [batch][max_nodes] (may be NULL) receives the drawn tokens. */
+size_t ss_tree_verify_sampled_workspace_bytes(int32_t batch, int32_t max_nodes, int32_t vocab);
+int32_t ss_tree_verify_sampled(const float* logits, const int32_t* draft_tokens, const ss_tree_desc* trees,
+                               const float* uniforms, int32_t batch, int32_t max_nodes, int32_t vocab, int32_t top_k,
+                               int32_t* accept_len, int32_t* accept_path, int32_t* last_node, int32_t* bonus_token,
+                               int32_t* node_token, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Stream insertion (Eq. 3) with the identity for the transformation f, as in all of the paper's experiments
+ * (App. A.2): S_tj = M_t + P_j.  bf16 in and out, one fp32 addition per element.
+ *   main_hidden [rows][hidden], stream_emb [gamma][hidden], out [rows][gamma][hidden]; hidden % 8 == 0. */
+int32_t ss_stream_insert(const void* main_hidden, const void* stream_emb, void* out, int64_t rows, int32_t gamma,
+                         int32_t hidden, void* stream);
+
+/* Value rotation (App. B, Eq. 7): V_tn = V_t e^{i epsilon n}, n = 1..gamma.  Consecutive pairs of a value
+ * vector are the real and imaginary part of a complex number; stream n's value is the main stream's rotated
+ * by the angle epsilon * n (cos and sin evaluated on the host in double, used as fp32).
+ *   v_main [rows][width] bf16, v_streams [rows][gamma][width] bf16; width % 8 == 0. */
+int32_t ss_value_rotate(const void* v_main, void* v_streams, int64_t rows, int32_t gamma, int32_t width, float epsilon,
+                        void* stream);
 
 /* Cache layout shared by all layers: layer l, slot s, head h, element c of K sits at
  * k_cache_all + l*layer_stride + s*slot_stride + h*head_stride + c (strides in elements). */

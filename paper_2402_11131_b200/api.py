@@ -32,7 +32,9 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libss_msa.
 _lib = None
 
 # number of kernels each entry point enqueues per call (for launch accounting in the benchmark)
-LAUNCHES_PER_CALL = {"ss_msa_attention": 1, "ss_tree_verify": 1, "ss_kv_compact": 2}
+LAUNCHES_PER_CALL = {"ss_msa_attention": 1, "ss_tree_verify": 1, "ss_kv_compact": 2, "ss_next_draft": 1,
+                     "ss_tree_prune": 1, "ss_tree_verify_soft": 1, "ss_tree_verify_sampled": 1, "ss_stream_insert": 1,
+                     "ss_value_rotate": 1}
 
 
 class SsError(RuntimeError):
@@ -66,7 +68,11 @@ class CacheLayout(C.Structure):
 
 EXPORTS = ("ss_tree_build", "ss_msa_attention_workspace_bytes", "ss_msa_attention",
            "ss_tree_verify_workspace_bytes", "ss_tree_verify", "ss_tree_verify_static", "ss_kv_compact", "ss_status",
-           "ss_version", "ss_error_string")
+           "ss_version", "ss_error_string",
+           "ss_next_draft_workspace_bytes", "ss_next_draft", "ss_tree_prune_workspace_bytes", "ss_tree_prune",
+           "ss_tree_verify_soft", "ss_tree_verify_sampled_workspace_bytes", "ss_tree_verify_sampled",
+           "ss_stream_insert", "ss_value_rotate")
+SS_MAX_TOPK = 8
 SS_VERIFY_STATIC_SCRATCH_BYTES = 1 << 20
 
 
@@ -96,6 +102,22 @@ def lib() -> C.CDLL:
         l.ss_kv_compact.restype = C.c_int32
         l.ss_kv_compact.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(CacheLayout), C.c_int32, C.c_void_p,
                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        vp, i32, f32 = C.c_void_p, C.c_int32, C.c_float
+        for name in ("ss_next_draft_workspace_bytes", "ss_tree_prune_workspace_bytes", "ss_tree_verify_sampled_workspace_bytes"):
+            getattr(l, name).restype = C.c_size_t
+            getattr(l, name).argtypes = [i32, i32, i32]
+        l.ss_next_draft.restype = i32
+        l.ss_next_draft.argtypes = [vp, i32, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, C.c_size_t, vp]
+        l.ss_tree_prune.restype = i32
+        l.ss_tree_prune.argtypes = [vp, vp, vp, i32, i32, i32, f32, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        l.ss_tree_verify_soft.restype = i32
+        l.ss_tree_verify_soft.argtypes = [vp, vp, vp, i32, i32, i32, f32, f32, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        l.ss_tree_verify_sampled.restype = i32
+        l.ss_tree_verify_sampled.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        l.ss_stream_insert.restype = i32
+        l.ss_stream_insert.argtypes = [vp, vp, vp, C.c_int64, i32, i32, vp]
+        l.ss_value_rotate.restype = i32
+        l.ss_value_rotate.argtypes = [vp, vp, C.c_int64, i32, i32, f32, vp]
         l.ss_status.restype = C.c_int32
         l.ss_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
         l.ss_version.restype = C.c_int32
@@ -199,6 +221,89 @@ def ss_tree_verify_static(logits, draft_tokens, trees, accept_len, accept_path, 
     _check(lib().ss_tree_verify_static(_ptr(logits), _ptr(draft_tokens), _ptr(trees), B, Tmax, V,
                                        _ptr(accept_len), _ptr(accept_path), _ptr(last_node), _ptr(bonus_token),
                                        _ptr(node_argmax), _stream(stream)), "ss_tree_verify_static")
+
+
+def _ws_bytes(t: torch.Tensor) -> int:
+    return t.numel() * t.element_size()
+
+
+def empty_trees(batch: int, device="cuda") -> torch.Tensor:
+    """Device storage for `batch` tree descriptors (written by ss_next_draft / ss_tree_prune)."""
+    return torch.zeros(batch * C.sizeof(TreeDesc), dtype=torch.uint8, device=device)
+
+
+def trees_from_device(trees: torch.Tensor):
+    """Descriptors back on the host (tests)."""
+    raw = trees.cpu().numpy().tobytes()
+    n = len(raw) // C.sizeof(TreeDesc)
+    return [TreeDesc.from_buffer_copy(raw[i * C.sizeof(TreeDesc):(i + 1) * C.sizeof(TreeDesc)]) for i in range(n)]
+
+
+def ss_next_draft_workspace_bytes(batch: int, gamma: int, vocab: int) -> int:
+    return int(lib().ss_next_draft_workspace_bytes(batch, gamma, vocab))
+
+
+def ss_next_draft(stream_logits, row_index, bonus_token, top_k: int, max_nodes: int, draft_tokens, trees, workspace,
+                  stream=None) -> None:
+    """Next tree draft.  stream_logits f32 [B][n_rows][gamma][V]; row_index int32 [B] or None; bonus_token int32 [B];
+    draft_tokens int32 [B][max_nodes] and trees (empty_trees(B)) are written on the device."""
+    B, n_rows, gamma, V = stream_logits.shape
+    _check(lib().ss_next_draft(_ptr(stream_logits), n_rows, _ptr(row_index), _ptr(bonus_token), B, gamma, V, int(top_k),
+                               int(max_nodes), _ptr(draft_tokens), _ptr(trees), _ptr(workspace), _ws_bytes(workspace),
+                               _stream(stream)), "ss_next_draft")
+
+
+def ss_tree_prune_workspace_bytes(batch: int, max_nodes: int, vocab: int) -> int:
+    return int(lib().ss_tree_prune_workspace_bytes(batch, max_nodes, vocab))
+
+
+def ss_tree_prune(exit_logits, draft_tokens, trees, threshold: float, edge_prob, new_index, kept_nodes, kept_tokens,
+                  pruned_trees, workspace, stream=None) -> None:
+    """Parallel tree pruning.  exit_logits f32 [B][Tmax][V]; outputs are written on the device."""
+    B, Tmax, V = exit_logits.shape
+    _check(lib().ss_tree_prune(_ptr(exit_logits), _ptr(draft_tokens), _ptr(trees), B, Tmax, V, float(threshold),
+                               _ptr(edge_prob), _ptr(new_index), _ptr(kept_nodes), _ptr(kept_tokens), _ptr(pruned_trees),
+                               _ptr(workspace), _ws_bytes(workspace), _stream(stream)), "ss_tree_prune")
+
+
+def ss_tree_verify_soft(logits, draft_tokens, trees, eps: float, delta: float, accept_len, accept_path, last_node,
+                        bonus_token, edge_prob, node_entropy, workspace, stream=None) -> None:
+    """Verification with the soft (typical-acceptance) criterion; workspace of ss_tree_prune_workspace_bytes."""
+    B, Tmax, V = logits.shape
+    _check(lib().ss_tree_verify_soft(_ptr(logits), _ptr(draft_tokens), _ptr(trees), B, Tmax, V, float(eps), float(delta),
+                                     _ptr(accept_len), _ptr(accept_path), _ptr(last_node), _ptr(bonus_token),
+                                     _ptr(edge_prob), _ptr(node_entropy), _ptr(workspace), _ws_bytes(workspace),
+                                     _stream(stream)), "ss_tree_verify_soft")
+
+
+def ss_tree_verify_sampled_workspace_bytes(batch: int, max_nodes: int, vocab: int) -> int:
+    return int(lib().ss_tree_verify_sampled_workspace_bytes(batch, max_nodes, vocab))
+
+
+def ss_tree_verify_sampled(logits, draft_tokens, trees, uniforms, top_k: int, accept_len, accept_path, last_node,
+                           bonus_token, node_token, workspace, stream=None) -> None:
+    """Verification against tokens drawn from the top-k softmax (temperature 1) with the caller's uniforms f32 [B][Tmax]."""
+    B, Tmax, V = logits.shape
+    _check(lib().ss_tree_verify_sampled(_ptr(logits), _ptr(draft_tokens), _ptr(trees), _ptr(uniforms), B, Tmax, V,
+                                        int(top_k), _ptr(accept_len), _ptr(accept_path), _ptr(last_node),
+                                        _ptr(bonus_token), _ptr(node_token), _ptr(workspace), _ws_bytes(workspace),
+                                        _stream(stream)), "ss_tree_verify_sampled")
+
+
+def ss_stream_insert(main_hidden, stream_emb, out, stream=None) -> None:
+    """out[t][j] = main_hidden[t] + stream_emb[j] (Eq. 3, identity transformation); bf16 [rows][hidden], [gamma][hidden]."""
+    rows, hidden = main_hidden.shape
+    gamma = stream_emb.shape[0]
+    _check(lib().ss_stream_insert(_ptr(main_hidden), _ptr(stream_emb), _ptr(out), rows, gamma, hidden, _stream(stream)),
+           "ss_stream_insert")
+
+
+def ss_value_rotate(v_main, v_streams, epsilon: float, stream=None) -> None:
+    """v_streams[t][n-1] = v_main[t] rotated by epsilon * n on (re, im) pairs (Eq. 7); bf16 [rows][width], [rows][gamma][width]."""
+    rows, width = v_main.shape
+    gamma = v_streams.shape[1]
+    _check(lib().ss_value_rotate(_ptr(v_main), _ptr(v_streams), rows, gamma, width, float(epsilon), _stream(stream)),
+           "ss_value_rotate")
 
 
 def make_cache_layout(k_all: torch.Tensor) -> CacheLayout:

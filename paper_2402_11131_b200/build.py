@@ -15,7 +15,10 @@ LIB = os.path.join(PKG, "libss_msa_trace.so" if TRACE else "libss_msa.so")
 OBJ = os.path.join(PKG, "_build_trace" if TRACE else "_build")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xcompiler", "-fPIC", "--use_fast_math", "-I", os.path.join(ROOT, "include"), "-I", CSRC] + (["-DSS_TRACE"] if TRACE else [])
+              "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC] + (["-DSS_TRACE"] if TRACE else [])
+# Only the attention kernels are built with fast-math (ex2.approx, flush to zero).  Everything whose result is
+# defined bit by bit (comparisons of logits, byte copies, single fp32 operations) keeps IEEE arithmetic.
+FAST_MATH = {"ss_attention.cu"}
 
 
 def nvcc() -> str:
@@ -45,7 +48,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
         if force or _stale(obj, [src, *headers]):
-            cmd = [nvcc(), *NVCC_FLAGS, "-c", src, "-o", obj]
+            cmd = [nvcc(), *NVCC_FLAGS, *(["--use_fast_math"] if os.path.basename(src) in FAST_MATH else []), "-c", src, "-o", obj]
             if verbose:
                 cmd.insert(1, "-Xptxas=-v")
             procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
