@@ -75,10 +75,11 @@ static int grid_for(long long items) {
 
 extern "C" int32_t ss_stream_insert(const void* main_hidden, const void* stream_emb, void* out, int64_t rows, int32_t gamma,
                                     int32_t hidden, void* stream) {
-    if (!main_hidden || !stream_emb || !out || rows < 0 || gamma < 1 || hidden < 8) return SS_ERR_INVALID_ARG;
+    if (rows < 0 || gamma < 1 || hidden < 8) return SS_ERR_INVALID_ARG;
     if (gamma > SS_MAX_GAMMA || (hidden & 7)) return SS_ERR_UNSUPPORTED;
+    if (rows == 0) return SS_OK;                                   // nothing to do: the buffers may be empty
+    if (!main_hidden || !stream_emb || !out) return SS_ERR_INVALID_ARG;
     if (!ss::aligned16(main_hidden) || !ss::aligned16(stream_emb) || !ss::aligned16(out)) return SS_ERR_INVALID_ARG;
-    if (rows == 0) return SS_OK;
     const int vec = hidden / 8;
     const cudaError_t err = ss::launch_after_previous(ss::stream_insert_kernel, dim3(ss::grid_for(rows * gamma * vec)), dim3(256),
                                                       static_cast<cudaStream_t>(stream), static_cast<const uint4*>(main_hidden),
@@ -89,10 +90,11 @@ extern "C" int32_t ss_stream_insert(const void* main_hidden, const void* stream_
 
 extern "C" int32_t ss_value_rotate(const void* v_main, void* v_streams, int64_t rows, int32_t gamma, int32_t width, float epsilon,
                                    void* stream) {
-    if (!v_main || !v_streams || rows < 0 || gamma < 1 || width < 8 || !(epsilon == epsilon)) return SS_ERR_INVALID_ARG;
+    if (rows < 0 || gamma < 1 || width < 8 || !(epsilon == epsilon)) return SS_ERR_INVALID_ARG;
     if (gamma > SS_MAX_GAMMA || (width & 7)) return SS_ERR_UNSUPPORTED;
+    if (rows == 0) return SS_OK;                                   // nothing to do: the buffers may be empty
+    if (!v_main || !v_streams) return SS_ERR_INVALID_ARG;
     if (!ss::aligned16(v_main) || !ss::aligned16(v_streams)) return SS_ERR_INVALID_ARG;
-    if (rows == 0) return SS_OK;
     ss::RotTable tab = {};
     for (int n = 0; n < gamma; ++n) {
         const double ang = static_cast<double>(epsilon) * (n + 1);
