@@ -125,12 +125,16 @@ def oracle_sample(st, heads_per_layer: int = 2):
     s0, cap = int(st.kv_start[0]), int(st.kv_capacity[0])
     nbytes = 0
     t0 = time.perf_counter()
+    layer_seconds = []
     for ly in inputs:
         gg = g if ly.is_msa else 0
+        t_ly = time.perf_counter()
         oracle.msa_attention(st.parent[0], L, gg, st.sm_scale, ly.q_main[0], ly.k_cache[s0:s0 + cap],
                              ly.v_cache[s0:s0 + cap], None if gg == 0 else ly.q_spec[0],
                              None if gg == 0 else ly.k_spec[0], None if gg == 0 else ly.v_spec[0], heads=(0, hp))
         nbytes += (4 * L * d + 4 * T * d + 4 * T * gg * d + 4 * T * (1 + gg) * d) * hp
+        layer_seconds.append((ly.is_msa, time.perf_counter() - t_ly))
+    oracle_sample.layer_seconds = layer_seconds
     r = oracle.tree_verify(lg[0], st.draft_tokens[0], st.parent[0], path_cap=64)
     nbytes += 4 * T * c.vocab
     k4 = np.stack([inputs[-1].k_cache[s0:s0 + cap]] * 4)
@@ -140,6 +144,46 @@ def oracle_sample(st, heads_per_layer: int = 2):
     desc = ("sequence 0: %d of %d heads of %d attention layer(s) (one plain, one multi-stream), full verification, "
             "compaction over 4 layers" % (hp, H, len(inputs)))
     return nbytes, dt, desc, oracle.max_threads()
+
+
+def cpu_model() -> str:
+    try:
+        with open("/proc/cpuinfo") as fh:
+            for ln in fh:
+                if ln.startswith("model name"):
+                    return ln.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
+def cpu_baseline(st):
+    """The oracle, as it stands, on a bounded sample of the workload: once with every core the process may use
+    and once with one thread.  The sampled heads are independent and equal in cost, so the time of a whole step
+    (every head of every layer) is the sampled layers' time scaled by the head and layer counts."""
+    import oracle
+    c = st.cfg
+    n_all = oracle.max_threads()
+    b, t_all, desc, thr = oracle_sample(st)
+    layer_secs = list(oracle_sample.layer_seconds)
+    oracle.set_threads(1)
+    try:
+        _, t_one, _, _ = oracle_sample(st, heads_per_layer=1)
+    finally:
+        oracle.set_threads(n_all)
+    # extrapolation of the all-core run: one plain and one multi-stream layer were timed on `hp` heads each
+    hp = min(2, c.n_heads)
+    scale_heads = c.n_heads / hp * c.batch
+    n_plain = c.n_layers - c.n_msa_layers
+    est_step_s = 0.0
+    for is_msa, sec in layer_secs:                          # every head of every sequence of every layer of that kind
+        est_step_s += sec * scale_heads * (c.n_msa_layers if is_msa else n_plain)
+    return {"value": b / t_all / 1e9, "unit": UNIT, "cores": thr, "kind": "oracle", "sample": desc, "seconds": t_all,
+            "one_thread": {"seconds": t_one, "sample_heads_per_layer": 1}, "cpu_model": cpu_model(),
+            "cores_available": len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else None,
+            "extrapolated_step_seconds": est_step_s,
+            "extrapolation": "attention only: each sampled layer's time x (heads x sequences / sampled heads) x layers of its kind "
+                             "(sequence 0's length stands for all sequences)"}
 
 
 def run_reference(args):
@@ -195,11 +239,26 @@ def main():
         dist.barrier()
     api.lib()
 
-    cfg = W.CONFIGS[args.workload]
+    names = list(W.CONFIGS) if args.workload == "all" else [args.workload]
+    for workload in names:
+        line = measure(args, workload, world, rank, local_rank)
+        if line is not None:
+            print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def measure(args, workload, world, rank, local_rank):
+    """One workload: builds its device state, times the step and its components, returns the JSON line (rank 0)."""
+    import torch
+    import torch.distributed as dist
+    from paper_2402_11131_b200 import api, replicas, workloads as W
+    from paper_2402_11131_b200.step import DeviceStep
+    cfg = W.CONFIGS[workload]
     st = W.make_step(cfg)
     if args.profile:
         run_profile(args, st)
-        return
+        return None
     distinct = 2 if cfg.batch > 1 else None       # the ragged batch reuses two host-generated slabs
     dev = DeviceStep(st, distinct_slabs=distinct, pinned_host=not args.no_e2e)
     stream = torch.cuda.Stream()
@@ -288,9 +347,7 @@ def main():
         e2e = time_e2e(dev, stream, max(3, min(K, 50)), world)
 
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
+        return None
 
     peak, peak_src = measured_peaks()
     value = world * step_bytes / (step_ms * 1e-3) / 1e9
@@ -300,7 +357,7 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": args.workload, "batch": cfg.batch, "n_layers": cfg.n_layers,
+        "config": {"workload": workload, "batch": cfg.batch, "n_layers": cfg.n_layers,
                    "n_msa_layers": cfg.n_msa_layers, "n_heads": cfg.n_heads, "head_dim": cfg.head_dim,
                    "prefix_len": [int(x) for x in st.kv_len] if cfg.batch > 1 else int(st.kv_len[0]),
                    "tree_nodes": cfg.n_nodes, "gamma": cfg.gamma, "vocab": cfg.vocab,
@@ -319,20 +376,18 @@ def main():
         "attention_tflops": attn_flops / (attn_ms * 1e-3) / 1e12,
         "gpu_launches": launches_per_step * K,
         "clocks": clocks,
-        "roofline": {"kernel": "msa_attention_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
+        "pct_of_measured_peak": value / world / peak * 100,
+        "roofline": {"kernel": "msa_attention_small_kernel (plain layers) / msa_attention_kernel (multi-stream layers)", "bound": "hbm", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
                      "bytes_per_launch": attn_bytes / nl, "us_per_launch": attn_launch_us,
                      "timed": "CUDA events around replays of a graph of the step's %d attention launches, right after the timed region" % nl,
-                     "traffic": ncu_traffic() if args.workload == "7b" else None},
+                     "traffic": ncu_traffic() if workload == "7b" else None},
         "e2e": e2e,
     }
     if not args.no_cpu_baseline and world == 1:
-        b, t, desc, thr = oracle_sample(st)
-        line["cpu_baseline"] = {"value": b / t / 1e9, "unit": UNIT, "cores": thr, "kind": "oracle", "sample": desc,
-                                "seconds": t}
-    print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+        line["cpu_baseline"] = cpu_baseline(st)
+    return line
+
 
 
 def run_profile(args, st):

@@ -108,7 +108,14 @@ int32_t ss_tree_build(const int32_t* parent, int32_t n_nodes, int32_t gamma, ss_
  * query rows) and the partial rows of blocks whose keys are split over several CTAs
  * (ss_msa_attention_workspace_bytes).  Calls of different shapes may share one workspace as long as they
  * are ordered on one stream and it is large enough for each: a call leaves every counter at a multiple
- * of 4096.
+ * of 4096.  Word 1 of the workspace, if positive, shortens the bound of the device-side waits to that many
+ * units of 1024 cycles (default: about one second) for calls whose heads have at most 64 query rows; the
+ * library reads it and never writes it.
+ * Precondition of a split (batch * n_heads * row blocks below the SM count): the CTAs that share a block's
+ * keys wait for one another at the end, so they must all be resident at once.  The call sizes the split from
+ * the device's SM count; if other work holds SMs for the whole duration of the call (another stream, another
+ * process, a partition of the GPU) the wait can run out: the CTAs then give up, the status word reads
+ * SS_ERR_DEVICE_TIMEOUT and the outputs of the blocks concerned are not written.
  * Reads no K/V row past slot kv_start[b]+L_b+T_b-1 whose value can reach an output (a tile may touch
  * later slots of the slab; what it finds there is masked or cleared); writes only o_*, lse_* and the
  * workspace.
@@ -121,8 +128,12 @@ int32_t ss_tree_build(const int32_t* parent, int32_t n_nodes, int32_t gamma, ss_
  * kv_capacity or the tree descriptors.  The call is launched so that it can be scheduled while the
  * previous kernel of the stream drains (programmatic dependent launch); with the promise it reads the
  * lengths and starts streaming the prefix during that time.  Queries, the tree nodes' K/V, the stream K/V
- * and every output keep plain stream order either way.  A decode step satisfies the promise naturally:
- * the kernels before a layer's attention write this step's queries and tree-node K/V, never the prefix. */
+ * and every output keep plain stream order either way.  Inside a decode step the promise holds naturally:
+ * the kernels before a layer's attention write this step's queries and tree-node K/V, never the prefix.
+ * It does NOT hold for a call that directly follows ss_kv_compact on the same cache when that call writes
+ * the kv_len array the attention reads (kv_len_out == kv_len) or when the attention's lengths already
+ * include the compacted slots: compaction turns tree slots into prefix and writes the lengths.  Pass
+ * flags = 0 to the first attention call after such a compaction, or put any other kernel between them. */
 #define SS_ATTN_PREFIX_STABLE 1u
 
 typedef struct ss_attn_params {
