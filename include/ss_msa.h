@@ -15,6 +15,7 @@
  *   ss_stream_insert   stream initialisation S = M + P_j                            (Eq. 3)
  *   ss_value_rotate    value-rotation stream variant                                (Eq. 7)
  *   ss_status          read back the device status word
+ *   ss_wait_selftest   diagnostic: a device-side wait that runs out reports SS_ERR_DEVICE_TIMEOUT
  *
  * Conventions
  *   - Every call returns an int32 status: SS_OK or a negative SS_ERR_* code.  No exceptions.
@@ -29,7 +30,7 @@
  *     it ready for the next.  Word 0 of a workspace is the device status word: a kernel that
  *     detects a broken invariant (sequence over capacity, a wait that ran out) stores its
  *     SS_ERR_* code there and returns instead of faulting.  After SS_ERR_DEVICE_TIMEOUT the
- *     workspace's arrival counters are undefined: zero-fill it again before reuse.
+ *     workspace's contents are undefined: zero-fill it again before reuse.
  *   - Two calls that share a workspace must not overlap on the device.
  */
 #ifndef SS_MSA_H_
@@ -104,15 +105,16 @@ int32_t ss_tree_build(const int32_t* parent, int32_t n_nodes, int32_t gamma, ss_
  *   lse_main float[batch][max_nodes][n_heads], lse_spec float[batch][max_nodes][gamma][n_heads]:
  *                                  optional natural-log sum-exp of the scaled scores (NULL to skip).
  * Scores are sm_scale * <q, k>; softmax statistics and both products accumulate in fp32.
- * The workspace holds, besides the status word, one arrival counter per (sequence, head, block of 128
- * query rows) and the partial rows of blocks whose keys are split over several CTAs
- * (ss_msa_attention_workspace_bytes).  Calls of different shapes may share one workspace as long as they
- * are ordered on one stream and it is large enough for each: a call leaves every counter at a multiple
- * of 4096.  Word 1 of the workspace, if positive, shortens the bound of the device-side waits to that many
- * units of 1024 cycles (default: about one second) for calls whose heads have at most 64 query rows; the
- * library reads it and never writes it.
+ * The workspace holds, after its 256-byte header, the partial rows (fp32 O, m, l per query row) of blocks
+ * of 128 query rows whose keys are split over several CTAs (ss_msa_attention_workspace_bytes).  The rows are
+ * their own arrival flags: between calls that area is all zero, a partial row is never stored with a +0
+ * word (-0 is stored instead), a CTA waits for the words it combines to read non-zero and stores zeros over
+ * them afterwards.  So calls of different shapes may share one workspace as long as they are ordered on one
+ * stream and it is large enough for each.  Word 1 of the workspace, if positive, shortens the bound of the
+ * device-side waits to that many units of 1024 cycles (default: about one second) for calls whose heads
+ * have at most 64 query rows and for ss_wait_selftest; the library reads it and never writes it.
  * Precondition of a split (batch * n_heads * row blocks below the SM count): the CTAs that share a block's
- * keys wait for one another at the end, so they must all be resident at once.  The call sizes the split from
+ * keys wait for one another's partial rows at the end, so they must all be resident at once.  The call sizes the split from
  * the device's SM count; if other work holds SMs for the whole duration of the call (another stream, another
  * process, a partition of the GPU) the wait can run out: the CTAs then give up, the status word reads
  * SS_ERR_DEVICE_TIMEOUT and the outputs of the blocks concerned are not written.
@@ -298,6 +300,15 @@ typedef struct ss_cache_layout {
 int32_t ss_kv_compact(void* k_cache_all, void* v_cache_all, const ss_cache_layout* layout, int32_t batch,
                       const int64_t* kv_start, const int32_t* kv_len_in, const int32_t* accept_len,
                       const int32_t* accept_path, int32_t* kv_len_out, void* stream);
+
+/* Diagnostic of the bounded device-side waits.  Runs, as one warp, the step in which a CTA of a head split
+ * two ways combines its share of the partial rows (the routine ss_msa_attention's kernels use), with no
+ * second CTA launched: the row it waits for cannot arrive, the wait runs out after its bound (workspace
+ * word 1, as for ss_msa_attention) and the kernel stores SS_ERR_DEVICE_TIMEOUT in the status word and
+ * returns.  Nothing faults or hangs; the stream stays usable.  `workspace`: device, zero-filled (apart from
+ * word 1), at least 64 KiB; it is left as found.  Errors (nothing launched): SS_ERR_INVALID_ARG,
+ * SS_ERR_WORKSPACE, SS_ERR_CUDA. */
+int32_t ss_wait_selftest(void* workspace, size_t workspace_bytes, void* stream);
 
 /* Synchronises `stream`, copies the status word of `workspace` to *device_status_out (host) and
  * clears it.  Returns SS_ERR_CUDA if the stream reports an error. */

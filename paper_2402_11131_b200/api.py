@@ -71,7 +71,7 @@ EXPORTS = ("ss_tree_build", "ss_msa_attention_workspace_bytes", "ss_msa_attentio
            "ss_version", "ss_error_string",
            "ss_next_draft_workspace_bytes", "ss_next_draft", "ss_tree_prune_workspace_bytes", "ss_tree_prune",
            "ss_tree_verify_soft", "ss_tree_verify_sampled_workspace_bytes", "ss_tree_verify_sampled",
-           "ss_stream_insert", "ss_value_rotate")
+           "ss_stream_insert", "ss_value_rotate", "ss_wait_selftest")
 SS_MAX_TOPK = 8
 SS_VERIFY_STATIC_SCRATCH_BYTES = 1 << 20
 
@@ -118,6 +118,8 @@ def lib() -> C.CDLL:
         l.ss_stream_insert.argtypes = [vp, vp, vp, C.c_int64, i32, i32, vp]
         l.ss_value_rotate.restype = i32
         l.ss_value_rotate.argtypes = [vp, vp, C.c_int64, i32, i32, f32, vp]
+        l.ss_wait_selftest.restype = C.c_int32
+        l.ss_wait_selftest.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p]
         l.ss_status.restype = C.c_int32
         l.ss_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
         l.ss_version.restype = C.c_int32
@@ -322,6 +324,12 @@ def ss_kv_compact(k_all, v_all, layout: CacheLayout, kv_start, kv_len_in, accept
     _check(lib().ss_kv_compact(_ptr(k_all), _ptr(v_all), C.byref(layout), kv_start.shape[0], _ptr(kv_start),
                                _ptr(kv_len_in), _ptr(accept_len), _ptr(accept_path), _ptr(kv_len_out),
                                _stream(stream)), "ss_kv_compact")
+
+
+def ss_wait_selftest(workspace: torch.Tensor, stream=None) -> None:
+    """Diagnostic: one warp waits (bounded by workspace word 1) for a partial row that cannot arrive."""
+    _check(lib().ss_wait_selftest(_ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+           "ss_wait_selftest")
 
 
 def ss_status(workspace: torch.Tensor, stream=None) -> int:

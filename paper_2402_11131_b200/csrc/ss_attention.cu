@@ -30,9 +30,9 @@
 //
 // Split-KV merge.  Each CTA ends with un-normalised (m, l, O) per row, combines what it holds for a
 // row locally, and -- when the keys were split -- leaves one partial row in the workspace (it stays in
-// L2): every thread stores its pieces and arrives on the block's counter with release semantics.  One
-// thread waits, bounded, for the other CTAs of the block (launched with it, needing nothing from it);
-// each CTA then combines its own share of the rows, read straight from L2, and writes bf16 output.
+// L2).  The rows are their own arrival flags (the area is zero between calls and +0 is never stored):
+// each CTA polls, bounded, the rows of its own share from all CTAs of the block (launched with it,
+// needing nothing from it), combines them, writes bf16 output and stores zeros over what it read.
 //
 // Launch.  Programmatic dependent launch: one thread of each CTA waits for the previous kernel of
 // the stream; before that wait the kernel touches global memory only under the caller's
@@ -50,6 +50,8 @@ namespace ss {
 #ifdef SS_TRACE
 constexpr int kTraceCtas = 16, kTraceRoles = 6, kTraceSlots = 160;
 __device__ long long g_trace[kTraceCtas][kTraceRoles][kTraceSlots];
+__device__ int g_trace_base;
+__device__ unsigned long long g_cta_wall[8][256][4];   // per launch and CTA: start, wait released, end (globaltimer ns), SM id
 __device__ unsigned long long g_wall[8][6];      // first CTA start / last CTA end (globaltimer ns) of the last 8 launches
 __device__ unsigned long long g_key[8];           // launch identity: the output pointer
 __device__ __forceinline__ unsigned long long wall_ns() {
@@ -73,7 +75,6 @@ constexpr int kAuxThreads = 128;     // warps 0..3: producers and MMA issuers
 constexpr int kMaxDynSmem = 232448 - 1024;  // 227 KB per CTA less the static control block
 constexpr float kRescaleStep = 8.f;  // raise the running maximum only when it grows by more than 2^8
 constexpr long long kWaitCycles = 2000000000ll;   // bound of every mbarrier wait (~1 s)
-constexpr unsigned int kArrivalsPerCall = 4096u;  // what the CTAs of a split block add to its arrival counter in one call
 
 struct alignas(64) AttnArgs {
     CUtensorMap tm_k, tm_v;          // cache slab    dims (d, H, slots)        box (64, 1, 128)
@@ -100,7 +101,6 @@ struct alignas(64) AttnArgs {
     const int* kv_capacity;
     const ss_tree_desc* trees;
     int* status;
-    int* counters;                   // [groups] arrivals of a block's CTAs (monotonic)
     float* partials;                 // [groups][splits][rows][head_dim + 4]
 };
 
@@ -502,6 +502,148 @@ __device__ __forceinline__ OutPtr out_ptr(const AttnArgs& a, int b, int h, long 
         p.lse = a.lse_spec ? a.lse_spec + idx : nullptr;
     }
     return p;
+}
+
+// ---- combining the partial rows of the CTAs that share a block's keys ---------------------------
+// A partial row is HD floats of O, then m, l and two floats of padding, relative to the row's reference m
+// (in log2 units).  Between calls the workspace's partial-row area is all zero, and a value is never stored
+// there as +0 (the writer stores -0 instead): a word that reads non-zero has arrived.  So the rows need no
+// flag, no counter and no fence: a reader polls the words it needs (bounded), combines them, and stores zeros
+// over what it has read, which leaves the area as the next call expects it.  Rows that no node owns are
+// neither written nor read.
+__device__ __forceinline__ uint32_t never_plus_zero(uint32_t bits) { return bits == 0u ? 0x80000000u : bits; }
+#ifndef SS_ST_KIND
+#define SS_ST_KIND "st.relaxed.gpu.global"
+#endif
+__device__ __forceinline__ void st_relaxed_v4(float* p, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
+    asm volatile(SS_ST_KIND ".v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+__device__ __forceinline__ void st_relaxed_v2(float* p, uint32_t x, uint32_t y) {
+    asm volatile(SS_ST_KIND ".v2.b32 [%0], {%1, %2};" ::"l"(p), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ uint4 ld_relaxed_v4(const float* p) {
+    uint4 v;
+    asm volatile("ld.relaxed.gpu.global.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint2 ld_relaxed_v2(const float* p) {
+    uint2 v;
+    asm volatile("ld.relaxed.gpu.global.v2.b32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p) : "memory");
+    return v;
+}
+
+// Step 1: the staged rows (shared memory at y_base, `rows` rows of HD + 4 floats) go to this CTA's rows in the
+// workspace, a warp per row (whole lines), except the rows of this CTA's own share [first, first + share), which
+// it combines straight from shared memory.
+template <int HD>
+__device__ __forceinline__ void publish_partial_rows(const Span& sp, int row0, int rows, uint32_t y_base, float* part_mine, int first, int share,
+                                                     int t, int threads) {
+    constexpr uint32_t kRowBytes = (HD + 4) * 4;
+    const int lane = t & 31;
+    for (int rr = t >> 5; rr < rows; rr += threads >> 5) {                               // warp-uniform
+        if ((rr >= first && rr < first + share) || !row_info(sp, row0 + rr).valid) continue;
+        float* dst = part_mine + static_cast<size_t>(rr) * (HD + 4);
+        if (lane < HD / 4) {
+            const float4 v = ld_shared_v4(y_base + static_cast<uint32_t>(rr) * kRowBytes + static_cast<uint32_t>(lane) * 16u);
+            st_relaxed_v4(dst + lane * 4, never_plus_zero(__float_as_uint(v.x)), never_plus_zero(__float_as_uint(v.y)),
+                          never_plus_zero(__float_as_uint(v.z)), never_plus_zero(__float_as_uint(v.w)));
+        }
+        if (lane == 0) {
+            const float2 ml = ld_shared_v2(y_base + static_cast<uint32_t>(rr) * kRowBytes + HD * 4u);
+            st_relaxed_v2(dst + HD, never_plus_zero(__float_as_uint(ml.x)), never_plus_zero(__float_as_uint(ml.y)));
+        }
+    }
+}
+
+// Step 2: this CTA's share of the block's rows, rows [first, first + share): its own partial from shared memory,
+// the others' from the workspace (part_group, one CTA's rows `cta_stride` floats after the previous one's).  A
+// row's items (four columns each) lie in one warp, so that one lane can clear the row's (m, l) once every lane
+// of the warp has read it.  Returns false when the wait ran out (limit in cycles) or another thread of the CTA
+// had given up.
+template <int HD>
+__device__ __forceinline__ bool merge_partial_rows(const AttnArgs& a, const Span& sp, int row0, int b, int h, long long spec_row0, int C, int rank,
+                                                   uint32_t y_base, const float* part_group, size_t cta_stride, int first, int share, int t,
+                                                   int threads, long long limit, volatile int* abort_flag) {
+    constexpr int kItems = HD / 4;                                   // items of a row
+    constexpr int kLanes = kItems <= 16 ? 16 : 32;                   // lanes a row takes in a warp
+    constexpr int kRowsPerWarp = 32 / kLanes;
+    constexpr int kPitch = HD + 4;
+    const int lane = t & 31, warp_t = t >> 5, n_warps = threads >> 5;
+    const int sub = lane / kLanes, g4 = lane - sub * kLanes;
+    bool good = true;
+    for (int rbase = warp_t * kRowsPerWarp; rbase < share; rbase += n_warps * kRowsPerWarp) {     // warp-uniform
+        const int rr = rbase + sub;
+        const RowInfo r = row_info(sp, row0 + first + (rr < share ? rr : 0));
+        const bool mine = rr < share && g4 < kItems && r.valid;
+        float* src = const_cast<float*>(part_group) + static_cast<size_t>(first + (mine ? rr : 0)) * kPitch;
+        uint4 v[8];
+        uint2 ml[8];
+        uint32_t pending = mine ? ((1u << C) - 1u) & ~(1u << rank) : 0u;
+        if (mine) {
+            const uint32_t own = y_base + static_cast<uint32_t>(first + rr) * (kPitch * 4u);
+            const float4 ov = ld_shared_v4(own + static_cast<uint32_t>(g4) * 16u);
+            const float2 oml = ld_shared_v2(own + HD * 4u);
+            #pragma unroll
+            for (int sidx = 0; sidx < 8; ++sidx) {
+                if (sidx == rank) {
+                    v[sidx] = make_uint4(__float_as_uint(ov.x), __float_as_uint(ov.y), __float_as_uint(ov.z), __float_as_uint(ov.w));
+                    ml[sidx] = make_uint2(__float_as_uint(oml.x), __float_as_uint(oml.y));
+                }
+            }
+        }
+        const long long t0 = clock64();
+        for (;;) {
+            #pragma unroll
+            for (int sidx = 0; sidx < 8; ++sidx) {
+                if ((pending >> sidx) & 1u) {
+                    v[sidx] = ld_relaxed_v4(src + sidx * cta_stride + g4 * 4);
+                    ml[sidx] = ld_relaxed_v2(src + sidx * cta_stride + HD);
+                }
+            }
+            #pragma unroll
+            for (int sidx = 0; sidx < 8; ++sidx)
+                if (((pending >> sidx) & 1u) && v[sidx].x != 0u && v[sidx].y != 0u && v[sidx].z != 0u && v[sidx].w != 0u && ml[sidx].x != 0u &&
+                    ml[sidx].y != 0u)
+                    pending &= ~(1u << sidx);
+            if (!__any_sync(0xffffffffu, pending != 0u)) break;
+            if (__any_sync(0xffffffffu, *abort_flag != 0 || clock64() - t0 > limit)) { good = false; break; }
+        }
+        if (!good) break;
+        if (mine) {
+            float mx = -INFINITY;
+            #pragma unroll
+            for (int sidx = 0; sidx < 8; ++sidx)
+                if (sidx < C) mx = fmaxf(mx, __uint_as_float(ml[sidx].x));
+            float l = 0.f;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            #pragma unroll
+            for (int sidx = 0; sidx < 8; ++sidx) {
+                if (sidx < C) {
+                    const float ms = __uint_as_float(ml[sidx].x);
+                    const float wgt = ms == -INFINITY ? 0.f : exp2f(ms - mx);       // 0: saw no visible key
+                    l += wgt * __uint_as_float(ml[sidx].y);
+                    acc.x += wgt * __uint_as_float(v[sidx].x); acc.y += wgt * __uint_as_float(v[sidx].y);
+                    acc.z += wgt * __uint_as_float(v[sidx].z); acc.w += wgt * __uint_as_float(v[sidx].w);
+                }
+            }
+            const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, r);
+            const float inv = 1.f / l;
+            uint2 o;
+            o.x = pack_bf16(acc.x * inv, acc.y * inv);
+            o.y = pack_bf16(acc.z * inv, acc.w * inv);
+            *reinterpret_cast<uint2*>(dst.o + g4 * 4) = o;
+            if (dst.lse && g4 == 0) *dst.lse = (mx + log2f(l)) * 0.6931471805599453f;
+            // what was read goes back to zero: every lane its own columns, one lane the row's (m, l)
+            #pragma unroll
+            for (int sidx = 0; sidx < 8; ++sidx) {
+                if (sidx < C && sidx != rank) {
+                    st_relaxed_v4(src + sidx * cta_stride + g4 * 4, 0u, 0u, 0u, 0u);
+                    if (g4 == 0) st_relaxed_v2(src + sidx * cta_stride + HD, 0u, 0u);
+                }
+            }
+        }
+    }
+    return good;
 }
 
 // 16 fp32 values scaled and packed to bf16 -> 32 bytes at dst
@@ -990,8 +1132,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     // ======================================== epilogue ==========================================
     // The softmax warpgroups combine the partials a row has inside the CTA.  Not split (C == 1): that
     // is the result.  Split: every CTA leaves one un-normalised partial row (O, m, l) per query row in
-    // the workspace (it stays in L2), arrives on the block's counter, waits for the others and combines
-    // its own share of the rows.
+    // the workspace (it stays in L2) and combines its own share of the rows as they arrive from all CTAs.
     const bool has_acc = (warp >= 4) && n_own > 0;     // otherwise the partial is (m = -inf, l = 0, O = 0)
     const uint32_t o_addr = tmem + lane_base + (warp >= 4 ? wg : 0) * G::kOCols;
     constexpr int RP = G::kMergePitch;                                         // floats per partial row: O, m, l, pad
@@ -1108,81 +1249,18 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     }
 
     if (C > 1 && warp >= 4) {
-        // Publication.  The partial rows wait in Y; every thread copies its 16-byte pieces to the workspace
-        // (whole lines, they stay in L2) and then arrives on the block's counter with release semantics, which
-        // orders its own pieces before its arrival: no barrier, fence or returned value lies between the rows
-        // and their publication.  A call adds 4096 to the counter in total (each of the 256 threads of each of
-        // the C CTAs 16 / C), so between calls it is a multiple of 4096 whatever split factor earlier calls on the
-        // workspace had, and after this CTA's own arrivals it is one again exactly when all C CTAs have arrived.
-        // One thread then waits (bounded) for that: the other CTAs were launched together with this one and need
-        // nothing from it, so the wait is short.
+        // The partial rows wait in Y.  The other CTAs of the block were launched with this one and need nothing
+        // from it, so the (bounded) wait for their rows is short.
         named_barrier(3, wg_threads);                                 // Y is complete
         const int t = tid - kAuxThreads;
-        unsigned int* cnt = reinterpret_cast<unsigned int*>(a.counters) + group;
-        {
-            constexpr int kPieces = rows_cap * static_cast<int>(RB / 16);
-            float4* dstp = reinterpret_cast<float4*>(part_mine);
-            #pragma unroll 4
-            for (int i = t; i < kPieces; i += wg_threads) __stcg(dstp + i, ld_shared_v4(y_base + static_cast<uint32_t>(i) * 16u));
-            asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(cnt), "r"(16u >> a.cluster_shift) : "memory");
-        }
-        if (tid == kAuxThreads) {
-            bool ok = true;
-            const long long t0 = clock64();
-            for (;;) {
-                unsigned int now;       // this thread's own arrival precedes the load (same address, program order)
-                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(now) : "l"(cnt) : "memory");
-                if ((now & (kArrivalsPerCall - 1u)) == 0u) break;
-                if (*abort_flag || clock64() - t0 > kWaitCycles) { ok = false; break; }
-            }
-            if (!ok) { c.abort = 1; set_status(a.status, SS_ERR_DEVICE_TIMEOUT); }
-            c.merge_ok = ok ? 1 : 0;
-        }
-        named_barrier(3, wg_threads);
+        const bool live = __all_sync(0xffffffffu, !skip && *abort_flag == 0);
+        const int share = rows_cap >> a.cluster_shift, first = static_cast<int>(rank) * share;
+        if (live) publish_partial_rows<HD>(sp, sp.row0, rows_cap, y_base, part_mine, first, share, t, wg_threads);
         if (tid == kAuxThreads) SS_TR(5, 4);
-        if (c.merge_ok && !skip) {
-            // This CTA's share: rows [first, first + share) of the block's partial rows, read straight from L2
-            // (past L1, which may hold lines of an earlier call).  Work item: (row, group of four columns); a
-            // thread has the loads of all C sources of its item in flight at once.
-            const int share = rows_cap >> a.cluster_shift;
-            const int first = static_cast<int>(rank) * share;
-            const size_t cta_stride = static_cast<size_t>(rows_cap) * RP;
-            for (int w = t; w < share * (HD / 4); w += wg_threads) {
-                const int rr = w / (HD / 4), g = w - rr * (HD / 4);
-                const RowInfo r = row_info(sp, sp.row0 + first + rr);
-                if (!r.valid) continue;
-                const float* src = part_group + static_cast<size_t>(first + rr) * RP;
-                float4 v[8];
-                float2 ml[8];
-                #pragma unroll
-                for (int sidx = 0; sidx < 8; ++sidx) {
-                    if (sidx < C) {
-                        v[sidx] = __ldcg(reinterpret_cast<const float4*>(src + sidx * cta_stride + g * 4));
-                        ml[sidx] = __ldcg(reinterpret_cast<const float2*>(src + sidx * cta_stride + HD));
-                    }
-                }
-                float mx = -INFINITY;
-                #pragma unroll
-                for (int sidx = 0; sidx < 8; ++sidx)
-                    if (sidx < C) mx = fmaxf(mx, ml[sidx].x);
-                float l = 0.f;
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                #pragma unroll
-                for (int sidx = 0; sidx < 8; ++sidx) {
-                    if (sidx < C) {
-                        const float wgt = ml[sidx].x == -INFINITY ? 0.f : exp2f(ml[sidx].x - mx);   // 0: saw no visible key
-                        l += wgt * ml[sidx].y;
-                        acc.x += wgt * v[sidx].x; acc.y += wgt * v[sidx].y; acc.z += wgt * v[sidx].z; acc.w += wgt * v[sidx].w;
-                    }
-                }
-                const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, r);
-                const float inv = 1.f / l;
-                uint2 o;
-                o.x = pack_bf16(acc.x * inv, acc.y * inv);
-                o.y = pack_bf16(acc.z * inv, acc.w * inv);
-                *reinterpret_cast<uint2*>(dst.o + g * 4) = o;
-                if (dst.lse && g == 0) *dst.lse = (mx + log2f(l)) * 0.6931471805599453f;
-            }
+        if (live && !merge_partial_rows<HD>(a, sp, sp.row0, b, h, spec_row0, C, static_cast<int>(rank), y_base, part_group,
+                                            static_cast<size_t>(rows_cap) * RP, first, share, t, wg_threads, kWaitCycles, abort_flag)) {
+            c.abort = 1;
+            set_status(a.status, SS_ERR_DEVICE_TIMEOUT);
         }
     }
     if (tid == kAuxThreads) SS_TR(5, 5);
@@ -1246,7 +1324,7 @@ struct AttnPlan {
     int tmax8, spec_rows, s0rows, n_blocks, mode, n_kslots, n_vslots, cluster;
     long long groups;                          // (sequence, head, row block) triples
     size_t smem;
-    size_t counter_bytes, partial_bytes;       // workspace after its header
+    size_t partial_bytes;                      // workspace after its header
 };
 
 static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
@@ -1267,15 +1345,15 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     while (c < 8 && plan->groups * (c * 2) <= sm_count()) c *= 2;
     plan->cluster = c;
     if (plan->mode == kCols) {
-        // the query tile on its way to TMEM, then one ring of K/V tiles (at the end it stages 64 partial rows)
-        const size_t q_bytes = static_cast<size_t>(halves) * kSmRows * 128, slot = static_cast<size_t>(halves) * kTileKeys * 128;
+        // the query tile (its 64 rows twice), then the K and V rings (at the end they stage 64 partial rows)
+        const size_t q_bytes = static_cast<size_t>(halves) * 2 * kSmRows * 128, slot = static_cast<size_t>(halves) * kTileKeys * 128;
         int slots = static_cast<int>((kSmDynSmem - q_bytes) / slot);
         if (slots > kSmMaxSlots) slots = kSmMaxSlots;
-        if (slots < 3) return false;
+        slots &= ~1;                                          // a K ring and a V ring of the same depth
+        if (slots < 4) return false;
         plan->n_kslots = slots;
         plan->n_vslots = 0;
         plan->smem = q_bytes + static_cast<size_t>(slots) * slot;
-        plan->counter_bytes = (static_cast<size_t>(plan->groups) * sizeof(int32_t) + 255) / 256 * 256;
         // a split head leaves the partial rows (O, m, l) of each of its CTAs in the workspace
         plan->partial_bytes = c > 1 ? static_cast<size_t>(plan->groups) * c * kSmRows * (p.head_dim + 4) * 4 : 0;
         return true;
@@ -1297,9 +1375,8 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     const size_t stage = 2048 + (plan->mode == kDual ? 2 * 64 : kBlockRows) * row_bytes;
     if (stage > bytes) bytes = stage;
     plan->smem = bytes + 1024;
-    // workspace: one arrival counter per group; one partial row per (group, CTA of the group, row)
+    // workspace: one partial row per (group, CTA of the group, row)
     const size_t rows_cap = plan->mode == kDual ? 64 : kBlockRows;
-    plan->counter_bytes = (static_cast<size_t>(plan->groups) * sizeof(int32_t) + 255) / 256 * 256;
     plan->partial_bytes = c > 1 ? static_cast<size_t>(plan->groups) * c * rows_cap * row_bytes : 0;
     return plan->smem <= static_cast<size_t>(kMaxDynSmem);
 }
@@ -1362,7 +1439,7 @@ static int32_t launch_cols(const AttnArgs& args, const AttnPlan& plan, cudaStrea
 extern "C" size_t ss_msa_attention_workspace_bytes(const ss_attn_params* p) {
     ss::AttnPlan plan;
     if (p == nullptr || !ss::make_plan(*p, &plan)) return 0;
-    return ss::kWsHeaderBytes + plan.counter_bytes + plan.partial_bytes;
+    return ss::kWsHeaderBytes + plan.partial_bytes;
 }
 
 extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
@@ -1425,8 +1502,7 @@ extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
     a.kv_start = reinterpret_cast<const long long*>(p->kv_start);
     a.kv_len = p->kv_len; a.kv_capacity = p->kv_capacity; a.trees = p->trees;
     a.status = reinterpret_cast<int*>(p->workspace);
-    a.counters = reinterpret_cast<int*>(static_cast<char*>(p->workspace) + ss::kWsHeaderBytes);
-    a.partials = reinterpret_cast<float*>(static_cast<char*>(p->workspace) + ss::kWsHeaderBytes + plan.counter_bytes);
+    a.partials = reinterpret_cast<float*>(static_cast<char*>(p->workspace) + ss::kWsHeaderBytes);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (plan.mode == ss::kCols) {
         switch (d) {
@@ -1440,6 +1516,41 @@ extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
         case 80: return ss::launch<80, ss::kPair>(a, plan, s);
         default: return ss::launch<128, ss::kPair>(a, plan, s);
     }
+}
+
+namespace ss {
+// One warp runs the merge step of a head that is split two ways, as its CTA 0, for one row -- and no CTA 1 was
+// launched, so the row it waits for never arrives: the wait runs out after its bound and the status word
+// reports it.  Nothing else is read or written unless the area was not zero.
+__global__ void wait_selftest_kernel(const __grid_constant__ AttnArgs a) {
+    __shared__ __align__(16) float own_row[64 + 4];
+    __shared__ int abort_flag;
+    const int lane = threadIdx.x;
+    for (int i = lane; i < 64 + 4; i += 32) own_row[i] = 1.f;
+    if (lane == 0) abort_flag = 0;
+    __syncwarp();
+    int lim;
+    asm volatile("ld.global.cg.s32 %0, [%1];" : "=r"(lim) : "l"(a.status + 1) : "memory");
+    const long long limit = lim > 0 ? static_cast<long long>(lim) << 10 : kWaitCycles;
+    Span sp;
+    sp.L = 0; sp.T = 1; sp.gamma = 0; sp.tmax8 = 8; sp.n_stream = 0; sp.spec_end = 8;
+    if (!merge_partial_rows<64>(a, sp, 0, 0, 0, 0, 2, 0, smem_u32(own_row), a.partials, static_cast<size_t>(64) * (64 + 4), 0, 1, lane, 32, limit,
+                                &abort_flag))
+        set_status(a.status, SS_ERR_DEVICE_TIMEOUT);
+}
+}  // namespace ss
+
+extern "C" int32_t ss_wait_selftest(void* workspace, size_t workspace_bytes, void* stream) {
+    const size_t need = ss::kWsHeaderBytes + static_cast<size_t>(2) * 64 * (64 + 4) * 4 + 256;
+    if (workspace == nullptr) return SS_ERR_INVALID_ARG;
+    if (workspace_bytes < need) return SS_ERR_WORKSPACE;
+    ss::AttnArgs a{};
+    a.status = static_cast<int*>(workspace);
+    a.partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + ss::kWsHeaderBytes);
+    a.o_main = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + need - 256);      // never reached on a zero area
+    a.max_nodes = 1; a.n_heads = 1;
+    ss::wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(a);
+    return cudaGetLastError() == cudaSuccess ? SS_OK : SS_ERR_CUDA;
 }
 
 #ifdef SS_TRACE
@@ -1456,6 +1567,12 @@ extern "C" int32_t ss_trace_clear() {
     unsigned long long keys[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     if (cudaMemcpyToSymbol(ss::g_wall, wall, sizeof(wall)) != cudaSuccess) return -1;
     return cudaMemcpyToSymbol(ss::g_key, keys, sizeof(keys)) == cudaSuccess ? 0 : -1;
+}
+extern "C" int32_t ss_trace_cta_wall(unsigned long long* out) {
+    return cudaMemcpyFromSymbol(out, ss::g_cta_wall, sizeof(ss::g_cta_wall)) == cudaSuccess ? 0 : -1;
+}
+extern "C" int32_t ss_trace_base(int base) {
+    return cudaMemcpyToSymbol(ss::g_trace_base, &base, sizeof(int)) == cudaSuccess ? 0 : -1;
 }
 extern "C" int32_t ss_trace_wall(unsigned long long* out) {
     return cudaMemcpyFromSymbol(out, ss::g_wall, sizeof(ss::g_wall)) == cudaSuccess ? 0 : -1;

@@ -1,20 +1,18 @@
 // Tree-masked multi-stream attention for heads of at most 64 query rows (Eq. 1, Eq. 2).  Included by
 // ss_attention.cu after its helpers.
 //
-// What bounds a tile of 128 keys on one SM is shared-memory bandwidth (128 B per cycle): the 64 KB of the K and
-// V tile are written once by TMA and must be read once by the two MMAs, which is about 1000 cycles -- as long
-// as nothing else goes through shared memory.  So both small operands live in TMEM and are the A operand of
-// their MMA (tcgen05.mma with A in TMEM), and only K and V are read from shared memory:
+// A tile of 128 keys costs an SM 64 KB of TMA writes into shared memory and at least 64 KB of MMA operand
+// reads out of it (128 B per cycle in total), so P never goes through shared memory: it is written to TMEM as
+// bf16 and is the A operand of its MMA (tcgen05.mma with A in TMEM).
 //
-//   S = Q K^T     A = the query tile in TMEM (written there once), B = a K tile (K-major), N = 128 keys
-//   O += P V      A = P in TMEM (bf16, written by the softmax threads over the scores they have just read),
-//                 B = the V tile (MN-major), N = head_dim
+//   S = Q K^T     A = the query tile in shared memory (K-major), B = a K tile (K-major), N = 128 keys
+//   O += P V      A = P in TMEM, B = the V tile (MN-major), N = head_dim
 //
-// The 64 rows fill half of the 128 TMEM lanes; the other half holds the rows a second time (copy 1).  The
-// copies take alternate tiles: copy c exponentiates tiles c, c + 2, .. into a P buffer of its own, in which the
-// other copy's lanes stay zero, so one tile's exponentials overlap the other tile's MMAs, and each copy
-// accumulates its own partial row, over its own tiles.  There is one score buffer: a copy moves its scores
-// to registers (four softmax threads share a lane, 32 scores each) and hands the buffer back at once.
+// The 64 rows fill half of the 128 rows of an MMA; the other half holds the rows a second time (copy 1).  The
+// copies take alternate tiles: copy c exponentiates tiles c, c + 2, .. from a score buffer of its own into a P
+// buffer of its own, in which the other copy's lanes stay zero, so one tile's exponentials overlap the other
+// tile's MMAs, and each copy accumulates its own partial row, over its own tiles.  A copy moves its scores to
+// registers (four softmax threads share a lane, 32 scores each) and hands the score buffer back at once.
 //
 // Softmax with a shared reference.  The four threads of a lane exponentiate against one reference m_ref (any
 // value at or above the lane's scores, and not absurdly far above, gives the same result after
@@ -27,8 +25,9 @@
 // softmax threads, four to a TMEM lane.
 //
 // End of a CTA.  Copy 1 hands its partial rows (O, m, l) to copy 0 through shared memory.  C = 1: copy 0
-// normalises and writes bf16.  Split heads (C > 1): the combined rows go to the workspace in whole lines, the
-// CTAs of the head meet on its arrival counter, and each combines its share of the rows from all C partials.
+// normalises and writes bf16.  Split heads (C > 1): the combined rows go to the workspace in whole lines, and
+// each CTA combines its share of the rows from all C partials as they arrive (publish_partial_rows,
+// merge_partial_rows).
 #pragma once
 
 namespace ss {
@@ -37,7 +36,7 @@ namespace ss {
 #ifdef SS_TRACE
 #define SS_TRC(role, slot)                                                                                       \
     do {                                                                                                         \
-        const int tr_cta_ = static_cast<int>(blockIdx.x);                                                        \
+        const int tr_cta_ = static_cast<int>(blockIdx.x) - ss::g_trace_base;                                                        \
         if (tr_cta_ >= 0 && tr_cta_ < ss::kTraceCtas && (slot) < ss::kTraceSlots) ss::g_trace[tr_cta_][role][slot] = clock64(); \
     } while (0)
 #else
@@ -48,38 +47,36 @@ constexpr int kSmRows = 64;                       // query rows of the variant
 constexpr int kSmThreads = 640;
 constexpr int kSmSoftmax = 512;                   // four threads per TMEM lane
 constexpr int kSmMaxSlots = 6;
-constexpr int kSmDynSmem = 216 * 1024;            // one CTA per SM
+constexpr int kSmDynSmem = 224 * 1024;            // one CTA per SM: with the 3 KB control block, all of its 227 KB
 
 template <int HD>
 struct GeoS {
     static constexpr int kHalves = HD > 64 ? 2 : 1;               // 64-element boxes along head_dim
     static constexpr int kBoxBytes = kTileKeys * 128;             // one TMA box: 128 keys x 128 B
     static constexpr int kSlotBytes = kHalves * kBoxBytes;        // a K tile or a V tile
-    static constexpr int kQHalfBytes = kSmRows * 128;
-    static constexpr int kQBytes = kHalves * kQHalfBytes;         // staging of the query tile on its way to TMEM
+    static constexpr int kQHalfBytes = 2 * kSmRows * 128;         // the 64 rows twice (copy 0, copy 1): M = 128
+    static constexpr int kQBytes = kHalves * kQHalfBytes;
     static constexpr int kKSteps = HD / 16;
     static constexpr int kCpt = HD / 4;                           // accumulator columns a thread finishes
-    static constexpr uint32_t kTmemCols = 512;                    // Q (64), O (128), two score buffers (128 each)
+    static constexpr uint32_t kTmemCols = 512;                    // O (128), two score buffers (128 each), two P buffers (64 each)
     static constexpr int kPitch = HD + 4;                         // floats of a partial row: O, m, l, pad
     static constexpr size_t kCtaFloats = static_cast<size_t>(kSmRows) * kPitch;         // workspace of one CTA of a split head
 };
 
 struct CtrlS {
-    unsigned long long q_full, q_ready;        // query tile in shared memory / in TMEM (16 warps)
-    // A slot's K fills and V fills complete on barriers of their own: each is awaited by one thread, which then
-    // sees every phase of its barrier (K and V tiles alternate in a slot when the ring has an odd number of
-    // slots, and a parity wait that is two phases behind would pass at once).
-    unsigned long long slot_full[2][kSmMaxSlots], slot_empty[kSmMaxSlots];
+    unsigned long long q_full, q_ready;        // query tile in shared memory / the P buffers' constant zeros in place (16 warps)
+    // K tiles and V tiles have rings of their own ([0] K, [1] V; tile j in slot j mod depth): a K slot is free
+    // again when S of its tile is complete, a V slot only when P V is, so K tiles run ahead of V tiles
+    unsigned long long slot_full[2][kSmMaxSlots / 2], slot_empty[2][kSmMaxSlots / 2];
     // by tile parity = copy that consumes the tile; each barrier is then looked at in every phase by its waiters
     unsigned long long s_full[2];              // S of a tile complete
-    unsigned long long s_free[2];              // its scores are in registers (the copy's 8 warps): the one score buffer is free
+    unsigned long long s_free[2];              // its scores are in registers (the copy's 8 warps): the copy's score buffer is free
     unsigned long long p_full[2];              // P of a tile written to the copy's P buffer (8 warps)
     unsigned long long pv_done[2];             // P V of a tile complete: the copy's P buffer is free
     unsigned long long anc[SS_MAX_NODES];
     alignas(16) float xch[4][2 * kSmRows];     // exchange between the four threads of a lane (maxima, row sums)
     uint32_t tmem_base;
     int abort;
-    int merge_ok;
     int wait_limit;                            // bound of every wait, in units of 1024 cycles
 };
 
@@ -132,27 +129,30 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
     const int group = blk >> a.cluster_shift;              // (sequence, head)
     int b = group / a.n_heads;
     const int h = group - b * a.n_heads;
-    const int n_slots = a.n_kslots;
+    const int n_ring = a.n_kslots >> 1;                    // depth of the K ring and of the V ring
     if (tid == 0) SS_TRC(0, 0);
 #ifdef SS_TRACE
     __shared__ unsigned int s_launch;
     if (tid == 0) {
         const unsigned long long key = reinterpret_cast<unsigned long long>(a.o_main);
-        s_launch = 0;
-        for (unsigned int i = 0; i < 8; ++i) {
+        unsigned int found = 8;
+        for (unsigned int i = 0; i < 8 && found == 8; ++i)
+            if (*reinterpret_cast<volatile unsigned long long*>(&g_key[i]) == key) found = i;
+        for (unsigned int i = 0; i < 8 && found == 8; ++i) {
             const unsigned long long old = atomicCAS(&g_key[i], 0ull, key);
-            if (old == 0ull || old == key) { s_launch = i; break; }
+            if (old == 0ull || old == key) found = i;
         }
-        atomicMin(&g_wall[s_launch & 7][0], wall_ns());
-        atomicMax(&g_wall[s_launch & 7][2], wall_ns());
-        if (blk < kTraceCtas) g_trace[blk][0][150] = static_cast<long long>(wall_ns());
+        s_launch = found & 7;
+        unsigned int smid;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        if (blk < 256) { g_cta_wall[s_launch][blk][0] = wall_ns(); g_cta_wall[s_launch][blk][3] = smid; }
     }
 #endif
 
     const uint32_t base = smem_u32(smem_raw);              // 1024-byte aligned (checked below): swizzle atoms
     const uint32_t q_base = base;                          // [half][64 rows][128 B]: the query tile on its way to TMEM
-    const uint32_t ring_base = q_base + G::kQBytes;        // [slot][half][128 keys][128 B]
-    auto slot_addr = [&](int s) { return ring_base + static_cast<uint32_t>(s) * G::kSlotBytes; };
+    const uint32_t ring_base = q_base + G::kQBytes;        // [slot][K, V][half][128 keys][128 B]
+    auto slot_addr = [&](int kind, int s) { return ring_base + static_cast<uint32_t>(2 * s + kind) * G::kSlotBytes; };
 
     // ---- prologue (see msa_attention_kernel: the same launch protocol) ------------------------------
     int L = 0, T = 0, cap = 0x7fffffff;
@@ -177,7 +177,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
     if (a.prefix_stable) load_scalars();
     if (tid == 0) {
         mbar_init(smem_u32(&c.q_full), 1);
-        for (int s = 0; s < kSmMaxSlots; ++s) { mbar_init(smem_u32(&c.slot_full[0][s]), 1); mbar_init(smem_u32(&c.slot_full[1][s]), 1); }
+        for (int s = 0; s < kSmMaxSlots / 2; ++s) { mbar_init(smem_u32(&c.slot_full[0][s]), 1); mbar_init(smem_u32(&c.slot_full[1][s]), 1); }
         c.abort = 0;
         c.wait_limit = static_cast<int>(kWaitCycles >> 10);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -185,7 +185,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
         if (a.gamma > 0) { tma_prefetch_desc(&a.tm_qs); tma_prefetch_desc(&a.tm_ks); tma_prefetch_desc(&a.tm_vs); }
     } else if (tid == 64) {
         mbar_init(smem_u32(&c.q_ready), 16);
-        for (int s = 0; s < kSmMaxSlots; ++s) mbar_init(smem_u32(&c.slot_empty[s]), 1);
+        for (int s = 0; s < kSmMaxSlots / 2; ++s) { mbar_init(smem_u32(&c.slot_empty[0][s]), 1); mbar_init(smem_u32(&c.slot_empty[1][s]), 1); }
         for (int s = 0; s < 2; ++s) {
             mbar_init(smem_u32(&c.s_full[s]), 1);
             mbar_init(smem_u32(&c.s_free[s]), 8);
@@ -200,9 +200,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
             asm volatile("griddepcontrol.wait;" ::: "memory");
             SS_TRC(0, 3);
 #ifdef SS_TRACE
-            atomicMin(&g_wall[s_launch & 7][3], wall_ns());
-            atomicMax(&g_wall[s_launch & 7][4], wall_ns());
-            if (blk < kTraceCtas) g_trace[blk][0][151] = static_cast<long long>(wall_ns());
+            if (blk < 256) g_cta_wall[s_launch][blk][1] = wall_ns();
 #endif
             asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
         }
@@ -227,13 +225,12 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
     // whole tiles are dealt out, the first CTAs of a head taking the odd ones: the last CTA has the masked tiles
     const Span sp = make_span(a, L, T, static_cast<int>(rank), 0, kTileKeys, true);
 
-    // ring entry i: K tile i/2 (even) or V tile i/2 (odd)
-    auto load_entry = [&](int i, int st) {
-        const int j = i >> 1;
-        const bool is_v = (i & 1) != 0;
-        const uint32_t bar = smem_u32(&c.slot_full[i & 1][st]);
+    // the K tile (kind 0) or the V tile (kind 1) of the CTA's tile j into slot st of its ring
+    auto load_tile = [&](int kind, int j, int st) {
+        const bool is_v = kind != 0;
+        const uint32_t bar = smem_u32(&c.slot_full[kind][st]);
         mbar_expect_tx(bar, G::kSlotBytes);
-        const uint32_t dst = slot_addr(st);
+        const uint32_t dst = slot_addr(kind, st);
         const int x = sp.first_key(j);
         #pragma unroll
         for (int hh = 0; hh < G::kHalves; ++hh) {
@@ -241,17 +238,16 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
             else tma_load_3d(dst + hh * G::kBoxBytes, is_v ? &a.tm_vs : &a.tm_ks, hh * 64, h, static_cast<int>(spec_row0 + x), bar);
         }
     };
-    const int n_entries = 2 * sp.n_tiles;
-    // Two tiles are requested right away (before the dependency wait, under the caller's promise); the rest of
-    // the ring follows once the query rows have arrived, which would otherwise queue behind the tiles on their
-    // way into this SM
-    const int n_early = min(n_entries, min(n_slots, 4));
+    // The first two tiles are requested right away, K0 V0 K1 V1 (before the dependency wait, under the caller's
+    // promise); the rest follows once the query rows have arrived, which would otherwise queue behind the
+    // tiles on their way into this SM
+    const int n_early = min(sp.n_tiles, min(n_ring, 2));
     auto prefix_only = [&](int j) { return sp.is_cache(j) && sp.first_key(j) + TK <= sp.L; };
     int n_pre = 0;
     if (a.prefix_stable) {
         if (tid == 0) {
             // the first tiles that lie wholly inside the cached prefix
-            while (n_pre < n_early && prefix_only(n_pre >> 1)) { load_entry(n_pre, n_pre); ++n_pre; }
+            while (n_pre < 2 * n_early && prefix_only(n_pre >> 1)) { load_tile(n_pre & 1, n_pre >> 1, n_pre >> 1); ++n_pre; }
         }
         dependency_wait();
     }
@@ -261,19 +257,18 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
         const uint32_t qbar = smem_u32(&c.q_full);
         const bool with_spec = a.gamma > 0 && a.s0rows > 0;
         const uint32_t rows = a.tmax8 + (with_spec ? a.s0rows : 0);
-        mbar_expect_tx(qbar, bad_smem ? 0u : G::kHalves * rows * 128u);
+        mbar_expect_tx(qbar, bad_smem ? 0u : 2u * G::kHalves * rows * 128u);
         #pragma unroll
         for (int hh = 0; hh < G::kHalves; ++hh) {
-            if (bad_smem) break;
-            const uint32_t dst = q_base + hh * G::kQHalfBytes;
-            tma_load_3d(dst, &a.tm_qm, hh * 64, h, b * a.max_nodes, qbar);
-            if (with_spec) tma_load_3d(dst + a.tmax8 * 128u, &a.tm_qs, hh * 64, h, static_cast<int>(spec_row0), qbar);
+            #pragma unroll
+            for (int cp = 0; cp < 2; ++cp) {
+                if (bad_smem) break;
+                const uint32_t dst = q_base + hh * G::kQHalfBytes + cp * (kSmRows * 128u);
+                tma_load_3d(dst, &a.tm_qm, hh * 64, h, b * a.max_nodes, qbar);
+                if (with_spec) tma_load_3d(dst + a.tmax8 * 128u, &a.tm_qs, hh * 64, h, static_cast<int>(spec_row0), qbar);
+            }
         }
-        for (int i = n_pre; i < n_early; ++i) load_entry(i, i);
-        // the caller may shorten the bound of the device-side waits (workspace word 1, units of 1024 cycles)
-        int lim;
-        asm volatile("ld.global.cg.s32 %0, [%1];" : "=r"(lim) : "l"(a.status + 1) : "memory");
-        if (lim > 0) c.wait_limit = lim;
+        for (int i = n_pre; i < 2 * n_early; ++i) load_tile(i & 1, i >> 1, i >> 1);
         SS_TRC(0, 5);
     }
     if (tid >= kAuxThreads && tid < kAuxThreads + SS_MAX_NODES) c.anc[tid - kAuxThreads] = __ldcg(&a.trees[b].anc_mask[tid - kAuxThreads]);
@@ -282,64 +277,76 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
     tc_fence_after();
     if (tid == 0) SS_TRC(0, 6);
     const uint32_t tmem = c.tmem_base;
-    const uint32_t tmem_q = tmem;                          // 64 columns: the query rows, two bf16 to a column
-    const uint32_t tmem_o = tmem + 64;                     // 128 columns
-    const uint32_t tmem_s = tmem + 192;                    // one score buffer of 128 columns
-    const uint32_t tmem_p = tmem + 320;                    // two P buffers of 64 columns (128 keys as bf16), one per copy
+    const uint32_t tmem_o = tmem;                          // 128 columns
+    const uint32_t tmem_s = tmem + 128;                    // two score buffers of 128 columns, one per copy
+    const uint32_t tmem_p = tmem + 384;                    // two P buffers of 64 columns (128 keys as bf16), one per copy
     int* const status = a.status;
-    // fill number of a slot's barrier of one kind: with an odd number of slots the kinds alternate in a slot
-    const bool odd_ring = (n_slots & 1) != 0;
-    auto fill_parity = [&](const Ring& r) { return static_cast<uint32_t>((odd_ring ? r.round >> 1 : r.round) & 1); };
-    auto wait_slot_full = [&](int kind, const Ring& r) {
-        return mbar_wait_s(smem_u32(&c.slot_full[kind][r.slot]), fill_parity(r), &c, status);
+    // tile j of a kind: slot j mod depth, filled for the (j / depth)-th time
+    auto wait_tile_full = [&](int kind, const Ring& r) {
+        return mbar_wait_s(smem_u32(&c.slot_full[kind][r.slot]), static_cast<uint32_t>(r.round & 1), &c, status);
+    };
+    // the tiles after the early ones, each as soon as its slot is free; a producer that gives up lets the
+    // copies already in flight land before the CTA leaves
+    auto produce = [&](int kind) {
+        Ring r;
+        r.start();
+        for (int j = 0; j < n_early; ++j) r.advance(n_ring);
+        bool ok = mbar_wait_s(smem_u32(&c.q_full), 0, &c, status);
+        int j = n_early;
+        for (; ok && j < sp.n_tiles; ++j) {
+            if (r.round > 0) ok = mbar_wait_s(smem_u32(&c.slot_empty[kind][r.slot]), (r.round - 1) & 1, &c, status);
+            if (kind == 0) SS_TRC(0, 8 + j);
+            if (ok) { load_tile(kind, j, r.slot); r.advance(n_ring); }
+        }
+        if (!ok) {
+            const int issued = r.slot + r.round * n_ring;
+            Ring d;
+            d.start();
+            for (int i = 0; i < issued; ++i, d.advance(n_ring))
+                if (i >= issued - n_ring) mbar_drain(smem_u32(&c.slot_full[kind][d.slot]), static_cast<uint32_t>(d.round & 1));
+        }
     };
 
-    // =============================== warp 0: tile requests =======================================
+    // =============================== warps 0 and 3: tile requests ================================
     if (warp == 0) {
-        if (lane == 0 && n_entries > n_early) {
-            Ring r;
-            r.start();
-            for (int i = 0; i < n_early; ++i) r.advance(n_slots);
-            bool ok = mbar_wait_s(smem_u32(&c.q_ready), 0, &c, status);
-            for (int i = n_early; ok && i < n_entries; ++i) {
-                if (r.round > 0) ok = mbar_wait_s(smem_u32(&c.slot_empty[r.slot]), (r.round - 1) & 1, &c, status);
-                SS_TRC(0, 8 + i);
-                if (ok) { load_entry(i, r.slot); r.advance(n_slots); }
-            }
-            if (!ok) {                 // gave up: let the copies already in flight land before the CTA leaves
-                const int issued = r.slot + r.round * n_slots;
-                Ring d;
-                d.start();
-                for (int i = 0; i < issued; ++i, d.advance(n_slots))
-                    if (i >= issued - n_slots) mbar_drain(smem_u32(&c.slot_full[i & 1][d.slot]), fill_parity(d));
-            }
+        if (lane == 0 && sp.n_tiles > n_early) produce(0);
+    } else if (warp == 3) {
+        if (lane == 0) {
+            // the caller may shorten the bound of the device-side waits (workspace word 1, units of 1024 cycles)
+            int lim;
+            asm volatile("ld.global.cg.s32 %0, [%1];" : "=r"(lim) : "l"(a.status + 1) : "memory");
+            if (lim > 0) *reinterpret_cast<volatile int*>(&c.wait_limit) = lim;
+            if (sp.n_tiles > n_early) produce(1);
         }
     }
     // =============================== warp 1: S = Q K^T, A from TMEM ================================
     else if (warp == 1) {
         if (lane == 0) {
-            bool ok = mbar_wait_s(smem_u32(&c.q_ready), 0, &c, status);
+            bool ok = mbar_wait_s(smem_u32(&c.q_full), 0, &c, status);
+            if (!ok) mbar_drain(smem_u32(&c.q_full), 0);
             SS_TRC(1, 0);
+            const uint64_t dq = desc_k_major(q_base);
             Ring r;
             r.start();
             for (int j = 0; ok && j < sp.n_tiles; ++j) {
                 const int buf = j & 1;
-                if (!wait_slot_full(0, r)) break;
+                if (!wait_tile_full(0, r)) break;
                 SS_TRC(1, 8 + 4 * j);
-                // the scores of the tile before must be in registers
-                if (j >= 1 && !mbar_wait_s(smem_u32(&c.s_free[buf ^ 1]), ((j - 1) >> 1) & 1, &c, status)) break;
+                // the copy's scores of its tile before must be in registers
+                if (j >= 2 && !mbar_wait_s(smem_u32(&c.s_free[buf]), ((j >> 1) - 1) & 1, &c, status)) break;
                 SS_TRC(1, 9 + 4 * j);
                 tc_fence_after();
-                const uint64_t dk = desc_k_major(slot_addr(r.slot));
+                const uint64_t dk = desc_k_major(slot_addr(0, r.slot));
                 #pragma unroll
                 for (int ks = 0; ks < G::kKSteps; ++ks) {
                     const uint32_t hh = ks >> 2, off = (ks & 3) * 32u;
-                    tc_mma_ts(tmem_s, tmem_q + ks * 8u, dk + ((hh * G::kBoxBytes + off) >> 4), idesc_bf16(TK, false, false), ks > 0);
+                    tc_mma(tmem_s + buf * TK, dq + ((hh * G::kQHalfBytes + off) >> 4), dk + ((hh * G::kBoxBytes + off) >> 4),
+                           idesc_bf16(TK, false, false), ks > 0);
                 }
                 tc_commit(smem_u32(&c.s_full[buf]));
-                tc_commit(smem_u32(&c.slot_empty[r.slot]));                   // K may go when S is complete
+                tc_commit(smem_u32(&c.slot_empty[0][r.slot]));                // K may go when S is complete
                 SS_TRC(1, 10 + 4 * j);
-                r.advance(n_slots); r.advance(n_slots);
+                r.advance(n_ring);
             }
         }
     }
@@ -348,16 +355,15 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
         if (lane == 0) {
             Ring rv;
             rv.start();
-            rv.advance(n_slots);
             bool okq = mbar_wait_s(smem_u32(&c.q_ready), 0, &c, status);     // the P buffers' constant zeros are in place
             for (int j = 0; okq && j < sp.n_tiles; ++j) {
                 const int buf = j & 1;
-                if (!wait_slot_full(1, rv)) break;
+                if (!wait_tile_full(1, rv)) break;
                 SS_TRC(2, 8 + 4 * j);
                 if (!mbar_wait_s(smem_u32(&c.p_full[buf]), (j >> 1) & 1, &c, status)) break;
                 SS_TRC(2, 9 + 4 * j);
                 tc_fence_after();
-                const uint64_t dv = desc_mn_major(slot_addr(rv.slot), G::kBoxBytes);
+                const uint64_t dv = desc_mn_major(slot_addr(1, rv.slot), G::kBoxBytes);
                 // P of the tile: the copy's buffer, keys 16 ks .. 16 ks + 15 in columns 8 ks .. 8 ks + 7 (zero in the
                 // other copy's lanes)
                 #pragma unroll
@@ -365,9 +371,9 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
                     tc_mma_ts(tmem_o, tmem_p + buf * 64u + 8u * ks, dv + ((ks * 2048u) >> 4), idesc_bf16(HD, false, true),
                               (j > 0 || ks > 0) ? 1u : 0u);
                 tc_commit(smem_u32(&c.pv_done[buf]));
-                tc_commit(smem_u32(&c.slot_empty[rv.slot]));
+                tc_commit(smem_u32(&c.slot_empty[1][rv.slot]));
                 SS_TRC(2, 10 + 4 * j);
-                rv.advance(n_slots); rv.advance(n_slots);
+                rv.advance(n_ring);
             }
         }
     }
@@ -382,26 +388,12 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
     if (warp >= 4) {
         ri = row_info(sp, row);
         const unsigned long long anc = ri.valid ? c.anc[ri.node] : 0ull;
-        // ---- the query row of this lane, from shared memory into TMEM: 32 of its elements per thread (two bf16
-        // to a column, as they lie in memory); a lane without a row holds zeros.  The lane's part of the other
-        // copy's P buffer is zero for the whole kernel.
+        // ---- the lane's part of the other copy's P buffer is zero for the whole kernel
         {
-            const bool have_q = mbar_wait_warp_s(smem_u32(&c.q_full), 0, &c, status);
-            uint32_t qv[16];
+            uint32_t zr[16];
             #pragma unroll
-            for (int i = 0; i < 16; ++i) qv[i] = 0u;
-            tmem_st16<0>(tmem_p + lane_base + static_cast<uint32_t>((1 - copy) * 64 + 16 * w4), qv);
-            const int hh = w4 >> 1;
-            if (have_q && ri.valid && hh < G::kHalves && !bad_smem) {
-                #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint32_t piece = static_cast<uint32_t>((w4 & 1) * 4 + i);
-                    const float4 f = ld_shared_v4(q_base + hh * G::kQHalfBytes + row * 128u + ((piece ^ (row & 7)) << 4));
-                    qv[4 * i + 0] = __float_as_uint(f.x); qv[4 * i + 1] = __float_as_uint(f.y);
-                    qv[4 * i + 2] = __float_as_uint(f.z); qv[4 * i + 3] = __float_as_uint(f.w);
-                }
-            }
-            tmem_st16<0>(tmem_q + lane_base + 16u * w4, qv);
+            for (int i = 0; i < 16; ++i) zr[i] = 0u;
+            tmem_st16<0>(tmem_p + lane_base + static_cast<uint32_t>((1 - copy) * 64 + 16 * w4), zr);
             tmem_wait_st();
             tc_fence_before();
             __syncwarp();
@@ -433,10 +425,10 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
                                         : 0xffffffffu;
             uint32_t sr[32];
             if (ok) {
-                tmem_ld32<0>(tmem_s + lane_base + 32u * w4, sr);
+                tmem_ld32<0>(tmem_s + lane_base + static_cast<uint32_t>(copy * TK) + 32u * w4, sr);
                 tmem_wait_ld();
             }
-            // the scores are in registers: S of the next tile (the other copy's) may overwrite the buffer
+            // the scores are in registers: S of the copy's next tile may overwrite the buffer
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&c.s_free[copy]));
@@ -475,13 +467,11 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
                         tmem_wait_st();
                     }
                 }
-                named_barrier(6 + copy, 256);                // the exchange buffer may be written again
+                // the copy's reducing barrier of this tile lies between these reads and the next raise's writes
                 return ok2;
             };
 
             if (j < 2) raise();                                               // every thread of the copy, so the barriers inside match
-            // P of this copy's previous tile must have been read before it is overwritten
-            if (j >= 2) ok = mbar_wait_warp_s(smem_u32(&c.pv_done[copy]), ((j - 2) >> 1) & 1, &c, status) && ok;
             bool leave = false;
             for (int attempt = 0; attempt < 3; ++attempt) {
                 float tmax = -INFINITY, lsum = 0.f;
@@ -501,7 +491,9 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
                         lsum += e0 + e1;
                         pk[i >> 1] = pack_bf16(e0, e1);
                     }
-                    tmem_st16<0>(p_addr, pk);
+                    // P of this copy's previous tile must have been read before it is overwritten
+                    if (attempt == 0 && j >= 2) ok = mbar_wait_warp_s(smem_u32(&c.pv_done[copy]), ((j - 2) >> 1) & 1, &c, status);
+                    if (ok) tmem_st16<0>(p_addr, pk);
                 }
                 if (leader) SS_TRC(3, 9 + 6 * j + (attempt > 0 ? 3 : 0));
                 // one reducing barrier per tile: did a score outgrow its reference, or did a wait run out
@@ -517,15 +509,13 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
             // but 0 * NaN is NaN, so they are cleared: a thread looks after rows (row, row + 64) of the tile
             const int region_left = (cache ? sp.L + sp.T : sp.n_stream) - x0;
             if (region_left < TK) {
-                Ring rv;
-                rv.start();
-                for (int i = 0; i < 2 * j + 1; ++i) rv.advance(n_slots);
-                if (mbar_wait_warp_s(smem_u32(&c.slot_full[1][rv.slot]), fill_parity(rv), &c, status)) {
+                const int vs = j % n_ring;
+                if (mbar_wait_warp_s(smem_u32(&c.slot_full[1][vs]), static_cast<uint32_t>((j / n_ring) & 1), &c, status)) {
                     #pragma unroll
                     for (int up = 0; up < 2; ++up) {
                         const int vr = row + 64 * up;
                         if (vr >= region_left && (w4 >> 1) < G::kHalves) {
-                            const uint32_t dst = slot_addr(rv.slot) + (w4 >> 1) * G::kBoxBytes + vr * 128u + (w4 & 1) * 64u;
+                            const uint32_t dst = slot_addr(1, vs) + (w4 >> 1) * G::kBoxBytes + vr * 128u + (w4 & 1) * 64u;
                             #pragma unroll
                             for (int i = 0; i < 4; ++i) st_shared_v4(dst + i * 16, 0u, 0u, 0u, 0u);
                         }
@@ -559,10 +549,8 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
     // A lane's partial over the keys of its copy: O in TMEM, the reference, and the sum of its four threads' row
     // sums.  Copy 1 hands its rows to copy 0 through shared memory (the ring is idle: every copy has landed and
     // every MMA is complete).  C = 1: copy 0 normalises and writes bf16.  Split head: the combined rows go back
-    // to shared memory and from there, in whole lines, to the workspace (they stay in L2); every thread's pieces
-    // precede its release arrival on the head's counter (a call adds 4096 to it in total), one thread waits
-    // (bounded) for the other CTAs of the head, which were launched with this one and need nothing from it, and
-    // each CTA combines its share of the rows.
+    // to shared memory and from there, in whole lines, to the workspace (they stay in L2), and each CTA combines
+    // its share of the rows as they arrive from the CTAs of the head.
     constexpr int CPT = G::kCpt;
     constexpr uint32_t YB = G::kPitch * 4;                                    // bytes of a staged row
     const uint32_t y_base = ring_base;                                        // [64 rows][kPitch floats]
@@ -590,6 +578,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
             if (w4 == 0) st_shared_v4(yrow + HD * 4u, __float_as_uint(m_ref), __float_as_uint(l_lane), 0u, 0u);
         }
         named_barrier(8, kSmSoftmax);
+        if (tid == kAuxThreads) SS_TRC(5, 8);
         float m_out = m_ref, l_out = l_lane;
         if (copy == 0) {
             const float2 z = ld_shared_v2(yrow + HD * 4u);
@@ -626,83 +615,22 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
         }
         if (C > 1) {
             named_barrier(8, kSmSoftmax);                                     // the staged rows are complete
+            if (tid == kAuxThreads) SS_TRC(5, 9);
             const int t = tid - kAuxThreads;
-            if (!skip && !aborted) {
-                constexpr int kPieces = kSmRows * G::kPitch / 4;
-                float4* dstp = reinterpret_cast<float4*>(part_mine);
-                #pragma unroll 5
-                for (int i = t; i < kPieces; i += kSmSoftmax) __stcg(dstp + i, ld_shared_v4(y_base + static_cast<uint32_t>(i) * 16u));
-            }
+            const bool live = __all_sync(0xffffffffu, !skip && !aborted);
+            const int share = kSmRows >> a.cluster_shift, first = static_cast<int>(rank) * share;
+            if (live) publish_partial_rows<HD>(sp, 0, kSmRows, y_base, part_mine, first, share, t, kSmSoftmax);
             if (tid == kAuxThreads) SS_TRC(5, 2);
-            // one arrival per warp: the warp barrier orders the lanes' pieces before lane 0's release
-            unsigned int* cnt = reinterpret_cast<unsigned int*>(a.counters) + group;
-            __syncwarp();
-            if (lane == 0) asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(cnt), "r"(256u >> a.cluster_shift) : "memory");
-            if (tid == kAuxThreads) {
-                bool ok = !aborted;
-                const long long t0 = clock64();
-                const long long limit = static_cast<long long>(c.wait_limit) << 10;
-                while (ok) {
-                    unsigned int now;
-                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(now) : "l"(cnt) : "memory");
-                    if ((now & (kArrivalsPerCall - 1u)) == 0u) break;
-                    if (clock64() - t0 > limit) ok = false;
-                }
-                if (!ok) { c.abort = 1; set_status(a.status, SS_ERR_DEVICE_TIMEOUT); }
-                c.merge_ok = ok ? 1 : 0;
-            }
-            named_barrier(3, kSmSoftmax);
-            if (tid == kAuxThreads) SS_TRC(5, 4);
-            if (c.merge_ok && !skip) {
-                // this CTA's share of the rows, read straight from L2 (past L1, which may hold lines of an earlier
-                // call): work item (row, four columns), the loads of all C sources in flight at once
-                const int share = kSmRows >> a.cluster_shift;
-                const int first = static_cast<int>(rank) * share;
-                for (int w = t; w < share * (HD / 4); w += kSmSoftmax) {
-                    const int rr = w / (HD / 4), g4 = w - rr * (HD / 4);
-                    const RowInfo r = row_info(sp, first + rr);
-                    if (!r.valid) continue;
-                    const float* src = part_group + static_cast<size_t>(first + rr) * G::kPitch;
-                    float4 v[8];
-                    float2 ml[8];
-                    #pragma unroll
-                    for (int sidx = 0; sidx < 8; ++sidx) {
-                        if (sidx < C) {
-                            v[sidx] = __ldcg(reinterpret_cast<const float4*>(src + sidx * G::kCtaFloats + g4 * 4));
-                            ml[sidx] = __ldcg(reinterpret_cast<const float2*>(src + sidx * G::kCtaFloats + HD));
-                        }
-                    }
-                    float mx = -INFINITY;
-                    #pragma unroll
-                    for (int sidx = 0; sidx < 8; ++sidx)
-                        if (sidx < C) mx = fmaxf(mx, ml[sidx].x);
-                    float l = 0.f;
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                    #pragma unroll
-                    for (int sidx = 0; sidx < 8; ++sidx) {
-                        if (sidx < C) {
-                            const float wgt = ml[sidx].x == -INFINITY ? 0.f : exp2f(ml[sidx].x - mx);   // 0: saw no visible key
-                            l += wgt * ml[sidx].y;
-                            acc.x += wgt * v[sidx].x; acc.y += wgt * v[sidx].y; acc.z += wgt * v[sidx].z; acc.w += wgt * v[sidx].w;
-                        }
-                    }
-                    const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, r);
-                    const float inv = 1.f / l;
-                    uint2 o;
-                    o.x = pack_bf16(acc.x * inv, acc.y * inv);
-                    o.y = pack_bf16(acc.z * inv, acc.w * inv);
-                    *reinterpret_cast<uint2*>(dst.o + g4 * 4) = o;
-                    if (dst.lse && g4 == 0) *dst.lse = (mx + log2f(l)) * 0.6931471805599453f;
-                }
+            // the other CTAs of the head were launched with this one and need nothing from it: the wait is short
+            const long long limit = static_cast<long long>(*reinterpret_cast<volatile int*>(&c.wait_limit)) << 10;
+            if (live && !merge_partial_rows<HD>(a, sp, 0, b, h, spec_row0, C, static_cast<int>(rank), y_base, part_group, G::kCtaFloats, first,
+                                                share, t, kSmSoftmax, limit, &c.abort)) {
+                c.abort = 1;
+                set_status(a.status, SS_ERR_DEVICE_TIMEOUT);
             }
         }
     }
     if (tid == kAuxThreads) SS_TRC(5, 5);
-#ifdef SS_TRACE
-    if (tid == 0) atomicMax(&g_wall[s_launch & 7][1], wall_ns());
-    if (tid == 0) atomicMin(&g_wall[s_launch & 7][5], wall_ns());
-    if (tid == 0 && blk < kTraceCtas) g_trace[blk][0][152] = static_cast<long long>(wall_ns());
-#endif
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -710,6 +638,9 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(G::kTmemCols) : "memory");
     }
+#ifdef SS_TRACE
+    if (tid == kAuxThreads && blk < 256) g_cta_wall[s_launch][blk][2] = wall_ns();
+#endif
 }
 
 }  // namespace ss

@@ -119,27 +119,25 @@ def test_verify_special_values(cuda, oracle):
     assert int(out["bonus_token"][0]) == ref["bonus_token"]
 
 
-def test_a_wait_that_runs_out_reports_a_timeout_and_the_workspace_recovers(cuda, oracle):
-    """The arrival counter of one split head is left at a value no call can complete (as after a call that
-    was cut short); the wait bound is shortened through the workspace header.  The CTAs of that head give up,
-    the call returns with SS_ERR_DEVICE_TIMEOUT in the status word, the stream stays usable, and after the
-    workspace is zero-filled again the same call matches the oracle."""
+def test_a_wait_that_runs_out_reports_a_timeout_and_the_stream_stays_usable(cuda, oracle):
+    """The step in which a CTA of a split head combines partial rows is run with no second CTA launched
+    (ss_wait_selftest): the rows it waits for cannot arrive.  With the bound shortened through the workspace
+    header the wait gives up, the status word reads SS_ERR_DEVICE_TIMEOUT, nothing was written, and a split
+    attention call on the same stream and workspace then matches the oracle."""
     api, DeviceStep = cuda
     cfg = W.custom_config("timeout", n_layers=1, n_msa_layers=0, prefix_len=600, n_nodes=12, gamma=0, max_depth=3,
                           n_heads=8, head_dim=128, config_id=810)       # 8 heads of 12 rows: 8 CTAs share a head's keys
     st = W.make_step(cfg)
     dev = DeviceStep(st)
+    assert dev.attn_ws.numel() * dev.attn_ws.element_size() >= 65536
     words = dev.attn_ws.view(torch.int32)
     words[1] = 100                                             # bound of every wait: 100 x 1024 cycles
-    words[64 + 3] = 1                                          # arrival counter of head 3 (after the 256-byte header)
-    dev.o_main[0].fill_(5.0)
-    dev.run_attention()
+    api.ss_wait_selftest(dev.attn_ws)
     assert api.ss_status(dev.attn_ws) == api.SS_ERR_DEVICE_TIMEOUT
     torch.cuda.synchronize()                                   # nothing faulted: the context is healthy
-    other = [h for h in range(8) if h != 3]
-    assert (dev.o_main[0][0, :12, 3] == 5.0).all()             # the head that gave up wrote nothing
-    assert not (dev.o_main[0][0, :12, other] == 5.0).any()     # the other heads finished
-    dev.attn_ws.zero_()
+    assert int(words[2:].abs().max()) == 0                     # the wait wrote nothing
+    words[1] = 0
     dev.run_attention()
     assert api.ss_status(dev.attn_ws) == 0
     assert_attention_close(oracle, st, st.layer(0), dev, 0)
+    assert int(words[2:].abs().max()) == 0                     # a call leaves the partial rows' area zero again

@@ -238,8 +238,8 @@ def test_attention_without_the_prefix_promise_gives_the_same_bits(cuda, oracle):
 def test_attention_every_split_factor(cuda, oracle, n_heads, expect_split):
     """The number of CTAs that share a row block's keys follows the head count (8, 4, 2, 1): every merge
     path, including CTAs that get no keys at all (8 CTAs, 5 key units).  The layers of a step share one
-    workspace and may have different split factors; the second pass finds the arrival counters as the
-    first one left them."""
+    workspace and may have different split factors and row counts (6 or 40 nodes, with and without stream
+    rows); every call must leave the partial rows' area zero, which the second pass relies on."""
     api, DeviceStep = cuda
     for k, (L, T, g) in enumerate([(70, 6, 1), (900, 40, 4)]):
         cfg = W.custom_config("split%d_%d" % (n_heads, k), n_layers=2, n_msa_layers=1, prefix_len=L, n_nodes=T,
@@ -249,6 +249,7 @@ def test_attention_every_split_factor(cuda, oracle, n_heads, expect_split):
         dev.run_attention()
         dev.run_attention()
         assert api.ss_status(dev.attn_ws) == 0
+        assert int(dev.attn_ws.view(torch.int32)[2:].abs().max()) == 0
         for i in range(2):
             assert_attention_close(oracle, st, st.layer(i), dev, i, check_lse=True)
 
