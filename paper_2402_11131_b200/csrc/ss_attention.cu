@@ -256,6 +256,25 @@ __device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t (&r)[64]) {
     tmem_ld32<32>(taddr + 32, r);
 }
 
+// packed pairs of fp32 (one instruction for two values)
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi) {
+    unsigned long long v;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
+    return v;
+}
+__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long d;
+    asm("fma.rn.ftz.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long add_f32x2(unsigned long long a, unsigned long long b) {
+    unsigned long long d;
+    asm("add.rn.ftz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -439,21 +458,26 @@ __device__ __forceinline__ float chunk_exp_store(const uint32_t (&v)[64], float 
 template <bool MASKED>
 __device__ __forceinline__ float chunk_exp_pack(const uint32_t (&v)[64], float scale, float m_use, unsigned long long vis,
                                                 uint32_t (&pk)[32]) {
-    float sum[4] = {0.f, 0.f, 0.f, 0.f};
+    // two scores per instruction (packed fp32 pairs) for the scaling and for the row sum
     const uint32_t vlo = static_cast<uint32_t>(vis), vhi = static_cast<uint32_t>(vis >> 32);
-    const float neg_m = -m_use;
+    const unsigned long long scale2 = pack_f32x2(scale, scale), shift2 = pack_f32x2(-m_use, -m_use);
+    unsigned long long sum2[2] = {pack_f32x2(0.f, 0.f), pack_f32x2(0.f, 0.f)};
     #pragma unroll
     for (int k = 0; k < 64; k += 2) {
-        float e0 = exp2f(fmaf(__uint_as_float(v[k]), scale, neg_m));
-        float e1 = exp2f(fmaf(__uint_as_float(v[k + 1]), scale, neg_m));
+        float t0, t1;
+        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[k]), __uint_as_float(v[k + 1])), scale2, shift2), t0, t1);
+        float e0 = exp2f(t0), e1 = exp2f(t1);
         if (MASKED) {
             e0 = (((k < 32 ? vlo : vhi) >> (k & 31)) & 1u) ? e0 : 0.f;
             e1 = (((k < 32 ? vlo : vhi) >> ((k + 1) & 31)) & 1u) ? e1 : 0.f;
         }
-        sum[(k >> 1) & 3] += e0 + e1;
+        sum2[(k >> 1) & 1] = add_f32x2(sum2[(k >> 1) & 1], pack_f32x2(e0, e1));
         pk[k >> 1] = pack_bf16(e0, e1);
     }
-    return (sum[0] + sum[1]) + (sum[2] + sum[3]);
+    float s0, s1, s2, s3;
+    unpack_f32x2(sum2[0], s0, s1);
+    unpack_f32x2(sum2[1], s2, s3);
+    return (s0 + s1) + (s2 + s3);
 }
 
 // Kernel variants.  kPair: a block of up to 128 rows; warpgroup w takes keys 64w .. 64w+63 of every

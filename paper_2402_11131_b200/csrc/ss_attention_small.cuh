@@ -474,30 +474,36 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
             if (j < 2) raise();                                               // every thread of the copy, so the barriers inside match
             bool leave = false;
             for (int attempt = 0; attempt < 3; ++attempt) {
-                float tmax = -INFINITY, lsum = 0.f;
+                float lsum = 0.f;
                 if (ok) {
+                    // two scores per instruction (packed fp32 pairs) for the scaling and for the row sum
                     uint32_t pk[16];
+                    const unsigned long long scale2 = pack_f32x2(a.scale_log2, a.scale_log2), shift2 = pack_f32x2(-m_ref, -m_ref);
+                    unsigned long long sum2 = pack_f32x2(0.f, 0.f);
                     #pragma unroll
                     for (int i = 0; i < 32; i += 2) {
-                        float t0 = fmaf(__uint_as_float(sr[i]), a.scale_log2, -m_ref);
-                        float t1 = fmaf(__uint_as_float(sr[i + 1]), a.scale_log2, -m_ref);
+                        float t0, t1;
+                        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sr[i]), __uint_as_float(sr[i + 1])), scale2, shift2), t0, t1);
                         float e0 = exp2f(t0), e1 = exp2f(t1);
                         if (masked) {
-                            const bool v0 = (vis >> i) & 1u, v1 = (vis >> (i + 1)) & 1u;
-                            t0 = v0 ? t0 : -INFINITY; t1 = v1 ? t1 : -INFINITY;
-                            e0 = v0 ? e0 : 0.f; e1 = v1 ? e1 : 0.f;
+                            e0 = ((vis >> i) & 1u) ? e0 : 0.f;
+                            e1 = ((vis >> (i + 1)) & 1u) ? e1 : 0.f;
                         }
-                        tmax = fmaxf(tmax, fmaxf(t0, t1));
-                        lsum += e0 + e1;
+                        sum2 = add_f32x2(sum2, pack_f32x2(e0, e1));
                         pk[i >> 1] = pack_bf16(e0, e1);
                     }
+                    float s0, s1;
+                    unpack_f32x2(sum2, s0, s1);
+                    lsum = s0 + s1;
                     // P of this copy's previous tile must have been read before it is overwritten
                     if (attempt == 0 && j >= 2) ok = mbar_wait_warp_s(smem_u32(&c.pv_done[copy]), ((j - 2) >> 1) & 1, &c, status);
                     if (ok) tmem_st16<0>(p_addr, pk);
                 }
                 if (leader) SS_TRC(3, 9 + 6 * j + (attempt > 0 ? 3 : 0));
                 // one reducing barrier per tile: did a score outgrow its reference, or did a wait run out
-                const uint32_t any = bar_red_or(4 + copy, 256, !ok || tmax > kRescaleStep);
+                // (a thread's 32 exponentials sum to at most 32 unless a score is above the reference; past
+                // 32 * 2^8 one of them is more than 2^8 above it)
+                const uint32_t any = bar_red_or(4 + copy, 256, !ok || lsum > 32.f * 256.f);
                 if (leader) SS_TRC(3, 10 + 6 * j);
                 if (!any) { l_part += lsum; break; }
                 if (*reinterpret_cast<volatile int*>(&c.abort)) { leave = true; break; }
