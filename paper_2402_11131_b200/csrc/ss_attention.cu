@@ -582,75 +582,91 @@ __device__ __forceinline__ void publish_partial_rows(const Span& sp, int row0, i
 // Step 2: this CTA's share of the block's rows, rows [first, first + share): its own partial from shared memory,
 // the others' from the workspace (part_group, one CTA's rows `cta_stride` floats after the previous one's).  A
 // row's items (four columns each) lie in one warp, so that one lane can clear the row's (m, l) once every lane
-// of the warp has read it.  Returns false when the wait ran out (limit in cycles) or another thread of the CTA
-// had given up.
-template <int HD>
-__device__ __forceinline__ bool merge_partial_rows(const AttnArgs& a, const Span& sp, int row0, int b, int h, long long spec_row0, int C, int rank,
-                                                   uint32_t y_base, const float* part_group, size_t cta_stride, int first, int share, int t,
-                                                   int threads, long long limit, volatile int* abort_flag) {
+// of the warp has read it.  A lane has the loads of BATCH rows x SLOTS sources in flight at once (the more rows
+// the fewer sources there are: every pass over a warp's rows costs a round trip to L2).  Returns false when the
+// wait ran out (limit in cycles) or another thread of the CTA had given up.
+template <int HD, int SLOTS, int BATCH>
+__device__ __forceinline__ bool merge_partial_rows_impl(const AttnArgs& a, const Span& sp, int row0, int b, int h, long long spec_row0, int C,
+                                                        int rank, uint32_t y_base, const float* part_group, size_t cta_stride, int first,
+                                                        int share, int t, int threads, long long limit, volatile int* abort_flag) {
     constexpr int kItems = HD / 4;                                   // items of a row
     constexpr int kLanes = kItems <= 16 ? 16 : 32;                   // lanes a row takes in a warp
     constexpr int kRowsPerWarp = 32 / kLanes;
     constexpr int kPitch = HD + 4;
     const int lane = t & 31, warp_t = t >> 5, n_warps = threads >> 5;
     const int sub = lane / kLanes, g4 = lane - sub * kLanes;
-    bool good = true;
-    for (int rbase = warp_t * kRowsPerWarp; rbase < share; rbase += n_warps * kRowsPerWarp) {     // warp-uniform
-        const int rr = rbase + sub;
-        const RowInfo r = row_info(sp, row0 + first + (rr < share ? rr : 0));
-        const bool mine = rr < share && g4 < kItems && r.valid;
-        float* src = const_cast<float*>(part_group) + static_cast<size_t>(first + (mine ? rr : 0)) * kPitch;
-        uint4 v[8];
-        uint2 ml[8];
-        uint32_t pending = mine ? ((1u << C) - 1u) & ~(1u << rank) : 0u;
-        if (mine) {
-            const uint32_t own = y_base + static_cast<uint32_t>(first + rr) * (kPitch * 4u);
-            const float4 ov = ld_shared_v4(own + static_cast<uint32_t>(g4) * 16u);
-            const float2 oml = ld_shared_v2(own + HD * 4u);
-            #pragma unroll
-            for (int sidx = 0; sidx < 8; ++sidx) {
-                if (sidx == rank) {
-                    v[sidx] = make_uint4(__float_as_uint(ov.x), __float_as_uint(ov.y), __float_as_uint(ov.z), __float_as_uint(ov.w));
-                    ml[sidx] = make_uint2(__float_as_uint(oml.x), __float_as_uint(oml.y));
+    for (int rbase = warp_t * kRowsPerWarp * BATCH; rbase < share; rbase += n_warps * kRowsPerWarp * BATCH) {     // warp-uniform
+        uint4 v[BATCH][SLOTS];
+        uint2 ml[BATCH][SLOTS];
+        uint32_t pending[BATCH];
+        float* src[BATCH];
+        RowInfo r[BATCH];
+        #pragma unroll
+        for (int bi = 0; bi < BATCH; ++bi) {
+            const int rr = rbase + bi * kRowsPerWarp + sub;
+            r[bi] = row_info(sp, row0 + first + (rr < share ? rr : 0));
+            const bool mine = rr < share && g4 < kItems && r[bi].valid;
+            r[bi].valid = mine;
+            src[bi] = const_cast<float*>(part_group) + static_cast<size_t>(first + (mine ? rr : 0)) * kPitch;
+            pending[bi] = mine ? ((1u << C) - 1u) & ~(1u << rank) : 0u;
+            if (mine) {
+                const uint32_t own = y_base + static_cast<uint32_t>(first + rr) * (kPitch * 4u);
+                const float4 ov = ld_shared_v4(own + static_cast<uint32_t>(g4) * 16u);
+                const float2 oml = ld_shared_v2(own + HD * 4u);
+                #pragma unroll
+                for (int sidx = 0; sidx < SLOTS; ++sidx) {
+                    if (sidx == rank) {
+                        v[bi][sidx] = make_uint4(__float_as_uint(ov.x), __float_as_uint(ov.y), __float_as_uint(ov.z), __float_as_uint(ov.w));
+                        ml[bi][sidx] = make_uint2(__float_as_uint(oml.x), __float_as_uint(oml.y));
+                    }
                 }
             }
         }
         const long long t0 = clock64();
         for (;;) {
             #pragma unroll
-            for (int sidx = 0; sidx < 8; ++sidx) {
-                if ((pending >> sidx) & 1u) {
-                    v[sidx] = ld_relaxed_v4(src + sidx * cta_stride + g4 * 4);
-                    ml[sidx] = ld_relaxed_v2(src + sidx * cta_stride + HD);
+            for (int bi = 0; bi < BATCH; ++bi) {
+                #pragma unroll
+                for (int sidx = 0; sidx < SLOTS; ++sidx) {
+                    if ((pending[bi] >> sidx) & 1u) {
+                        v[bi][sidx] = ld_relaxed_v4(src[bi] + sidx * cta_stride + g4 * 4);
+                        ml[bi][sidx] = ld_relaxed_v2(src[bi] + sidx * cta_stride + HD);
+                    }
                 }
             }
+            uint32_t left = 0u;
             #pragma unroll
-            for (int sidx = 0; sidx < 8; ++sidx)
-                if (((pending >> sidx) & 1u) && v[sidx].x != 0u && v[sidx].y != 0u && v[sidx].z != 0u && v[sidx].w != 0u && ml[sidx].x != 0u &&
-                    ml[sidx].y != 0u)
-                    pending &= ~(1u << sidx);
-            if (!__any_sync(0xffffffffu, pending != 0u)) break;
-            if (__any_sync(0xffffffffu, *abort_flag != 0 || clock64() - t0 > limit)) { good = false; break; }
+            for (int bi = 0; bi < BATCH; ++bi) {
+                #pragma unroll
+                for (int sidx = 0; sidx < SLOTS; ++sidx)
+                    if (((pending[bi] >> sidx) & 1u) && v[bi][sidx].x != 0u && v[bi][sidx].y != 0u && v[bi][sidx].z != 0u && v[bi][sidx].w != 0u &&
+                        ml[bi][sidx].x != 0u && ml[bi][sidx].y != 0u)
+                        pending[bi] &= ~(1u << sidx);
+                left |= pending[bi];
+            }
+            if (!__any_sync(0xffffffffu, left != 0u)) break;
+            if (__any_sync(0xffffffffu, *abort_flag != 0 || clock64() - t0 > limit)) return false;
         }
-        if (!good) break;
-        if (mine) {
+        #pragma unroll
+        for (int bi = 0; bi < BATCH; ++bi) {
+            if (!r[bi].valid) continue;
             float mx = -INFINITY;
             #pragma unroll
-            for (int sidx = 0; sidx < 8; ++sidx)
-                if (sidx < C) mx = fmaxf(mx, __uint_as_float(ml[sidx].x));
+            for (int sidx = 0; sidx < SLOTS; ++sidx)
+                if (sidx < C) mx = fmaxf(mx, __uint_as_float(ml[bi][sidx].x));
             float l = 0.f;
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             #pragma unroll
-            for (int sidx = 0; sidx < 8; ++sidx) {
+            for (int sidx = 0; sidx < SLOTS; ++sidx) {
                 if (sidx < C) {
-                    const float ms = __uint_as_float(ml[sidx].x);
+                    const float ms = __uint_as_float(ml[bi][sidx].x);
                     const float wgt = ms == -INFINITY ? 0.f : exp2f(ms - mx);       // 0: saw no visible key
-                    l += wgt * __uint_as_float(ml[sidx].y);
-                    acc.x += wgt * __uint_as_float(v[sidx].x); acc.y += wgt * __uint_as_float(v[sidx].y);
-                    acc.z += wgt * __uint_as_float(v[sidx].z); acc.w += wgt * __uint_as_float(v[sidx].w);
+                    l += wgt * __uint_as_float(ml[bi][sidx].y);
+                    acc.x += wgt * __uint_as_float(v[bi][sidx].x); acc.y += wgt * __uint_as_float(v[bi][sidx].y);
+                    acc.z += wgt * __uint_as_float(v[bi][sidx].z); acc.w += wgt * __uint_as_float(v[bi][sidx].w);
                 }
             }
-            const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, r);
+            const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, r[bi]);
             const float inv = 1.f / l;
             uint2 o;
             o.x = pack_bf16(acc.x * inv, acc.y * inv);
@@ -659,15 +675,23 @@ __device__ __forceinline__ bool merge_partial_rows(const AttnArgs& a, const Span
             if (dst.lse && g4 == 0) *dst.lse = (mx + log2f(l)) * 0.6931471805599453f;
             // what was read goes back to zero: every lane its own columns, one lane the row's (m, l)
             #pragma unroll
-            for (int sidx = 0; sidx < 8; ++sidx) {
+            for (int sidx = 0; sidx < SLOTS; ++sidx) {
                 if (sidx < C && sidx != rank) {
-                    st_relaxed_v4(src + sidx * cta_stride + g4 * 4, 0u, 0u, 0u, 0u);
-                    if (g4 == 0) st_relaxed_v2(src + sidx * cta_stride + HD, 0u, 0u);
+                    st_relaxed_v4(src[bi] + sidx * cta_stride + g4 * 4, 0u, 0u, 0u, 0u);
+                    if (g4 == 0) st_relaxed_v2(src[bi] + sidx * cta_stride + HD, 0u, 0u);
                 }
             }
         }
     }
-    return good;
+    return true;
+}
+template <int HD>
+__device__ __forceinline__ bool merge_partial_rows(const AttnArgs& a, const Span& sp, int row0, int b, int h, long long spec_row0, int C, int rank,
+                                                   uint32_t y_base, const float* part_group, size_t cta_stride, int first, int share, int t,
+                                                   int threads, long long limit, volatile int* abort_flag) {
+    if (C > 4) return merge_partial_rows_impl<HD, 8, 1>(a, sp, row0, b, h, spec_row0, C, rank, y_base, part_group, cta_stride, first, share, t, threads, limit, abort_flag);
+    if (C > 2) return merge_partial_rows_impl<HD, 4, 2>(a, sp, row0, b, h, spec_row0, C, rank, y_base, part_group, cta_stride, first, share, t, threads, limit, abort_flag);
+    return merge_partial_rows_impl<HD, 2, 4>(a, sp, row0, b, h, spec_row0, C, rank, y_base, part_group, cta_stride, first, share, t, threads, limit, abort_flag);
 }
 
 // 16 fp32 values scaled and packed to bf16 -> 32 bytes at dst
