@@ -341,6 +341,11 @@ def measure(args, workload, world, rank, local_rank):
     if status != 0:
         raise RuntimeError("device status %d after the timed region" % status)
 
+    # ---- the draft-management calls around the step (not part of it), each timed alone --------------
+    draft_us = None
+    if rank == 0:
+        draft_us = time_draft_management(dev, stream, capture, time_graph, max(10, min(K, 100)))
+
     # ---- end to end: per-step inputs from pinned host memory, results read back ------------------
     e2e = None
     if not args.no_e2e:
@@ -372,6 +377,7 @@ def measure(args, workload, world, rank, local_rank):
         "us_plain_layer": None if plain_ms is None else plain_ms * 1e3 / len(plain_idx),
         "us_msa_layer": None if msa_ms is None else msa_ms * 1e3 / len(msa_idx),
         "us_verify": verify_ms * 1e3, "us_compact": compact_ms * 1e3,
+        "draft_management_us": draft_us,
         "mean_accept_len": float(acc.mean()),
         "attention_tflops": attn_flops / (attn_ms * 1e-3) / 1e12,
         "gpu_launches": launches_per_step * K,
@@ -388,6 +394,60 @@ def measure(args, workload, world, rank, local_rank):
         line["cpu_baseline"] = cpu_baseline(st)
     return line
 
+
+
+def time_draft_management(dev, stream, capture, time_graph, reps):
+    """Microseconds per call of the entry points that build, prune and otherwise verify a draft, at the
+    workload's shapes (batch, tree size, streams, vocabulary, hidden = heads x head_dim), each replayed alone
+    as a CUDA graph on L2-warm synthetic logits.  They run once per step at most; the step timed above does
+    not contain them."""
+    import torch
+    from paper_2402_11131_b200 import api
+    c = dev.cfg
+    B, T, g, V = c.batch, c.n_nodes, max(1, c.gamma), c.vocab
+    hidden = c.n_heads * c.head_dim
+    gen = torch.Generator(device="cuda").manual_seed(1234)
+    k = 4
+    stream_logits = torch.randn((B, 1, g, V), device="cuda", generator=gen)
+    node_logits = dev.logits if dev.logits.shape == (B, T, V) else torch.randn((B, T, V), device="cuda", generator=gen)
+    uniforms = torch.rand((B, T), device="cuda", generator=gen)
+    bonus = torch.zeros(B, dtype=torch.int32, device="cuda")
+    new_tokens = torch.zeros((B, T), dtype=torch.int32, device="cuda")
+    new_trees, pruned_trees = api.empty_trees(B), api.empty_trees(B)
+    i32 = lambda *shape: torch.zeros(shape, dtype=torch.int32, device="cuda")
+    f32 = lambda *shape: torch.zeros(shape, dtype=torch.float32, device="cuda")
+    accept_len, accept_path, last_node, bonus_out, node_token = i32(B), i32(B, 64), i32(B), i32(B), i32(B, T)
+    edge_prob, entropy, new_index, kept_nodes, kept_tokens = f32(B, T), f32(B, T), i32(B, T), i32(B, T), i32(B, T)
+    ws_draft = api.workspace(api.ss_next_draft_workspace_bytes(B, g, V))
+    ws_stats = api.workspace(api.ss_tree_prune_workspace_bytes(B, T, V))
+    ws_sampled = api.workspace(api.ss_tree_verify_sampled_workspace_bytes(B, T, V))
+    rows = B * T
+    m_hidden = torch.randn((rows, hidden), device="cuda", generator=gen).to(torch.bfloat16)
+    p_emb = torch.randn((g, hidden), device="cuda", generator=gen).to(torch.bfloat16)
+    s_hidden = torch.empty((rows, g, hidden), dtype=torch.bfloat16, device="cuda")
+    v_main = torch.randn((rows, hidden), device="cuda", generator=gen).to(torch.bfloat16)
+    v_streams = torch.empty((rows, g, hidden), dtype=torch.bfloat16, device="cuda")
+    calls = {
+        "ss_next_draft": lambda s: api.ss_next_draft(stream_logits, None, bonus, k, T, new_tokens, new_trees, ws_draft, s),
+        "ss_tree_prune": lambda s: api.ss_tree_prune(node_logits, dev.tokens, dev.trees, 0.01, edge_prob, new_index, kept_nodes,
+                                                     kept_tokens, pruned_trees, ws_stats, s),
+        "ss_tree_verify_soft": lambda s: api.ss_tree_verify_soft(node_logits, dev.tokens, dev.trees, 0.09, 0.3, accept_len, accept_path,
+                                                                 last_node, bonus_out, edge_prob, entropy, ws_stats, s),
+        "ss_tree_verify_sampled": lambda s: api.ss_tree_verify_sampled(node_logits, dev.tokens, dev.trees, uniforms, k, accept_len,
+                                                                       accept_path, last_node, bonus_out, node_token, ws_sampled, s),
+        "ss_stream_insert": lambda s: api.ss_stream_insert(m_hidden, p_emb, s_hidden, s),
+        "ss_value_rotate": lambda s: api.ss_value_rotate(v_main, v_streams, 0.05, s),
+    }
+    out = {}
+    for name, fn in calls.items():
+        graph, _ = capture(fn)
+        out[name] = time_graph(graph, reps, 3) * 1e3
+    for ws in (ws_draft, ws_stats, ws_sampled):
+        status = api.ss_status(ws, stream)
+        if status != 0:
+            raise RuntimeError("device status %d after the draft-management calls" % status)
+    out["shapes"] = "batch %d, %d nodes, %d streams, vocabulary %d, top-%d, hidden %d" % (B, T, g, V, k, hidden)
+    return out
 
 
 def run_profile(args, st):
