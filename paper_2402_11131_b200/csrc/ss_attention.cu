@@ -188,6 +188,9 @@ __device__ __forceinline__ void named_barrier(int id, int threads) {
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
 }
+__device__ __forceinline__ void st_shared_v2(uint32_t addr, uint32_t x, uint32_t y) {
+    asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(addr), "r"(x), "r"(y) : "memory");
+}
 __device__ __forceinline__ float2 ld_shared_v2(uint32_t addr) {
     float2 v;
     asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
@@ -556,27 +559,35 @@ __device__ __forceinline__ uint2 ld_relaxed_v2(const float* p) {
     return v;
 }
 
-// Step 1: the staged rows (shared memory at y_base, `rows` rows of HD + 4 floats) go to this CTA's rows in the
-// workspace, a warp per row (whole lines), except the rows of this CTA's own share [first, first + share), which
-// it combines straight from shared memory.
+// Step 1: the staged rows (shared memory at y_base, `rows` rows of HD + 4 floats, no +0 among them) go to this
+// CTA's rows in the workspace as a few bulk copies (the copy engine moves them faster than the threads' stores
+// would -- those reach about 22 B per cycle and SM -- and leaves the load / store path to the polling that
+// follows): the rows that nodes own, [0, T) and [tmax8, spec_end) of the head, except those of this CTA's own
+// share [first, first + share), which it combines straight from shared memory.  Called by one thread once the
+// staged rows are complete (every thread that staged a row has executed fence.proxy.async before the barrier
+// that says so); bulk_copies_read() must follow before the shared memory is given up.
+__device__ __forceinline__ void bulk_copy_rows(float* dst, uint32_t src, int lo, int hi, uint32_t row_bytes) {
+    if (hi <= lo) return;
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(dst + static_cast<size_t>(lo) * (row_bytes / 4)), "r"(src + static_cast<uint32_t>(lo) * row_bytes),
+                   "r"(static_cast<uint32_t>(hi - lo) * row_bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_copies_read() {
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
 template <int HD>
-__device__ __forceinline__ void publish_partial_rows(const Span& sp, int row0, int rows, uint32_t y_base, float* part_mine, int first, int share,
-                                                     int t, int threads) {
+__device__ __forceinline__ void publish_partial_rows(const Span& sp, int row0, int rows, uint32_t y_base, float* part_mine, int first, int share) {
     constexpr uint32_t kRowBytes = (HD + 4) * 4;
-    const int lane = t & 31;
-    for (int rr = t >> 5; rr < rows; rr += threads >> 5) {                               // warp-uniform
-        if ((rr >= first && rr < first + share) || !row_info(sp, row0 + rr).valid) continue;
-        float* dst = part_mine + static_cast<size_t>(rr) * (HD + 4);
-        if (lane < HD / 4) {
-            const float4 v = ld_shared_v4(y_base + static_cast<uint32_t>(rr) * kRowBytes + static_cast<uint32_t>(lane) * 16u);
-            st_relaxed_v4(dst + lane * 4, never_plus_zero(__float_as_uint(v.x)), never_plus_zero(__float_as_uint(v.y)),
-                          never_plus_zero(__float_as_uint(v.z)), never_plus_zero(__float_as_uint(v.w)));
-        }
-        if (lane == 0) {
-            const float2 ml = ld_shared_v2(y_base + static_cast<uint32_t>(rr) * kRowBytes + HD * 4u);
-            st_relaxed_v2(dst + HD, never_plus_zero(__float_as_uint(ml.x)), never_plus_zero(__float_as_uint(ml.y)));
-        }
-    }
+    // the two ranges of owned rows, in rows of this block
+    const int a0 = 0, a1 = min(max(sp.T - row0, 0), rows);
+    const int b0 = max(min(max(sp.tmax8 - row0, 0), rows), a1), b1 = min(max(sp.spec_end - row0, 0), rows);
+    const int own0 = first, own1 = first + share;
+    // each range minus the own share: the part before it and the part after it
+    bulk_copy_rows(part_mine, y_base, a0, min(a1, own0), kRowBytes);
+    bulk_copy_rows(part_mine, y_base, max(a0, own1), a1, kRowBytes);
+    bulk_copy_rows(part_mine, y_base, b0, min(b1, own0), kRowBytes);
+    bulk_copy_rows(part_mine, y_base, max(b0, own1), b1, kRowBytes);
 }
 
 // Step 2: this CTA's share of the block's rows, rows [first, first + share): its own partial from shared memory,
@@ -1284,13 +1295,15 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                     if (dst.lse && wg == 0) *dst.lse = (m_out + log2f(l_out)) * 0.6931471805599453f;
                 }
             } else {
+                // (never +0: a word of a partial row that reads zero in the workspace has not arrived)
                 const uint32_t yrow = y_base + static_cast<uint32_t>(lrow) * RB;
                 #pragma unroll
                 for (int cc = 0; cc < G::kSplitCol; cc += 4)
                     if (c_lo + cc < c_hi)
-                        st_shared_v4(yrow + (c_lo + cc) * 4u, __float_as_uint(v[cc]), __float_as_uint(v[cc + 1]), __float_as_uint(v[cc + 2]),
-                                     __float_as_uint(v[cc + 3]));
-                if (wg == 0) st_shared_v4(yrow + HD * 4u, __float_as_uint(m_out), __float_as_uint(l_out), 0u, 0u);
+                        st_shared_v4(yrow + (c_lo + cc) * 4u, never_plus_zero(__float_as_uint(v[cc])), never_plus_zero(__float_as_uint(v[cc + 1])),
+                                     never_plus_zero(__float_as_uint(v[cc + 2])), never_plus_zero(__float_as_uint(v[cc + 3])));
+                if (wg == 0) st_shared_v4(yrow + HD * 4u, never_plus_zero(__float_as_uint(m_out)), never_plus_zero(__float_as_uint(l_out)), 0u, 0u);
+                fence_async_smem();                       // the copy engine reads these rows
             }
         }
         if (tid == kAuxThreads) SS_TR(5, 3);
@@ -1303,13 +1316,14 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
         const int t = tid - kAuxThreads;
         const bool live = __all_sync(0xffffffffu, !skip && *abort_flag == 0);
         const int share = rows_cap >> a.cluster_shift, first = static_cast<int>(rank) * share;
-        if (live) publish_partial_rows<HD>(sp, sp.row0, rows_cap, y_base, part_mine, first, share, t, wg_threads);
+        if (live && t == 0) publish_partial_rows<HD>(sp, sp.row0, rows_cap, y_base, part_mine, first, share);
         if (tid == kAuxThreads) SS_TR(5, 4);
         if (live && !merge_partial_rows<HD>(a, sp, sp.row0, b, h, spec_row0, C, static_cast<int>(rank), y_base, part_group,
                                             static_cast<size_t>(rows_cap) * RP, first, share, t, wg_threads, kWaitCycles, abort_flag)) {
             c.abort = 1;
             set_status(a.status, SS_ERR_DEVICE_TIMEOUT);
         }
+        if (live && t == 0) bulk_copies_read();
     }
     if (tid == kAuxThreads) SS_TR(5, 5);
 

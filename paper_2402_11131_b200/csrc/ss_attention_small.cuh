@@ -24,10 +24,10 @@
 // lane 0 issues S and hands K slots back; warp 2 lane 0 issues P V and hands V slots back; warps 4..19 are the
 // softmax threads, four to a TMEM lane.
 //
-// End of a CTA.  Copy 1 hands its partial rows (O, m, l) to copy 0 through shared memory.  C = 1: copy 0
-// normalises and writes bf16.  Split heads (C > 1): the combined rows go to the workspace in whole lines, and
-// each CTA combines its share of the rows from all C partials as they arrive (publish_partial_rows,
-// merge_partial_rows).
+// End of a CTA.  The copies exchange halves of their partial rows (O, m, l) through shared memory and each
+// combines the half it keeps.  C = 1: normalise and write bf16.  Split heads (C > 1): the combined rows go to the
+// workspace by bulk copy, and each CTA combines its share of the rows from all C partials as they arrive
+// (publish_partial_rows, merge_partial_rows).
 #pragma once
 
 namespace ss {
@@ -553,10 +553,10 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
 
     // ======================================== epilogue ==========================================
     // A lane's partial over the keys of its copy: O in TMEM, the reference, and the sum of its four threads' row
-    // sums.  Copy 1 hands its rows to copy 0 through shared memory (the ring is idle: every copy has landed and
-    // every MMA is complete).  C = 1: copy 0 normalises and writes bf16.  Split head: the combined rows go back
-    // to shared memory and from there, in whole lines, to the workspace (they stay in L2), and each CTA combines
-    // its share of the rows as they arrive from the CTAs of the head.
+    // sums.  The copies exchange halves of their rows through shared memory (the rings are idle: every copy has
+    // landed and every MMA is complete) and each combines the half it keeps.  C = 1: normalise and write bf16.
+    // Split head: the combined rows are staged in shared memory, the copy engine takes them to the workspace (they
+    // stay in L2), and each CTA combines its share of the rows as they arrive from the CTAs of the head.
     constexpr int CPT = G::kCpt;
     constexpr uint32_t YB = G::kPitch * 4;                                    // bytes of a staged row
     const uint32_t y_base = ring_base;                                        // [64 rows][kPitch floats]
@@ -577,47 +577,82 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
         }
         if (!has_acc || !ri.valid) { m_ref = -INFINITY; l_lane = 0.f; }
         if (tid == kAuxThreads) SS_TRC(5, 1);
-        const uint32_t yrow = y_base + static_cast<uint32_t>(row) * YB;
-        if (copy == 1) {
-            #pragma unroll
-            for (int i = 0; i < CPT; i += 4) st_shared_v4(yrow + static_cast<uint32_t>(CPT * w4 + i) * 4u, orr[i], orr[i + 1], orr[i + 2], orr[i + 3]);
-            if (w4 == 0) st_shared_v4(yrow + HD * 4u, __float_as_uint(m_ref), __float_as_uint(l_lane), 0u, 0u);
+        // The two threads that hold a row's columns [CPT w4, CPT w4 + CPT) -- one per copy -- each hand one half of
+        // them to the other through shared memory (X) and combine the half they keep: copy 0 the first CPT / 2
+        // columns, copy 1 the rest.
+        constexpr int HC = CPT / 2;                                           // columns a thread keeps
+        constexpr int VW = HC % 4 == 0 ? 4 : 2;                               // words per shared-memory access
+        const uint32_t x_base = y_base + kSmRows * YB;                        // [64 rows][kPitch floats], then (m, l) of both copies per row
+        const uint32_t xml = x_base + kSmRows * YB + static_cast<uint32_t>(row) * 16u;
+        const uint32_t yrow = y_base + static_cast<uint32_t>(row) * YB, xrow = x_base + static_cast<uint32_t>(row) * YB;
+        const int keep0 = copy == 0 ? 0 : HC, give0 = copy == 0 ? HC : 0;     // first kept / given column of my CPT
+        #pragma unroll
+        for (int i = 0; i < HC; ++i) {                                        // registers: kept columns first, then the given ones
+            const uint32_t lo = orr[i], hi = orr[HC + i];
+            orr[i] = copy == 0 ? lo : hi;
+            orr[HC + i] = copy == 0 ? hi : lo;
         }
+        #pragma unroll
+        for (int i = 0; i < HC; i += VW) {
+            const uint32_t at = xrow + static_cast<uint32_t>(CPT * w4 + give0 + i) * 4u;
+            if constexpr (VW == 4) st_shared_v4(at, orr[HC + i], orr[HC + i + 1], orr[HC + i + 2], orr[HC + i + 3]);
+            else st_shared_v2(at, orr[HC + i], orr[HC + i + 1]);
+        }
+        if (w4 == 0) st_shared_v2(xml + copy * 8u, __float_as_uint(m_ref), __float_as_uint(l_lane));
         named_barrier(8, kSmSoftmax);
         if (tid == kAuxThreads) SS_TRC(5, 8);
-        float m_out = m_ref, l_out = l_lane;
-        if (copy == 0) {
-            const float2 z = ld_shared_v2(yrow + HD * 4u);
-            m_out = fmaxf(m_ref, z.x);
-            const float wa = m_ref == -INFINITY ? 0.f : exp2f(m_ref - m_out), wb = z.x == -INFINITY ? 0.f : exp2f(z.x - m_out);
-            l_out = wa * l_lane + wb * z.y;
-            #pragma unroll
-            for (int i = 0; i < CPT; i += 4) {
-                const float4 t4 = ld_shared_v4(yrow + static_cast<uint32_t>(CPT * w4 + i) * 4u);
-                orr[i] = __float_as_uint(wa * __uint_as_float(orr[i]) + wb * t4.x);
-                orr[i + 1] = __float_as_uint(wa * __uint_as_float(orr[i + 1]) + wb * t4.y);
-                orr[i + 2] = __float_as_uint(wa * __uint_as_float(orr[i + 2]) + wb * t4.z);
-                orr[i + 3] = __float_as_uint(wa * __uint_as_float(orr[i + 3]) + wb * t4.w);
-            }
-            if (C == 1) {
-                if (ri.valid && !skip && !aborted) {
-                    const float inv = 1.f / l_out;
-                    const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, ri);
-                    #pragma unroll
-                    for (int i = 0; i < CPT; i += 4) {
-                        uint2 o;
-                        o.x = pack_bf16(__uint_as_float(orr[i]) * inv, __uint_as_float(orr[i + 1]) * inv);
-                        o.y = pack_bf16(__uint_as_float(orr[i + 2]) * inv, __uint_as_float(orr[i + 3]) * inv);
-                        *reinterpret_cast<uint2*>(dst.o + CPT * w4 + i) = o;
-                    }
-                    if (dst.lse && w4 == 0) *dst.lse = (m_out + log2f(l_out)) * 0.6931471805599453f;
-                }
+        const float2 z = ld_shared_v2(xml + (1 - copy) * 8u);                 // the other copy's (m, l)
+        const float m_out = fmaxf(m_ref, z.x);
+        const float wa = m_ref == -INFINITY ? 0.f : exp2f(m_ref - m_out), wb = z.x == -INFINITY ? 0.f : exp2f(z.x - m_out);
+        const float l_out = wa * l_lane + wb * z.y;
+        float keep[HC];
+        #pragma unroll
+        for (int i = 0; i < HC; i += VW) {
+            const uint32_t at = xrow + static_cast<uint32_t>(CPT * w4 + keep0 + i) * 4u;
+            if constexpr (VW == 4) {
+                const float4 t4 = ld_shared_v4(at);
+                keep[i] = wa * __uint_as_float(orr[i]) + wb * t4.x;
+                keep[i + 1] = wa * __uint_as_float(orr[i + 1]) + wb * t4.y;
+                keep[i + 2] = wa * __uint_as_float(orr[i + 2]) + wb * t4.z;
+                keep[i + 3] = wa * __uint_as_float(orr[i + 3]) + wb * t4.w;
             } else {
-                // same addresses this thread has just read: the combined row replaces copy 1's
-                #pragma unroll
-                for (int i = 0; i < CPT; i += 4) st_shared_v4(yrow + static_cast<uint32_t>(CPT * w4 + i) * 4u, orr[i], orr[i + 1], orr[i + 2], orr[i + 3]);
-                if (w4 == 0) st_shared_v4(yrow + HD * 4u, __float_as_uint(m_out), __float_as_uint(l_out), 0u, 0u);
+                const float2 t2 = ld_shared_v2(at);
+                keep[i] = wa * __uint_as_float(orr[i]) + wb * t2.x;
+                keep[i + 1] = wa * __uint_as_float(orr[i + 1]) + wb * t2.y;
             }
+        }
+        if (C == 1) {
+            if (ri.valid && !skip && !aborted) {
+                const float inv = 1.f / l_out;
+                const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, ri);
+                #pragma unroll
+                for (int i = 0; i < HC; i += VW) {
+                    __nv_bfloat16* at = dst.o + CPT * w4 + keep0 + i;
+                    if constexpr (VW == 4) {
+                        uint2 o;
+                        o.x = pack_bf16(keep[i] * inv, keep[i + 1] * inv);
+                        o.y = pack_bf16(keep[i + 2] * inv, keep[i + 3] * inv);
+                        *reinterpret_cast<uint2*>(at) = o;
+                    } else {
+                        *reinterpret_cast<uint32_t*>(at) = pack_bf16(keep[i] * inv, keep[i + 1] * inv);
+                    }
+                }
+                if (dst.lse && w4 == 0 && copy == 0) *dst.lse = (m_out + log2f(l_out)) * 0.6931471805599453f;
+            }
+        } else {
+            // the combined row, staged for the copy engine (never +0: a word of a partial row that reads zero in the
+            // workspace has not arrived)
+            #pragma unroll
+            for (int i = 0; i < HC; i += VW) {
+                const uint32_t at = yrow + static_cast<uint32_t>(CPT * w4 + keep0 + i) * 4u;
+                if constexpr (VW == 4)
+                    st_shared_v4(at, never_plus_zero(__float_as_uint(keep[i])), never_plus_zero(__float_as_uint(keep[i + 1])),
+                                 never_plus_zero(__float_as_uint(keep[i + 2])), never_plus_zero(__float_as_uint(keep[i + 3])));
+                else
+                    st_shared_v2(at, never_plus_zero(__float_as_uint(keep[i])), never_plus_zero(__float_as_uint(keep[i + 1])));
+            }
+            if (w4 == 0 && copy == 0) st_shared_v4(yrow + HD * 4u, never_plus_zero(__float_as_uint(m_out)), never_plus_zero(__float_as_uint(l_out)), 0u, 0u);
+            fence_async_smem();                           // the copy engine reads these rows
         }
         if (C > 1) {
             named_barrier(8, kSmSoftmax);                                     // the staged rows are complete
@@ -625,7 +660,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
             const int t = tid - kAuxThreads;
             const bool live = __all_sync(0xffffffffu, !skip && !aborted);
             const int share = kSmRows >> a.cluster_shift, first = static_cast<int>(rank) * share;
-            if (live) publish_partial_rows<HD>(sp, 0, kSmRows, y_base, part_mine, first, share, t, kSmSoftmax);
+            if (live && t == 0) publish_partial_rows<HD>(sp, 0, kSmRows, y_base, part_mine, first, share);
             if (tid == kAuxThreads) SS_TRC(5, 2);
             // the other CTAs of the head were launched with this one and need nothing from it: the wait is short
             const long long limit = static_cast<long long>(*reinterpret_cast<volatile int*>(&c.wait_limit)) << 10;
@@ -634,6 +669,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
                 c.abort = 1;
                 set_status(a.status, SS_ERR_DEVICE_TIMEOUT);
             }
+            if (live && t == 0) bulk_copies_read();
         }
     }
     if (tid == kAuxThreads) SS_TRC(5, 5);
