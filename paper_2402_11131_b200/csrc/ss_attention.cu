@@ -1,32 +1,30 @@
 // Tree-masked multi-stream attention, one layer (Eq. 1, Eq. 2): flash-decode for sm_100a.
 //
 // Work decomposition.  The query rows of a (sequence, head) pair -- T main rows, then the T*gamma
-// stream rows -- form one tile when there are at most 64 of them, else blocks of 128 rows that go to
-// separate CTAs (a block streams the keys it can see: the cached slots, and the stream keys of its own
-// nodes).  C CTAs (a power of two, chosen so that the grid fills the SMs once) share the keys of a
-// block: the cached slots [0, L+T) (prefix, then this step's tree nodes, masked by ancestry) and the
-// block's transient stream keys (node-major) are cut into 16-key units and CTA r takes units
-// [U*r/C, U*(r+1)/C), so every CTA of a block streams the same number of bytes.  The CTAs of a pair
-// run in the same wave, so a K/V tile crosses HBM once and is served from L2 to the other row blocks.
-// A batch (up to 32 sequences, no key split) is dispatched longest prefix first.
+// stream rows -- form one tile when there are at most 64 of them (msa_attention_small_kernel, in
+// ss_attention_small.cuh), else blocks of 128 rows that go to separate CTAs (msa_attention_kernel, here;
+// a block streams the keys it can see: the cached slots, and the stream keys of its own nodes).  C CTAs
+// (a power of two, chosen so that the grid fills the SMs once) share the keys of a block: the cached
+// slots [0, L+T) (prefix, then this step's tree nodes, masked by ancestry) and the block's transient
+// stream keys (node-major) are cut into 16-key units and CTA r takes units [U*r/C, U*(r+1)/C), so every
+// CTA of a block streams the same number of bytes.  The CTAs of a pair run in the same wave, so a K/V
+// tile crosses HBM once and is served from L2 to the other row blocks.  A batch (up to 32 sequences, no
+// key split) is dispatched longest prefix first.
 //
-// Inside a CTA.
+// Inside a CTA of msa_attention_kernel.
 //   threads 0, 96  TMA producers of the K ring and of the V ring (mbarrier complete_tx); swizzle-128B
 //               boxes straight from the caller's strided tensors.  A K slot is handed back as soon
 //               as S is queued, a V slot after P V.  Thread 0 also requests Q once.
 //   warp 1      tcgen05 issuer of S = Q K^T (128 x 128 keys x d) into one of two TMEM buffers;
-//   warp 2      tcgen05 issuer of O += P V into the TMEM accumulator of a warpgroup;
+//   warp 2      tcgen05 issuer of O += P V (A = P in TMEM) into the TMEM accumulator of a warpgroup;
 //               tcgen05.commit arrives on the mbarriers that hand buffers back.
-//   warps 4..11 two softmax warpgroups, one thread per TMEM lane: tcgen05.ld of 64 scores of the row,
-//               tree / stream mask from the node's 64-bit ancestor word, online softmax in fp32
-//               registers (the running maximum is only raised when it would grow by more than 2^8,
-//               which keeps the TMEM accumulator untouched on almost every tile), P as bf16 into a
-//               swizzled shared-memory tile that feeds the second MMA.
-// Two variants (enum Mode) map rows and keys to the warpgroups.  kPair: a block of up to 128 rows; of
-// every 128-key tile warpgroup 0 takes keys 0..63 and warpgroup 1 keys 64..127, each with its own P
-// tile, running maximum and accumulator.  kDual, for heads of at most 64 rows: the block holds the
-// rows twice (copy 0 takes keys 0..63, copy 1 keys 64..127) and the two warpgroups take alternate
-// tiles.  Either way all four sub-partitions of the SM share a tile's exponentials.
+//   warps 4..11 two softmax warpgroups, one thread per TMEM lane: of every 128-key tile warpgroup 0 takes
+//               keys 0..63 and warpgroup 1 keys 64..127, each with its own running maximum and
+//               accumulator: tcgen05.ld of 64 scores of the row, tree / stream mask from the node's
+//               64-bit ancestor word, online softmax in fp32 registers (the running maximum is only
+//               raised when it would grow by more than 2^8, which keeps the TMEM accumulator untouched
+//               on almost every tile), P as bf16 written over the first 32 of the score columns just
+//               read, from where the second MMA takes it.
 //
 // Split-KV merge.  Each CTA ends with un-normalised (m, l, O) per row, combines what it holds for a
 // row locally, and -- when the keys were split -- leaves one partial row in the workspace (it stays in
@@ -85,7 +83,7 @@ struct alignas(64) AttnArgs {
     int batch, n_heads, gamma, max_nodes;
     int tmax8;                       // max_nodes rounded up to 8: first stream row of the head's query tile
     int s0rows;                      // stream rows that share block 0 with the main rows
-    int n_blocks;                    // 128-row blocks per head (kPair), 1 for kDual
+    int n_blocks;                    // 128-row blocks per head (1 for heads of at most 64 rows)
     int cluster, cluster_shift;      // CTAs that share a block's keys; cluster = 1 << cluster_shift
     int n_kslots, n_vslots;          // ring depths
     int head_coord;                  // 1, or 0 when all heads share one K/V (head stride 0)
@@ -109,16 +107,15 @@ struct Ctrl {
     unsigned long long k_full[kMaxSlots], k_empty[kMaxSlots], v_full[kMaxSlots], v_empty[kMaxSlots];
     unsigned long long s_full[2][2];            // per (warpgroup, S buffer): a warpgroup sees every phase of its own
     unsigned long long s_free[2];
-    // P of a warpgroup written.  kDual: [w][0], one arrival per thread.  kPair: [w][tile & 1], one arrival per warp: a
-    // warp can only be two tiles ahead of another once the P V between them is complete, so it never arrives twice in a phase
+    // P of a warpgroup written: [w][tile & 1], one arrival per warp: a warp can only be two tiles ahead of another
+    // once the P V between them is complete, so it never arrives twice in a phase
     unsigned long long p_full[2][2];
-    // P V of a warpgroup complete.  kDual: [w][0].  kPair: [w][tile & 1]: a warpgroup that does not look at every
-    // phase is then never more than one phase behind, which a parity wait needs
+    // P V of a warpgroup complete: [w][tile & 1]: a warpgroup that does not look at every phase is then never more
+    // than one phase behind, which a parity wait needs
     unsigned long long o_done[2][2];
     unsigned long long anc[SS_MAX_NODES];
     uint32_t tmem_base;
     int abort;
-    int merge_ok;                // the block's other CTAs arrived in time
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -432,32 +429,7 @@ __device__ __forceinline__ float chunk_max(const uint32_t (&v)[64], float scale,
     }
     return fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
 }
-// p = exp2(s * scale - m) for 64 scores -> bf16 into the row's eight 16-byte chunks; returns sum of p
-template <bool MASKED>
-__device__ __forceinline__ float chunk_exp_store(const uint32_t (&v)[64], float scale, float m_use, unsigned long long vis,
-                                                 uint32_t p_row, int row_in_blk) {
-    float sum[4] = {0.f, 0.f, 0.f, 0.f};
-    const uint32_t vlo = static_cast<uint32_t>(vis), vhi = static_cast<uint32_t>(vis >> 32);
-    const float neg_m = -m_use;
-    #pragma unroll
-    for (int ch = 0; ch < 8; ++ch) {
-        float p[8];
-        #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int k = ch * 8 + i;
-            float e = exp2f(fmaf(__uint_as_float(v[k]), scale, neg_m));
-            if (MASKED) e = (((k < 32 ? vlo : vhi) >> (k & 31)) & 1u) ? e : 0.f;
-            p[i] = e;
-            sum[i & 3] += e;
-        }
-        const uint32_t dst = p_row + ((ch ^ (row_in_blk & 7)) << 4);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pack_bf16(p[0], p[1])),
-                     "r"(pack_bf16(p[2], p[3])), "r"(pack_bf16(p[4], p[5])), "r"(pack_bf16(p[6], p[7])) : "memory");
-    }
-    return (sum[0] + sum[1]) + (sum[2] + sum[3]);
-}
-
-// the same exponentials, packed two bf16 to a word (key 2c in the low half of word c); returns the sum
+// p = exp2(s * scale - m) for 64 scores, packed two bf16 to a word (key 2c in the low half of word c); returns the sum of p
 template <bool MASKED>
 __device__ __forceinline__ float chunk_exp_pack(const uint32_t (&v)[64], float scale, float m_use, unsigned long long vis,
                                                 uint32_t (&pk)[32]) {
@@ -483,15 +455,13 @@ __device__ __forceinline__ float chunk_exp_pack(const uint32_t (&v)[64], float s
     return (s0 + s1) + (s2 + s3);
 }
 
-// Kernel variants.  kPair: a block of up to 128 rows; warpgroup w takes keys 64w .. 64w+63 of every
-// tile, with its own P tile (64 keys wide), running maximum and accumulator.  kDual: at most 64 rows:
-// the block holds the rows twice, copy 0 takes keys 0..63 of a tile and copy 1 keys 64..127 (P is zero
-// in the other half), and the two warpgroups, each with its own accumulator, take alternate tiles, so
-// one tile's softmax overlaps the other's MMAs.  The partials a row then has inside the CTA (two, four)
-// are combined before the merge across CTAs.
-enum Mode { kPair = 0, kCols = 1, kDual = 2 };
+// Which kernel a call takes: kCols, heads of at most 64 rows (msa_attention_small_kernel); kPair, blocks of up to
+// 128 rows of larger heads (msa_attention_kernel: warpgroup w takes keys 64w .. 64w+63 of every tile, with its own
+// running maximum and accumulator; the two partials a row then has inside the CTA are combined before the merge
+// across CTAs).
+enum Mode { kPair = 0, kCols = 1 };
 
-template <int HD, int MODE>
+template <int HD>
 struct Geo {
     static constexpr int kHalves = HD > 64 ? 2 : 1;               // 64-element boxes along head_dim
     static constexpr int kBoxBytes = kTileKeys * 128;             // one TMA box: 128 keys x 128 B
@@ -502,13 +472,8 @@ struct Geo {
     static constexpr uint32_t kIdescPV = idesc_bf16(HD, false, true);
     static constexpr int kOCols = 128;                            // TMEM columns reserved per accumulator
     static constexpr int kThreads = kAuxThreads + 2 * kBlockRows; // two softmax warpgroups
-    static constexpr int kCopies = MODE == kDual ? 2 : 1;
-    // P of one warpgroup, 128 B rows of 64 keys (swizzled).  kPair: 128 rows.  kDual: [copy-0 rows 0..63 |
-    // 64 zero rows | copy-1 rows 0..63]; the MMA reads keys 0..63 from the first 128 rows and keys 64..127
-    // from the last 128 rows, so each copy's other half is zero.
-    static constexpr uint32_t kPBytes = MODE == kDual ? 3u * 64u * 128u : 0u;
-    static constexpr int kRowsCap = MODE == kDual ? 64 : kBlockRows;   // partial rows a CTA ships
-    static constexpr int kSplitCol = ((HD / 16 + 1) / 2) * 16;    // kPair: warpgroup 0 finishes columns [0, kSplitCol)
+    static constexpr int kRowsCap = kBlockRows;                   // partial rows a CTA ships
+    static constexpr int kSplitCol = ((HD / 16 + 1) / 2) * 16;    // warpgroup 0 finishes columns [0, kSplitCol)
 };
 
 // destination of a row's output and log-sum-exp
@@ -715,11 +680,10 @@ __device__ __forceinline__ void store_bf16x16(__nv_bfloat16* dst, const float (&
 }
 
 // ---------------------------------------------------------------------------------------------
-template <int HD, int MODE>
-__global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kernel(const __grid_constant__ AttnArgs a) {
-    using G = Geo<HD, MODE>;
+template <int HD>
+__global__ void __launch_bounds__(Geo<HD>::kThreads, 1) msa_attention_kernel(const __grid_constant__ AttnArgs a) {
+    using G = Geo<HD>;
     constexpr int TK = kTileKeys;
-    constexpr bool kIsDual = MODE == kDual;
     extern __shared__ unsigned char smem_raw[];
     __shared__ Ctrl c;
 
@@ -727,8 +691,8 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     const int C = a.cluster;
     const uint32_t rank = blockIdx.x & (C - 1);            // C is a power of two
     const int group = blockIdx.x >> a.cluster_shift;       // (pair, row block): the CTAs that share its keys
-    const int rb = kIsDual ? 0 : group % a.n_blocks;
-    const int pair = kIsDual ? group : group / a.n_blocks;
+    const int rb = group % a.n_blocks;
+    const int pair = group / a.n_blocks;
     int b = pair / a.n_heads;                              // the sequence (for a batch: its place in the dispatch order, see below)
     const int h = pair - b * a.n_heads;
     const int nk = a.n_kslots, nv_slots = a.n_vslots;
@@ -754,9 +718,8 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     // memory held, which only ever reaches padding rows of S and O.
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     constexpr uint32_t kQHalfBytes = kBlockRows * 128u;
-    const uint32_t q_base = base;                                       // [half][128 rows][128 B]; kDual: second copy at row 64
-    const uint32_t p_base = q_base + G::kHalves * kQHalfBytes;          // [warpgroup][kPBytes]
-    const uint32_t k_base = p_base + 2u * G::kPBytes;                   // [slot][half][128 keys][128 B]
+    const uint32_t q_base = base;                                       // [half][128 rows][128 B]
+    const uint32_t k_base = q_base + G::kHalves * kQHalfBytes;          // [slot][half][128 keys][128 B]
     const uint32_t v_base = k_base + nk * G::kSlotBytes;                // [slot][half][128 keys][128 B]
     const uint32_t merge_base = base;                                   // aliases everything above, after the main loop
 
@@ -804,10 +767,10 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     } else if (tid == 64) {                               // every other barrier (first used after the CTA-wide sync)
         for (int s = 0; s < kMaxSlots; ++s) { mbar_init(smem_u32(&c.k_empty[s]), 1); mbar_init(smem_u32(&c.v_empty[s]), 1); }
         for (int s = 0; s < 2; ++s) {
-            mbar_init(smem_u32(&c.s_free[s]), kIsDual ? 4 : 1);          // kDual: warps that read an S buffer; kPair: the P V commit
+            mbar_init(smem_u32(&c.s_free[s]), 1);                        // the P V commit
             mbar_init(smem_u32(&c.s_full[0][s]), 1);
             mbar_init(smem_u32(&c.s_full[1][s]), 1);
-            mbar_init(smem_u32(&c.p_full[s][0]), kIsDual ? kBlockRows : 4);   // kDual: threads; kPair: warps
+            mbar_init(smem_u32(&c.p_full[s][0]), 4);                     // the warps of a warpgroup
             mbar_init(smem_u32(&c.p_full[s][1]), 4);
             mbar_init(smem_u32(&c.o_done[s][0]), 1);
             mbar_init(smem_u32(&c.o_done[s][1]), 1);
@@ -893,18 +856,15 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
         const uint32_t qbar = smem_u32(&c.q_full);
         const bool with_spec = a.gamma > 0 && a.s0rows > 0;
         const uint32_t rows = rb > 0 ? kBlockRows : a.tmax8 + (with_spec ? a.s0rows : 0);
-        mbar_expect_tx(qbar, G::kCopies * G::kHalves * rows * 128u);
+        mbar_expect_tx(qbar, G::kHalves * rows * 128u);
         #pragma unroll
-        for (int cp = 0; cp < G::kCopies; ++cp) {
-            #pragma unroll
-            for (int hh = 0; hh < G::kHalves; ++hh) {
-                const uint32_t dst = q_base + hh * kQHalfBytes + cp * 64u * 128u;
-                if (rb > 0) {
-                    tma_load_3d(dst, &a.tm_qs1, hh * 64, h, static_cast<int>(spec_row0 + rb * kBlockRows - a.tmax8), qbar);
-                } else {
-                    tma_load_3d(dst, &a.tm_qm, hh * 64, h, b * a.max_nodes, qbar);
-                    if (with_spec) tma_load_3d(dst + a.tmax8 * 128u, &a.tm_qs, hh * 64, h, static_cast<int>(spec_row0), qbar);
-                }
+        for (int hh = 0; hh < G::kHalves; ++hh) {
+            const uint32_t dst = q_base + hh * kQHalfBytes;
+            if (rb > 0) {
+                tma_load_3d(dst, &a.tm_qs1, hh * 64, h, static_cast<int>(spec_row0 + rb * kBlockRows - a.tmax8), qbar);
+            } else {
+                tma_load_3d(dst, &a.tm_qm, hh * 64, h, b * a.max_nodes, qbar);
+                if (with_spec) tma_load_3d(dst + a.tmax8 * 128u, &a.tm_qs, hh * 64, h, static_cast<int>(spec_row0), qbar);
             }
         }
     } else if (tid == 96) {
@@ -912,14 +872,6 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     }
     if (tid >= kAuxThreads && tid < kAuxThreads + SS_MAX_NODES) c.anc[tid - kAuxThreads] = __ldcg(&a.trees[b].anc_mask[tid - kAuxThreads]);
     if (tid == 0) SS_TR(0, 5);
-    // kDual: the 64 zero rows in the middle of each warpgroup's P stay zero for the whole kernel
-    if (kIsDual && tid >= kAuxThreads) {
-        const int r = tid - kAuxThreads;                                  // 256 threads, 64 B each per warpgroup
-        const uint32_t dst = p_base + (r >> 7) * G::kPBytes + 64u * 128u + (r & 127) * 64u;
-        #pragma unroll
-        for (int i = 0; i < 4; ++i) st_shared_v4(dst + i * 16, 0u, 0u, 0u, 0u);
-        fence_async_smem();
-    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -932,9 +884,8 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     int n_own = 0;
     const int wg = (warp - 4) >> 2;                                           // softmax warpgroup 0 / 1
     const int row_in_blk = ((warp & 3) << 5) | lane;                          // TMEM lane of this thread
-    const int copy = kIsDual ? (row_in_blk >> 6) : 0;
-    const int lrow = kIsDual ? (row_in_blk & 63) : row_in_blk;                // row of the block this thread works for
-    const int chunk = kIsDual ? copy : wg;                                    // 64-key half of a tile this thread handles
+    const int lrow = row_in_blk;                                              // row of the block this thread works for
+    const int chunk = wg;                                                     // 64-key half of a tile this thread handles
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     RowInfo ri;
     ri.valid = false; ri.node = 0; ri.stream = 0;
@@ -997,12 +948,8 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                     tc_mma(tmem_s + buf * TK, dq + ((hh * kQHalfBytes + off) >> 4), dk + ((hh * G::kBoxBytes + off) >> 4), G::kIdescS, ks > 0);
                 }
                 SS_TR(1, 10 + 4 * j);
-                if (kIsDual) {
-                    tc_commit(smem_u32(&c.s_full[buf][buf]));            // tile j belongs to warpgroup j & 1
-                } else {
-                    tc_commit(smem_u32(&c.s_full[0][buf]));
-                    tc_commit(smem_u32(&c.s_full[1][buf]));
-                }
+                tc_commit(smem_u32(&c.s_full[0][buf]));
+                tc_commit(smem_u32(&c.s_full[1][buf]));
                 tc_commit(smem_u32(&c.k_empty[rk.slot]));                // S of tile j is queued: K may go
                 SS_TR(1, 11 + 4 * j);
             }
@@ -1018,19 +965,7 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 if (!mbar_wait(smem_u32(&c.v_full[rv.slot]), rv.round & 1, abort_flag, a.status)) break;
                 SS_TR(2, 8 + 4 * j);
                 const uint32_t va = v_base + rv.slot * G::kSlotBytes;
-                if (kIsDual) {
-                    // the whole tile for warpgroup j & 1: keys 0..63 from copy 0's rows, 64..127 from copy 1's
-                    const int w = j & 1;
-                    if (!mbar_wait(smem_u32(&c.p_full[w][0]), (j >> 1) & 1, abort_flag, a.status)) break;
-                    SS_TR(2, 9 + 4 * j);
-                    tc_fence_after();
-                    const uint64_t dp = desc_k_major(p_base + w * G::kPBytes), dv = desc_mn_major(va, G::kBoxBytes);
-                    #pragma unroll
-                    for (int ks = 0; ks < TK / 16; ++ks)
-                        tc_mma(tmem + w * G::kOCols, dp + (((ks >> 2) * (64u * 128u) + (ks & 3) * 32u) >> 4), dv + ((ks * 2048u) >> 4),
-                               G::kIdescPV, (j >= 2 || ks > 0) ? 1u : 0u);
-                    tc_commit(smem_u32(&c.o_done[w][0]));
-                } else {
+                {
                     // keys 64w .. 64w+63 into the accumulator of warpgroup w; P is read from TMEM, where the
                     // warpgroup left it over the first 32 columns of its half of the S buffer
                     const int buf = j & 1;
@@ -1062,15 +997,13 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
         // a warp whose 32 rows are all padding skips the arithmetic but keeps the barrier protocol
         const bool warp_active = __any_sync(0xffffffffu, ri.valid);
         const uint32_t o_addr = tmem + lane_base + wg * G::kOCols;
-        const uint32_t p_row = kIsDual ? p_base + wg * G::kPBytes + copy * (128u * 128u) + lrow * 128u
-                                       : p_base + wg * G::kPBytes + row_in_blk * 128u;
         Ring rv;                                       // V ring position of tile j
         rv.start();
         int v_tile = 0;
-        for (int j = kIsDual ? wg : 0; j < sp.n_tiles; j += kIsDual ? 2 : 1) {
+        for (int j = 0; j < sp.n_tiles; ++j) {
             while (v_tile < j) { rv.advance(nv_slots); ++v_tile; }
             const int buf = j & 1;
-            // uses of (warpgroup, buffer) so far: j >> 1 in either variant
+            // uses of (warpgroup, buffer) so far: j >> 1
             if (!mbar_wait_warp(smem_u32(&c.s_full[wg][buf]), (j >> 1) & 1, abort_flag, a.status)) break;
             [[maybe_unused]] const int trole = 3 + wg;
             [[maybe_unused]] const bool tr_on = row_in_blk == 0;
@@ -1099,19 +1032,8 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             }
             if (tr_on) SS_TR(trole, 9 + 6 * n_own);
             const bool rescale = n_own > 0 && __any_sync(0xffffffffu, need);
-            if (kIsDual) {
-                // the scores stay in registers: S can be overwritten
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&c.s_free[buf]));
-                // the previous PV of this warpgroup must be complete: it read the P tile that is about to
-                // be overwritten, and it wrote the accumulator that a raised maximum rescales
-                if (n_own > 0) {
-                    if (!mbar_wait_warp(smem_u32(&c.o_done[wg][0]), (n_own - 1) & 1, abort_flag, a.status)) break;
-                    tc_fence_after();
-                }
-            } else if (rescale) {
-                // kPair: P goes to the S buffer itself (handed back by the P V that reads it), so only a raised
+            if (rescale) {
+                // P goes to the S buffer itself (handed back by the P V that reads it), so only a raised
                 // maximum waits for the previous P V: it rescales the accumulator that P V wrote
                 // (S of this tile exists, so the P V two tiles back is complete: the barrier is at most one phase behind)
                 if (!mbar_wait_warp(smem_u32(&c.o_done[wg][(j - 1) & 1]), ((j - 1) >> 1) & 1, abort_flag, a.status)) break;
@@ -1133,23 +1055,18 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
                 }
                 // ---- pass 2: P = exp2(S - m) as bf16, row sum -------------------------------------------
                 const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
-                if (kIsDual) {
-                    l_run += masked ? chunk_exp_store<true>(sr, a.scale_log2, m_use, vis, p_row, row_in_blk)
-                                    : chunk_exp_store<false>(sr, a.scale_log2, m_use, 0ull, p_row, row_in_blk);
-                } else {
-                    // two bf16 to a column, over the first 32 of the 64 score columns this thread has read
-                    uint32_t pk[32];
-                    l_run += masked ? chunk_exp_pack<true>(sr, a.scale_log2, m_use, vis, pk) : chunk_exp_pack<false>(sr, a.scale_log2, m_use, 0ull, pk);
-                    tmem_st32(s_addr, pk);
-                    tmem_wait_st();
-                }
+                // two bf16 to a column, over the first 32 of the 64 score columns this thread has read
+                uint32_t pk[32];
+                l_run += masked ? chunk_exp_pack<true>(sr, a.scale_log2, m_use, vis, pk) : chunk_exp_pack<false>(sr, a.scale_log2, m_use, 0ull, pk);
+                tmem_st32(s_addr, pk);
+                tmem_wait_st();
             }
             if (tr_on) SS_TR(trole, 11 + 6 * n_own);
             // V rows past the end of the sequence's keys may hold anything (even NaN patterns): P is 0
-            // there, but 0 * NaN is NaN, so the warpgroup clears the ones its P V reads (kDual: the whole
-            // tile, kPair: its half).  Rows that only lie past this CTA's share of the keys are real data.
+            // there, but 0 * NaN is NaN, so the warpgroup clears the ones its P V reads (its half of the tile).
+            // Rows that only lie past this CTA's share of the keys are real data.
             const int region_left = (cache ? sp.L + sp.T : sp.n_stream) - x;      // real rows in the tile
-            const int fix_lo = max(region_left, kIsDual ? 0 : wg * 64), fix_hi = kIsDual ? TK : wg * 64 + 64;
+            const int fix_lo = max(region_left, wg * 64), fix_hi = wg * 64 + 64;
             if (fix_lo < fix_hi) {
                 if (!mbar_wait_warp(smem_u32(&c.v_full[rv.slot]), rv.round & 1, abort_flag, a.status)) break;
                 const uint32_t vdst = v_base + rv.slot * G::kSlotBytes;
@@ -1164,24 +1081,16 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             if (tr_on) SS_TR(trole, 12 + 6 * n_own);
             fence_async_smem();
             tc_fence_before();
-            if (kIsDual) {
-                mbar_arrive(smem_u32(&c.p_full[wg][0]));
-            } else {
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&c.p_full[wg][buf]));
-            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&c.p_full[wg][buf]));
             if (tr_on) SS_TR(trole, 13 + 6 * n_own);
             ++n_own;
         }
         // the warpgroup's last PV must have landed in TMEM before the accumulator is read
         if (n_own > 0) {
-            if (kIsDual) {
-                mbar_wait_warp(smem_u32(&c.o_done[wg][0]), (n_own - 1) & 1, abort_flag, a.status);
-            } else {
-                // the last two P V may both be outstanding: one barrier each
-                if (n_own > 1) mbar_wait_warp(smem_u32(&c.o_done[wg][(n_own - 2) & 1]), ((n_own - 2) >> 1) & 1, abort_flag, a.status);
-                mbar_wait_warp(smem_u32(&c.o_done[wg][(n_own - 1) & 1]), ((n_own - 1) >> 1) & 1, abort_flag, a.status);
-            }
+            // the last two P V may both be outstanding: one barrier each
+            if (n_own > 1) mbar_wait_warp(smem_u32(&c.o_done[wg][(n_own - 2) & 1]), ((n_own - 2) >> 1) & 1, abort_flag, a.status);
+            mbar_wait_warp(smem_u32(&c.o_done[wg][(n_own - 1) & 1]), ((n_own - 1) >> 1) & 1, abort_flag, a.status);
             tc_fence_after();
         }
     }
@@ -1202,15 +1111,12 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
     float* const part_mine = part_group + static_cast<size_t>(rank) * rows_cap * RP;
 
     // Shared memory after the main loop: 2 KB in which the warpgroups exchange their (m, l) (the first thing
-    // a finished warpgroup writes); once both warpgroups are done, kDual: Z, the rows of copy 1 on their way
-    // to copy 0; then Y, the outgoing partial rows of this CTA as they lie in the workspace.
-    // kPair: a warpgroup that is done has seen the last S land, so the query tile under merge_base is free.
-    // kDual: the other warpgroup may still have a tile to go, so the (m, l) get 2 KB of their own after the rings.
-    const uint32_t ml_base = kIsDual ? v_base + nv_slots * G::kSlotBytes : merge_base;   // [warpgroup][128 lanes] (m, l)
-    const uint32_t z_base = merge_base + 2048u;                                // kDual: [64 rows][RP floats]
-    const uint32_t y_base = z_base + (kIsDual ? 64u * RB : 0u);                // [rows_cap][RP floats]
+    // a finished warpgroup writes: it has seen the last S land, so the query tile under merge_base is free);
+    // then Y, the outgoing partial rows of this CTA as they lie in the workspace.
+    const uint32_t ml_base = merge_base;                                       // [warpgroup][128 lanes] (m, l)
+    const uint32_t y_base = merge_base + 2048u;                                // [rows_cap][RP floats]
     if (warp >= 4) {
-        // What is written below (except the (m, l)) overlaps the query tile, P and the K/V slots: the query copy
+        // What is written below (except the (m, l)) overlaps the query tile and the K/V slots: the query copy
         // must have landed and every MMA of the CTA must be complete (each warpgroup has seen its last P V land).
         mbar_wait_warp(smem_u32(&c.q_full), 0, abort_flag, a.status);
         const bool any_valid = __any_sync(0xffffffffu, ri.valid);
@@ -1228,8 +1134,8 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
         const float w_me = m_run != -INFINITY ? exp2f(m_run - m_out) : 0.f;      // 0: saw no visible key
         const float w_ot = other.x != -INFINITY ? exp2f(other.x - m_out) : 0.f;
         float l_out = w_me * l_run + w_ot * other.y;
-        // an accumulator that no MMA has written holds anything: it is not read (kDual: warpgroup w has tiles w, w+2, ..)
-        const bool has_ot = kIsDual ? sp.n_tiles > (wg ^ 1) : has_acc;
+        // an accumulator that no MMA has written holds anything: it is not read
+        const bool has_ot = has_acc;
         const uint32_t o_other = tmem + lane_base + (wg ^ 1) * G::kOCols;
         const int c_lo = wg == 0 ? 0 : G::kSplitCol, c_hi = wg == 0 ? G::kSplitCol : HD;
         float v[G::kSplitCol];                                                   // this thread's columns of the lane's combined partial
@@ -1247,38 +1153,8 @@ __global__ void __launch_bounds__(Geo<HD, MODE>::kThreads, 1) msa_attention_kern
             #pragma unroll
             for (int i = 0; i < 16; ++i) v[cc + i] = w_me * __uint_as_float(mine[i]) + w_ot * __uint_as_float(theirs[i]);
         }
-        if (kIsDual) {
-            // the lane's partial covers the keys of its copy; copy 1 hands its rows to copy 0 through Z
-            const uint32_t zrow = z_base + static_cast<uint32_t>(lrow) * RB;
-            if (copy == 1) {
-                #pragma unroll
-                for (int cc = 0; cc < G::kSplitCol; cc += 4)
-                    if (c_lo + cc < c_hi)
-                        st_shared_v4(zrow + (c_lo + cc) * 4u, __float_as_uint(v[cc]), __float_as_uint(v[cc + 1]), __float_as_uint(v[cc + 2]),
-                                     __float_as_uint(v[cc + 3]));
-                if (wg == 0) st_shared_v4(zrow + HD * 4u, __float_as_uint(m_out), __float_as_uint(l_out), 0u, 0u);
-            }
-            if (tid == kAuxThreads) SS_TR(5, 2);
-            named_barrier(1, wg_threads);
-            if (copy == 0) {
-                const float2 z = ld_shared_v2(zrow + HD * 4u);
-                const float m_f = fmaxf(m_out, z.x);
-                const float w_a = m_out != -INFINITY ? exp2f(m_out - m_f) : 0.f;
-                const float w_b = z.x != -INFINITY ? exp2f(z.x - m_f) : 0.f;
-                l_out = w_a * l_out + w_b * z.y;
-                m_out = m_f;
-                #pragma unroll
-                for (int cc = 0; cc < G::kSplitCol; cc += 4) {
-                    if (c_lo + cc < c_hi) {
-                        const float4 t = ld_shared_v4(zrow + (c_lo + cc) * 4u);
-                        v[cc] = w_a * v[cc] + w_b * t.x; v[cc + 1] = w_a * v[cc + 1] + w_b * t.y;
-                        v[cc + 2] = w_a * v[cc + 2] + w_b * t.z; v[cc + 3] = w_a * v[cc + 3] + w_b * t.w;
-                    }
-                }
-            }
-        }
-        // the thread now holds its columns of the row's partial over all keys of this CTA (kDual: copy 0 only)
-        if (!kIsDual || copy == 0) {
+        // the thread now holds its columns of the row's partial over all keys of this CTA
+        {
             if (C == 1) {
                 if (ri.valid && !skip) {
                     const OutPtr dst = out_ptr<HD>(a, b, h, spec_row0, ri);
@@ -1420,43 +1296,41 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
         plan->partial_bytes = c > 1 ? static_cast<size_t>(plan->groups) * c * kSmRows * (p.head_dim + 4) * 4 : 0;
         return true;
     }
-    const size_t p_total = plan->mode == kDual ? static_cast<size_t>(2) * 3 * 64 * 128 : 0;      // kPair keeps P in TMEM
-    const size_t qp = static_cast<size_t>(halves) * kBlockRows * 128 + p_total;
+    // row blocks: the query tile, then the K ring and the V ring (P lives in TMEM)
+    const size_t qp = static_cast<size_t>(halves) * kBlockRows * 128;
     const size_t slot = static_cast<size_t>(halves) * kTileKeys * 128;
-    const size_t ml_own = plan->mode == kDual ? 2048 : 0;    // kDual: the warpgroups' (m, l) exchange is not aliased
-    int slots = static_cast<int>((kMaxDynSmem - 1024 - ml_own - qp) / slot);
+    int slots = static_cast<int>((kMaxDynSmem - 1024 - qp) / slot);
     if (slots > 2 * kMaxSlots) slots = 2 * kMaxSlots;
     if (slots < 4) return false;
     // a K slot is held until S is queued, a V slot until P V has completed: the odd slot goes to V
     plan->n_kslots = slots / 2;
     plan->n_vslots = slots - plan->n_kslots > kMaxSlots ? kMaxSlots : slots - plan->n_kslots;
-    size_t bytes = qp + static_cast<size_t>(plan->n_kslots + plan->n_vslots) * slot + ml_own;
-    // after the pipeline the same memory stages partial rows ((head_dim + 4) floats each): 2 KB, then kDual 64
-    // rows in transit between the copies and 64 outgoing rows, kPair 128 outgoing rows
+    size_t bytes = qp + static_cast<size_t>(plan->n_kslots + plan->n_vslots) * slot;
+    // after the pipeline the same memory stages partial rows ((head_dim + 4) floats each): 2 KB, then the 128
+    // outgoing rows
     const size_t row_bytes = static_cast<size_t>(p.head_dim + 4) * 4;
-    const size_t stage = 2048 + (plan->mode == kDual ? 2 * 64 : kBlockRows) * row_bytes;
+    const size_t stage = 2048 + kBlockRows * row_bytes;
     if (stage > bytes) bytes = stage;
     plan->smem = bytes + 1024;
     // workspace: one partial row per (group, CTA of the group, row)
-    const size_t rows_cap = plan->mode == kDual ? 64 : kBlockRows;
-    plan->partial_bytes = c > 1 ? static_cast<size_t>(plan->groups) * c * rows_cap * row_bytes : 0;
+    plan->partial_bytes = c > 1 ? static_cast<size_t>(plan->groups) * c * kBlockRows * row_bytes : 0;
     return plan->smem <= static_cast<size_t>(kMaxDynSmem);
 }
 
-template <int HD, int MODE>
+template <int HD>
 static int32_t launch(const AttnArgs& args, const AttnPlan& plan, cudaStream_t stream) {
     static bool configured[64] = {false};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return SS_ERR_CUDA;
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        if (cudaFuncSetAttribute(msa_attention_kernel<HD, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem) !=
+        if (cudaFuncSetAttribute(msa_attention_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem) !=
             cudaSuccess)
             return SS_ERR_CUDA;
         configured[dev] = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(plan.groups * plan.cluster), 1, 1);
-    cfg.blockDim = dim3(static_cast<unsigned>(Geo<HD, MODE>::kThreads), 1, 1);
+    cfg.blockDim = dim3(static_cast<unsigned>(Geo<HD>::kThreads), 1, 1);
     // always more than half of an SM's shared memory: one CTA per SM, so a CTA never queues for TMEM
     cfg.dynamicSmemBytes = plan.smem < 120 * 1024 ? 120 * 1024 : plan.smem;
     cfg.stream = stream;
@@ -1467,7 +1341,7 @@ static int32_t launch(const AttnArgs& args, const AttnPlan& plan, cudaStream_t s
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, msa_attention_kernel<HD, MODE>, args) == cudaSuccess ? SS_OK : SS_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, msa_attention_kernel<HD>, args) == cudaSuccess ? SS_OK : SS_ERR_CUDA;
 }
 
 template <int HD>
@@ -1574,9 +1448,9 @@ extern "C" int32_t ss_msa_attention(const ss_attn_params* p, void* stream) {
         }
     }
     switch (d) {
-        case 64: return ss::launch<64, ss::kPair>(a, plan, s);
-        case 80: return ss::launch<80, ss::kPair>(a, plan, s);
-        default: return ss::launch<128, ss::kPair>(a, plan, s);
+        case 64: return ss::launch<64>(a, plan, s);
+        case 80: return ss::launch<80>(a, plan, s);
+        default: return ss::launch<128>(a, plan, s);
     }
 }
 
