@@ -475,10 +475,10 @@ def run_profile(args, st):
 
 def ncu_traffic():
     """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if present."""
-    path = os.path.join(ROOT, "profiles", "msa_attention_kernel_7b_traffic.txt")
+    path = os.path.join(ROOT, "profiles", "msa_attention_7b_traffic.txt")
     if os.path.exists(path):
         with open(path) as fh:
-            return json.load(fh).get("msa_attention_kernel_dram_bytes_per_launch")
+            return json.load(fh).get("msa_attention_dram_bytes_per_launch")
     return None
 
 
