@@ -358,3 +358,39 @@ def test_compaction_long_path_and_aliased_lengths(cuda, oracle):
     lens = _compact_and_compare(api, dev, st, oracle, host)
     assert list(lens) == [33, 33]
     assert list(dev.accept_path[0, :4].cpu().numpy()) == [0, 1, 3, 5]
+
+
+def test_two_steps_in_a_row_with_aliased_lengths(cuda, oracle):
+    """A second step on the cache that the first step's compaction left behind: the lengths are updated in
+    place (kv_len_out aliases kv_len), the accepted nodes have become prefix, new tree nodes are appended
+    after them.  The first attention call after a compaction may not promise a stable prefix, so the step
+    runs with flags = 0; its attention must match the oracle on the compacted cache and the new lengths."""
+    api, DeviceStep = cuda
+    cfg = W.custom_config("twostep", batch=2, n_layers=2, n_msa_layers=1, prefix_len=37, n_nodes=10, gamma=2,
+                          max_depth=3, vocab=97, p_accept=0.9, n_heads=3, head_dim=64, config_id=730)
+    st = W.make_step(cfg)
+    dev = DeviceStep(st, prefix_stable=False)
+    host = [st.layer(l) for l in dev.layers]
+    dev.kv_len_out = dev.kv_len                                  # the compaction updates the lengths in place
+    dev.run_attention()
+    lens = _compact_and_compare(api, dev, st, oracle, host)
+    assert api.ss_status(dev.attn_ws) == 0
+    k_now = api.bf16_to_host_bits(dev.k_all)
+    v_now = api.bf16_to_host_bits(dev.v_all)
+    rng = np.random.default_rng(731)
+    T, H, d = cfg.n_nodes, cfg.n_heads, cfg.head_dim
+    for b in range(cfg.batch):
+        s0, cap = int(st.kv_start[b]), int(st.kv_capacity[b])
+        L2 = int(st.kv_len[b]) + int(lens[b])
+        assert L2 + T <= cap
+        for arr, dev_arr in ((k_now, dev.k_all), (v_now, dev.v_all)):         # this step's tree nodes, after the new prefix
+            rows = W.f32_to_bf16_bits(rng.standard_normal((len(dev.layers), T, H, d)).astype(np.float32))
+            arr[:, s0 + L2:s0 + L2 + T] = rows
+            dev_arr[:, s0 + L2:s0 + L2 + T].copy_(api.bf16_to_device(rows))
+        st.kv_len[b] = L2
+    assert list(dev.kv_len.cpu().numpy()) == list(st.kv_len)
+    dev.run_attention()
+    assert api.ss_status(dev.attn_ws) == 0
+    for i, ly in enumerate(host):
+        now = W.LayerInputs(ly.layer, ly.is_msa, ly.q_main, ly.q_spec, ly.k_spec, ly.v_spec, k_now[i], v_now[i])
+        assert_attention_close(oracle, st, now, dev, i)
