@@ -17,10 +17,12 @@
 // Softmax with a shared reference.  The four threads of a lane exponentiate against one reference m_ref (any
 // value at or above the lane's scores, and not absurdly far above, gives the same result after
 // normalisation): the lane's maximum over the first tile.  A later score that exceeds it by more than 2^8
-// raises it: the copy's softmax threads agree on that through one reducing barrier per tile, exchange their
-// maxima through shared memory, rescale the lane's accumulator and their row sums, and redo the tile's P.
+// raises it: the copy's softmax threads agree on that through one reducing barrier per tile (each votes on the
+// sum of its 32 exponentials), exchange their maxima through shared memory, rescale the lane's accumulator and
+// their row sums, and redo the tile's P.
 //
-// Roles (640 threads): warp 0 lane 0 requests tiles (TMA) into one ring, K and V tiles alternating; warp 1
+// Roles (640 threads): warp 0 lane 0 requests the query tile and the K tiles (TMA), warp 3 lane 0 the V tiles,
+// into rings of their own (a K slot is free again after S, a V slot only after P V, so K runs ahead); warp 1
 // lane 0 issues S and hands K slots back; warp 2 lane 0 issues P V and hands V slots back; warps 4..19 are the
 // softmax threads, four to a TMEM lane.
 //
