@@ -149,6 +149,37 @@ __device__ Stats chunk_stats(const float* row, int vocab, int chunk) {
     return r;
 }
 
+// The k best of n_cand chunk candidates (kMaxTopK per chunk, the first k of each meaningful), by one warp: the lanes
+// share the candidates (four each in registers, more are read again in every round) and k rounds of a warp
+// maximum pick them in order (candidates are unique: the next best is the largest one below the last).
+// Every lane gets top[0 .. k).
+__device__ __forceinline__ void warp_topk(const unsigned long long* cand, int n_cand, int k, unsigned long long (&top)[kMaxTopK]) {
+    const int lane = threadIdx.x & 31;
+    unsigned long long mine[4];
+    #pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const int j = lane + 32 * q;
+        mine[q] = (j < n_cand && (j % kMaxTopK) < k) ? __ldcg(cand + j) : 0ull;
+    }
+    unsigned long long below = ~0ull;
+    #pragma unroll
+    for (int r = 0; r < kMaxTopK; ++r) top[r] = 0ull;
+    for (int q = 0; q < k; ++q) {
+        unsigned long long m = 0ull;
+        #pragma unroll
+        for (int r = 0; r < 4; ++r)
+            if (mine[r] < below && mine[r] > m) m = mine[r];
+        for (int j = lane + 128; j < n_cand; j += 32) {
+            const unsigned long long e = (j % kMaxTopK) < k ? __ldcg(cand + j) : 0ull;
+            if (e < below && e > m) m = e;
+        }
+        m = warp_max_u64(m);
+        #pragma unroll
+        for (int r = 0; r < kMaxTopK; ++r) top[r] = (r == q) ? m : top[r];
+        below = m;
+    }
+}
+
 // the last CTA of a sequence to get here returns true (its threads then see every other CTA's partials)
 __device__ bool arrive_last(int32_t* counter, int expected) {
     __shared__ bool s_last;
@@ -200,19 +231,11 @@ next_draft_kernel(const float* __restrict__ stream_logits, int n_rows, const int
     __shared__ int32_t s_top[SS_MAX_GAMMA][kMaxTopK];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (warp < gamma) {                                   // one warp per stream: k rounds over its chunks' candidates
-        const unsigned long long* cand = partials + (static_cast<size_t>(b) * gamma + warp) * n_chunks * kMaxTopK;
-        const int n = n_chunks * kMaxTopK;
-        unsigned long long taken_below = ~0ull;           // candidates are unique: the next best is the largest one below the last
-        for (int q = 0; q < k; ++q) {
-            unsigned long long m = 0ull;
-            for (int i = lane; i < n; i += 32) {
-                const unsigned long long e = (i % kMaxTopK) < k ? __ldcg(cand + i) : 0ull;
-                if (e < taken_below && e > m) m = e;
-            }
-            m = warp_max_u64(m);
-            if (lane == 0) s_top[warp][q] = entry_index(m);
-            taken_below = m;
-        }
+        unsigned long long top[kMaxTopK];
+        warp_topk(partials + (static_cast<size_t>(b) * gamma + warp) * n_chunks * kMaxTopK, n_chunks * kMaxTopK, k, top);
+        #pragma unroll
+        for (int q = 0; q < kMaxTopK; ++q)
+            if (lane == 0 && q < k) s_top[warp][q] = entry_index(top[q]);
     }
     __syncthreads();
     // node i of the full k-ary tree: level g (1-based), offset o within the level; parent = level(g-1) start + o / k
@@ -268,6 +291,53 @@ struct NodeTailArgs {
     int32_t *accept_len, *accept_path, *last_node, *bonus_token;   // mode 1
 };
 
+// Pruning, after the edges are judged: a node survives when every edge of its root path is ok; survivors keep
+// their order.  One thread sweeps the nodes (parent[c] < c) over shared-memory copies; all threads write the
+// results out.  Called by every thread of the CTA.
+__device__ void prune_tail(int T, int max_nodes, int b, unsigned long long ok, const int32_t* s_parent, const int32_t* s_depth,
+                           const int32_t* s_tok, int gamma, const NodeTailArgs& ta) {
+    __shared__ int32_t s_new[SS_MAX_NODES], s_kept[SS_MAX_NODES], s_np[SS_MAX_NODES];
+    __shared__ unsigned long long s_anc[SS_MAX_NODES];
+    __shared__ int s_n, s_md;
+    const int i = threadIdx.x;
+    if (i == 0) {
+        unsigned long long keep = T > 0 ? 1ull : 0ull;
+        int n = 0, md = 0;
+        for (int c = 0; c < T; ++c) {
+            const bool kp = c == 0 || (((keep >> s_parent[c]) & 1ull) && ((ok >> c) & 1ull));
+            if (kp) {
+                keep |= 1ull << c;
+                const int np = c == 0 ? -1 : s_new[s_parent[c]];
+                s_new[c] = n;
+                s_kept[n] = c;
+                s_np[n] = np;
+                s_anc[n] = (np >= 0 ? s_anc[np] : 0ull) | (1ull << n);
+                md = max(md, s_depth[c]);
+                ++n;
+            } else {
+                s_new[c] = -1;
+            }
+        }
+        s_n = n; s_md = md;
+    }
+    __syncthreads();
+    const int n = s_n;
+    ss_tree_desc* out = ta.pruned_trees + b;
+    if (i < max_nodes) ta.new_index[static_cast<size_t>(b) * max_nodes + i] = i < T ? s_new[i] : -1;
+    if (i < SS_MAX_NODES) {
+        const bool live = i < n;
+        const int c = live ? s_kept[i] : 0;
+        out->parent[i] = live ? s_np[i] : -1;
+        out->depth[i] = live ? s_depth[c] : 0;
+        out->anc_mask[i] = live ? s_anc[i] : 0ull;
+        if (i < max_nodes) {
+            ta.kept_nodes[static_cast<size_t>(b) * max_nodes + i] = live ? c : -1;
+            ta.kept_tokens[static_cast<size_t>(b) * max_nodes + i] = live ? s_tok[c] : -1;
+        }
+    }
+    if (i == 0) { out->n_nodes = n; out->gamma = gamma; out->max_depth = s_md; out->reserved = 0; }
+}
+
 __global__ void __launch_bounds__(kScanThreads)
 node_stats_kernel(const float* __restrict__ logits, const int32_t* __restrict__ tokens, const ss_tree_desc* __restrict__ trees,
                   int max_nodes, int vocab, int n_chunks, NodeTailArgs ta, int32_t* __restrict__ counters, Stats* __restrict__ partials) {
@@ -289,10 +359,16 @@ node_stats_kernel(const float* __restrict__ logits, const int32_t* __restrict__ 
         const Stats* p = partials + (static_cast<size_t>(b) * max_nodes + i) * n_chunks;
         Stats s;
         s.best = 0ull; s.z = 0.f; s.w = 0.f;
-        for (int q = 0; q < n_chunks; ++q) {
-            Stats o;
-            o.best = __ldcg(&p[q].best); o.z = __ldcg(&p[q].z); o.w = __ldcg(&p[q].w);
-            s = merge_stats(s, o);
+        for (int q0 = 0; q0 < n_chunks; q0 += 8) {          // eight partials' loads in flight at once, merged in order
+            Stats o[8];
+            #pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                o[q].best = 0ull; o[q].z = 0.f; o[q].w = 0.f;
+                if (q0 + q < n_chunks) { o[q].best = __ldcg(&p[q0 + q].best); o[q].z = __ldcg(&p[q0 + q].z); o[q].w = __ldcg(&p[q0 + q].w); }
+            }
+            #pragma unroll
+            for (int q = 0; q < 8; ++q)
+                if (q0 + q < n_chunks) s = merge_stats(s, o[q]);
         }
         const float logz = logf(s.z);
         s_lse[i] = entry_value(s.best) + logz;
@@ -318,44 +394,17 @@ node_stats_kernel(const float* __restrict__ logits, const int32_t* __restrict__ 
         if (ok && i > 0) atomicOr(&s_ok, 1ull << i);
     }
     __syncthreads();
-    if (i != 0) return;
     const unsigned long long ok = s_ok;
     if (ta.mode == 1) {
+        if (i != 0) return;
         int best = 0, len = 1;
         accept_walk(T, s_parent, s_depth, ok, ta.accept_path + static_cast<size_t>(b) * SS_PATH_STRIDE, &best, &len);
         ta.accept_len[b] = len;
         ta.last_node[b] = best;
         ta.bonus_token[b] = s_am[best];
     } else {
-        // a node survives when every edge of its root path is ok; survivors keep their order
-        unsigned long long keep = T > 0 ? 1ull : 0ull;
-        int n = 0;
-        ss_tree_desc* out = ta.pruned_trees + b;
-        int32_t* new_index = ta.new_index + static_cast<size_t>(b) * max_nodes;
-        int md = 0;
-        for (int c = 0; c < T; ++c) {
-            const bool kp = c == 0 || (((keep >> s_parent[c]) & 1ull) && ((ok >> c) & 1ull));
-            if (kp) {
-                keep |= 1ull << c;
-                const int np = c == 0 ? -1 : new_index[s_parent[c]];
-                new_index[c] = n;
-                ta.kept_nodes[static_cast<size_t>(b) * max_nodes + n] = c;
-                ta.kept_tokens[static_cast<size_t>(b) * max_nodes + n] = s_tok[c];
-                out->parent[n] = np;
-                out->depth[n] = s_depth[c];
-                out->anc_mask[n] = (np >= 0 ? out->anc_mask[np] : 0ull) | (1ull << n);
-                md = max(md, s_depth[c]);
-                ++n;
-            } else {
-                new_index[c] = -1;
-            }
-        }
-        for (int c = T; c < max_nodes; ++c) new_index[c] = -1;
-        for (int q = n; q < SS_MAX_NODES; ++q) {
-            out->parent[q] = -1; out->depth[q] = 0; out->anc_mask[q] = 0ull;
-            if (q < max_nodes) { ta.kept_nodes[static_cast<size_t>(b) * max_nodes + q] = -1; ta.kept_tokens[static_cast<size_t>(b) * max_nodes + q] = -1; }
-        }
-        out->n_nodes = n; out->gamma = trees[b].gamma; out->max_depth = md; out->reserved = 0;
+        prune_tail(T, max_nodes, b, ok, s_parent, s_depth, s_tok, trees[b].gamma, ta);
+        if (i != 0) return;
     }
     counters[b] = 0;
 }
@@ -378,20 +427,12 @@ sampled_verify_kernel(const float* __restrict__ logits, const int32_t* __restric
 
     __shared__ int32_t s_draw[SS_MAX_NODES], s_parent[SS_MAX_NODES], s_depth[SS_MAX_NODES], s_tok[SS_MAX_NODES];
     const int i = threadIdx.x;
-    if (i < T) {
-        const unsigned long long* cand = partials + (static_cast<size_t>(b) * max_nodes + i) * n_chunks * kMaxTopK;
+    // a warp per node picks the node's k best; its lane 0 draws the token
+    const int lane = i & 31, n_cand = n_chunks * kMaxTopK;
+    for (int node = i >> 5; node < T; node += kScanThreads / 32) {                     // warp-uniform
         unsigned long long top[kMaxTopK];
-        unsigned long long below = ~0ull;
-        for (int q = 0; q < k; ++q) {                     // the k best of the node, in order
-            unsigned long long m = 0ull;
-            for (int j = 0; j < n_chunks * kMaxTopK; ++j) {
-                const unsigned long long e = (j % kMaxTopK) < k ? __ldcg(cand + j) : 0ull;
-                if (e < below && e > m) m = e;
-            }
-            #pragma unroll
-            for (int r = 0; r < kMaxTopK; ++r) top[r] = (r == q) ? m : top[r];
-            below = m;
-        }
+        warp_topk(partials + (static_cast<size_t>(b) * max_nodes + node) * n_chunks * kMaxTopK, n_cand, k, top);
+        if (lane != 0) continue;
         float x0 = 0.f, z = 0.f, ex[kMaxTopK];
         #pragma unroll
         for (int r = 0; r < kMaxTopK; ++r) {
@@ -399,7 +440,7 @@ sampled_verify_kernel(const float* __restrict__ logits, const int32_t* __restric
             ex[r] = r < k ? expf(entry_value(top[r]) - x0) : 0.f;
             z += ex[r];
         }
-        const float u = uniforms[static_cast<size_t>(b) * max_nodes + i];
+        const float u = uniforms[static_cast<size_t>(b) * max_nodes + node];
         float cdf = 0.f;
         int pick = k - 1;
         bool found = false;
@@ -413,8 +454,10 @@ sampled_verify_kernel(const float* __restrict__ logits, const int32_t* __restric
         unsigned long long e = 0ull;
         #pragma unroll
         for (int r = 0; r < kMaxTopK; ++r) e = (r == pick) ? top[r] : e;
-        s_draw[i] = entry_index(e);
-        if (node_token) node_token[static_cast<size_t>(b) * max_nodes + i] = s_draw[i];
+        s_draw[node] = entry_index(e);
+        if (node_token) node_token[static_cast<size_t>(b) * max_nodes + node] = s_draw[node];
+    }
+    if (i < T) {
         s_parent[i] = trees[b].parent[i];
         s_depth[i] = trees[b].depth[i];
         s_tok[i] = tokens[static_cast<size_t>(b) * max_nodes + i];

@@ -91,11 +91,18 @@ tree_verify_kernel(const float* __restrict__ logits, const int32_t* __restrict__
         const Cand* p = partials + (static_cast<size_t>(b) * max_nodes + threadIdx.x) * n_chunks;
         float bv = -INFINITY;
         int32_t bi = 0x7fffffff;
-        for (int k = 0; k < n_chunks; ++k) {
-            const long long raw = __ldcg(reinterpret_cast<const long long*>(p + k));
-            const float v = __int_as_float(static_cast<int>(raw & 0xffffffffll));
-            const int32_t i = static_cast<int32_t>(raw >> 32);
-            if (better(v, i, bv, bi)) { bv = v; bi = i; }
+        for (int k0 = 0; k0 < n_chunks; k0 += 8) {             // eight candidates' loads in flight at once
+            long long raw[8];
+            #pragma unroll
+            for (int k = 0; k < 8; ++k) raw[k] = k0 + k < n_chunks ? __ldcg(reinterpret_cast<const long long*>(p + k0 + k)) : 0ll;
+            #pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                if (k0 + k < n_chunks) {
+                    const float v = __int_as_float(static_cast<int>(raw[k] & 0xffffffffll));
+                    const int32_t i = static_cast<int32_t>(raw[k] >> 32);
+                    if (better(v, i, bv, bi)) { bv = v; bi = i; }
+                }
+            }
         }
         // a row without any comparable value (all NaN) reports index 0, like a strict '>' scan
         if (bi == 0x7fffffff) bi = 0;
