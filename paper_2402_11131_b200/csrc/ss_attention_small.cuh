@@ -74,7 +74,12 @@ struct CtrlS {
     unsigned long long s_full[2];              // S of a tile complete
     unsigned long long s_free[2];              // its scores are in registers (the copy's 8 warps): the copy's score buffer is free
     unsigned long long p_full[2];              // P of a tile written to the copy's P buffer (8 warps)
-    unsigned long long pv_done[2];             // P V of a tile complete: the copy's P buffer is free
+    // P V of tile t complete, on barrier t mod 4 (its phase is t / 4): a waiter derives the parity from t and never
+    // counts phases.  Whoever waits for tile t does so before it publishes a P that tile t + 4 depends on, and
+    // after it has seen a tile later than t - 4 complete (MMAs complete in issue order), so the barrier is
+    // neither two phases ahead of the wait nor behind it.  With one barrier per copy a copy could find the other
+    // copy's barrier two phases ahead (tiles j - 3 and j - 1 both complete), and its parity wait then never ends.
+    unsigned long long pv_done[4];
     unsigned long long anc[SS_MAX_NODES];
     alignas(16) float xch[4][2 * kSmRows];     // exchange between the four threads of a lane (maxima, row sums)
     uint32_t tmem_base;
@@ -192,8 +197,8 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
             mbar_init(smem_u32(&c.s_full[s]), 1);
             mbar_init(smem_u32(&c.s_free[s]), 8);
             mbar_init(smem_u32(&c.p_full[s]), 8);
-            mbar_init(smem_u32(&c.pv_done[s]), 1);
         }
+        for (int s = 0; s < 4; ++s) mbar_init(smem_u32(&c.pv_done[s]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     auto dependency_wait = [&]() {
@@ -240,16 +245,22 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
             else tma_load_3d(dst + hh * G::kBoxBytes, is_v ? &a.tm_vs : &a.tm_ks, hh * 64, h, static_cast<int>(spec_row0 + x), bar);
         }
     };
-    // The first two tiles are requested right away, K0 V0 K1 V1 (before the dependency wait, under the caller's
-    // promise); the rest follows once the query rows have arrived, which would otherwise queue behind the
-    // tiles on their way into this SM
+    // The K tiles of the first two tiles are requested right away (before the dependency wait, under the caller's
+    // promise): S of a tile needs only K and Q.  After the wait come the query rows, then the V tiles of those two
+    // tiles (a CTA that starts late passes the wait at once, and its query rows then queue behind two K tiles
+    // instead of four tiles); the rest follows once the query rows have arrived
     const int n_early = min(sp.n_tiles, min(n_ring, 2));
+#ifdef SS_K3
+    const int n_early_k = min(sp.n_tiles, n_ring);
+#else
+    const int n_early_k = n_early;
+#endif
     auto prefix_only = [&](int j) { return sp.is_cache(j) && sp.first_key(j) + TK <= sp.L; };
     int n_pre = 0;
     if (a.prefix_stable) {
         if (tid == 0) {
-            // the first tiles that lie wholly inside the cached prefix
-            while (n_pre < 2 * n_early && prefix_only(n_pre >> 1)) { load_tile(n_pre & 1, n_pre >> 1, n_pre >> 1); ++n_pre; }
+            // the K tiles that lie wholly inside the cached prefix
+            while (n_pre < n_early && prefix_only(n_pre)) { load_tile(0, n_pre, n_pre); ++n_pre; }
         }
         dependency_wait();
     }
@@ -270,7 +281,8 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
                 if (with_spec) tma_load_3d(dst + a.tmax8 * 128u, &a.tm_qs, hh * 64, h, static_cast<int>(spec_row0), qbar);
             }
         }
-        for (int i = n_pre; i < 2 * n_early; ++i) load_tile(i & 1, i >> 1, i >> 1);
+        for (int j = n_pre; j < n_early_k; ++j) load_tile(0, j, j);
+        for (int j = 0; j < n_early; ++j) load_tile(1, j, j);
         SS_TRC(0, 5);
     }
     if (tid >= kAuxThreads && tid < kAuxThreads + SS_MAX_NODES) c.anc[tid - kAuxThreads] = __ldcg(&a.trees[b].anc_mask[tid - kAuxThreads]);
@@ -292,9 +304,10 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
     auto produce = [&](int kind) {
         Ring r;
         r.start();
-        for (int j = 0; j < n_early; ++j) r.advance(n_ring);
+        const int first = kind ? n_early : n_early_k;
+        for (int j = 0; j < first; ++j) r.advance(n_ring);
         bool ok = mbar_wait_s(smem_u32(&c.q_full), 0, &c, status);
-        int j = n_early;
+        int j = first;
         for (; ok && j < sp.n_tiles; ++j) {
             if (r.round > 0) ok = mbar_wait_s(smem_u32(&c.slot_empty[kind][r.slot]), (r.round - 1) & 1, &c, status);
             if (kind == 0) SS_TRC(0, 8 + j);
@@ -311,7 +324,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
 
     // =============================== warps 0 and 3: tile requests ================================
     if (warp == 0) {
-        if (lane == 0 && sp.n_tiles > n_early) produce(0);
+        if (lane == 0 && sp.n_tiles > n_early_k) produce(0);
     } else if (warp == 3) {
         if (lane == 0) {
             // the caller may shorten the bound of the device-side waits (workspace word 1, units of 1024 cycles)
@@ -372,7 +385,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
                 for (int ks = 0; ks < TK / 16; ++ks)
                     tc_mma_ts(tmem_o, tmem_p + buf * 64u + 8u * ks, dv + ((ks * 2048u) >> 4), idesc_bf16(HD, false, true),
                               (j > 0 || ks > 0) ? 1u : 0u);
-                tc_commit(smem_u32(&c.pv_done[buf]));
+                tc_commit(smem_u32(&c.pv_done[j & 3]));
                 tc_commit(smem_u32(&c.slot_empty[1][rv.slot]));
                 SS_TRC(2, 10 + 4 * j);
                 rv.advance(n_ring);
@@ -405,19 +418,13 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
         const bool leader = (tid == kAuxThreads) || (tid == kAuxThreads + 64);      // lane 0 of each copy's first warp
         const uint32_t p_addr = tmem_p + lane_base + static_cast<uint32_t>(copy * 64 + 16 * w4);   // my 32 keys of a tile as bf16
         const uint32_t o_addr = tmem_o + lane_base + 32u * w4;
-        int other_seen = 0;                                                    // phases of the other copy's completion barrier seen
+        auto wait_pv_tile = [&](int t) {                                       // P V of tile t complete
+            return mbar_wait_warp_s(smem_u32(&c.pv_done[t & 3]), static_cast<uint32_t>((t >> 2) & 1), &c, status);
+        };
         bool failed = false;
         // copy c takes the tiles j = c, c + 2, ..: all 128 keys of the tile for its 64 rows
         for (int j = copy; j < sp.n_tiles; j += 2) {
-            bool ok = true;
-            // every phase of both completion barriers is looked at, in order: a parity wait is then never more than
-            // one phase behind.  P V of tile j - 3 (the other copy's) completed before that of tile j - 2 (this
-            // copy's), which is awaited below before P is overwritten.
-            while (ok && j >= 3 && other_seen <= ((j - 3) >> 1)) {
-                ok = mbar_wait_warp_s(smem_u32(&c.pv_done[1 - copy]), other_seen & 1, &c, status);
-                ++other_seen;
-            }
-            ok = mbar_wait_warp_s(smem_u32(&c.s_full[copy]), (j >> 1) & 1, &c, status) && ok;
+            bool ok = mbar_wait_warp_s(smem_u32(&c.s_full[copy]), (j >> 1) & 1, &c, status);
             if (leader) SS_TRC(3, 8 + 6 * j);
             tc_fence_after();
             const int x0 = sp.first_key(j), nvk = sp.valid_keys(j);
@@ -454,10 +461,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
                 l_part *= corr;
                 bool ok2 = true;
                 if (j >= 2) {
-                    while (ok2 && other_seen <= ((j - 1) >> 1)) {
-                        ok2 = mbar_wait_warp_s(smem_u32(&c.pv_done[1 - copy]), other_seen & 1, &c, status);
-                        ++other_seen;
-                    }
+                    ok2 = wait_pv_tile(j - 1);
                     tc_fence_after();
                     if (ok2) {
                         uint32_t orr[32];
@@ -498,7 +502,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
                     unpack_f32x2(sum2, s0, s1);
                     lsum = s0 + s1;
                     // P of this copy's previous tile must have been read before it is overwritten
-                    if (attempt == 0 && j >= 2) ok = mbar_wait_warp_s(smem_u32(&c.pv_done[copy]), ((j - 2) >> 1) & 1, &c, status);
+                    if (attempt == 0 && j >= 2) ok = wait_pv_tile(j - 2);
                     if (ok) tmem_st16<0>(p_addr, pk);
                 }
                 if (leader) SS_TRC(3, 9 + 6 * j + (attempt > 0 ? 3 : 0));
@@ -537,16 +541,9 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
             if (lane == 0) mbar_arrive(smem_u32(&c.p_full[copy]));
             if (leader) SS_TRC(3, 11 + 6 * j);
         }
-        // every P V must be complete before the accumulator is read: this copy's last one, and the other copy's
-        if (!failed) {
-            const int n_mine = sp.n_tiles > copy ? (sp.n_tiles - copy + 1) >> 1 : 0;
-            const int n_other = sp.n_tiles > 1 - copy ? (sp.n_tiles - (1 - copy) + 1) >> 1 : 0;
-            bool ok = true;
-            if (n_mine > 0) ok = mbar_wait_warp_s(smem_u32(&c.pv_done[copy]), (n_mine - 1) & 1, &c, status);
-            while (ok && other_seen < n_other) {
-                ok = mbar_wait_warp_s(smem_u32(&c.pv_done[1 - copy]), other_seen & 1, &c, status);
-                ++other_seen;
-            }
+        // every P V must be complete before the accumulator is read: they complete in issue order, so the last one
+        if (!failed && sp.n_tiles > 0) {
+            wait_pv_tile(sp.n_tiles - 1);
             tc_fence_after();
         }
     }

@@ -141,3 +141,38 @@ def test_a_wait_that_runs_out_reports_a_timeout_and_the_stream_stays_usable(cuda
     assert api.ss_status(dev.attn_ws) == 0
     assert_attention_close(oracle, st, st.layer(0), dev, 0)
     assert int(words[2:].abs().max()) == 0                     # a call leaves the partial rows' area zero again
+
+
+def test_no_wait_runs_out_over_many_replays(cuda):
+    """The attention kernels' roles meet on phase-parity barriers; a waiter that falls two phases behind one of
+    them would wait until its bound runs out (a one-second stall and SS_ERR_DEVICE_TIMEOUT).  Whether that can
+    happen depends on timing, so the plain and the multi-stream layers of the 7B-class shape are replayed
+    back to back a few thousand times, as graphs of their own and as the whole step, with the status word read
+    after every batch of replays."""
+    api, DeviceStep = cuda
+    st = W.make_step(W.CONFIGS["7b"])
+    dev = DeviceStep(st)
+    stream = torch.cuda.Stream()
+    nl = len(dev.layers)
+    plain = [i for i in range(nl) if not dev.is_msa[i]]
+    msa = [i for i in range(nl) if dev.is_msa[i]]
+
+    def capture(fn):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            fn(stream)
+            stream.synchronize()
+            with torch.cuda.graph(g, stream=stream):
+                fn(stream)
+        return g
+
+    graphs = [capture(dev.run_step), capture(dev.run_attention), capture(lambda s: dev.run_attention(s, only=plain)),
+              capture(lambda s: dev.run_attention(s, only=msa))]
+    words = dev.attn_ws.view(torch.int32)
+    for _ in range(40):
+        for g in graphs:
+            with torch.cuda.stream(stream):
+                for _ in range(20):
+                    g.replay()
+            stream.synchronize()
+            assert int(words[0]) == 0
