@@ -246,15 +246,11 @@ __global__ void __launch_bounds__(kSmThreads, 1) msa_attention_small_kernel(cons
         }
     };
     // The K tiles of the first two tiles are requested right away (before the dependency wait, under the caller's
-    // promise): S of a tile needs only K and Q.  After the wait come the query rows, then the V tiles of those two
-    // tiles (a CTA that starts late passes the wait at once, and its query rows then queue behind two K tiles
-    // instead of four tiles); the rest follows once the query rows have arrived
+    // promise): S of a tile needs only K and Q.  After the wait come the query rows, then the third K tile, then the
+    // V tiles of the first two tiles (a CTA that starts late passes the wait at once, and its query rows then queue
+    // behind two K tiles instead of four tiles); the rest follows once the query rows have arrived
     const int n_early = min(sp.n_tiles, min(n_ring, 2));
-#ifdef SS_K3
-    const int n_early_k = min(sp.n_tiles, n_ring);
-#else
-    const int n_early_k = n_early;
-#endif
+    const int n_early_k = min(sp.n_tiles, n_ring);          // K tiles requested by thread 0: the ring's depth
     auto prefix_only = [&](int j) { return sp.is_cache(j) && sp.first_key(j) + TK <= sp.L; };
     int n_pre = 0;
     if (a.prefix_stable) {
