@@ -113,6 +113,10 @@ int32_t ss_tree_build(const int32_t* parent, int32_t n_nodes, int32_t gamma, ss_
  * stream and it is large enough for each.  Word 1 of the workspace, if positive, shortens the bound of the
  * device-side waits to that many units of 1024 cycles (default: about one second) for calls whose heads
  * have at most 64 query rows and for ss_wait_selftest; the library reads it and never writes it.
+ * Word 2 counts, over all calls since the caller last cleared it, the CTAs of unsplit 128-row blocks that
+ * started over: such a block first takes every row's exponentials against the maximum of the row's first
+ * 128 keys, and if a later tile exceeds that reference by more than about 2^57 it runs its tiles again
+ * with a running maximum (same result, about twice the time for that block).  Diagnostics only.
  * Precondition of a split (batch * n_heads * row blocks below the SM count): the CTAs that share a block's
  * keys wait for one another's partial rows at the end, so they must all be resident at once.  The call sizes the split from
  * the device's SM count; if other work holds SMs for the whole duration of the call (another stream, another

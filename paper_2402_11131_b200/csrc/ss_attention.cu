@@ -38,6 +38,7 @@
 // kernel is bounded and reports SS_ERR_DEVICE_TIMEOUT.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <type_traits>
 
 #include "ss_common.cuh"
 
@@ -70,7 +71,11 @@ constexpr int kBlockRows = 128;      // query rows per block (M of both MMAs)
 constexpr int kTileKeys = 128;       // keys per tile: N = 128 MMAs run at the full tensor rate
 constexpr int kMaxSlots = 4;         // slots per ring (K ring, V ring)
 constexpr int kAuxThreads = 128;     // warps 0..3: producers and MMA issuers
-constexpr int kMaxDynSmem = 232448 - 1024;  // 227 KB per CTA less the static control block
+constexpr int kPairMaxDynSmem = 232448 - 2048;   // 227 KB per CTA less the static control block (up to 2 KB) of msa_attention_kernel
+// Row blocks that are not split take the shared-reference pipeline: a row's exponentials are taken against the
+// maximum of its first tile for as long as a tile's 128 of them sum to at most 2^64 (no overflow anywhere: bf16
+// and fp32 reach 2^127); past that the CTA starts over with a running maximum per warpgroup.
+constexpr float kSharedRefLimit = 18446744073709551616.f;
 constexpr float kRescaleStep = 8.f;  // raise the running maximum only when it grows by more than 2^8
 constexpr long long kWaitCycles = 2000000000ll;   // bound of every mbarrier wait (~1 s)
 
@@ -114,9 +119,17 @@ struct Ctrl {
     // than one phase behind, which a parity wait needs
     unsigned long long o_done[2][2];
     unsigned long long anc[SS_MAX_NODES];
+    // shared-reference pipeline: the reference of each row (warpgroup 0 sets it from the first tile, one barrier per
+    // warp of 32 rows), and the barriers on which the MMA issuers wait for their last MMAs when the CTA starts over
+    unsigned long long mref_full[4], drain[2];
+    float m_ref[kBlockRows];
     uint32_t tmem_base;
-    int abort;
+    int abort;                                  // 1: a wait ran out of time; 2: the shared reference did not hold, start over
+#ifdef SS_TRACE
+    unsigned int trace_launch;
+#endif
 };
+static_assert(sizeof(Ctrl) + 16 <= 232448 - kPairMaxDynSmem, "control block and dynamic shared memory exceed an SM");
 
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -680,6 +693,27 @@ __device__ __forceinline__ void store_bf16x16(__nv_bfloat16* dst, const float (&
 }
 
 // ---------------------------------------------------------------------------------------------
+// The barriers that hand score buffers, P and accumulators around, for either pipeline of msa_attention_kernel.
+//   running maximum per warpgroup: s_full[w][b] S of buffer b complete (seen by warpgroup w); p_full[w][b] the
+//     warpgroup's half of P written (4 warps); s_free[b] the P V that read the buffer complete; o_done[w][b] the
+//     warpgroup's P V of a tile of parity b complete.
+//   shared reference (tile j: buffer b = j & 1, warpgroup b): s_full[0][b] S complete; s_free[b] the scores are in
+//     registers (4 warps); p_full[0][b] P written (4 warps); o_done[b][(j >> 1) & 1] P V of tile j complete.
+__device__ __forceinline__ void init_tile_barriers(Ctrl& c, bool shared_ref) {
+    for (int s = 0; s < 2; ++s) {
+        mbar_init(smem_u32(&c.s_free[s]), shared_ref ? 4 : 1);
+        mbar_init(smem_u32(&c.s_full[0][s]), 1);
+        mbar_init(smem_u32(&c.s_full[1][s]), 1);
+        mbar_init(smem_u32(&c.p_full[s][0]), 4);
+        mbar_init(smem_u32(&c.p_full[s][1]), 4);
+        mbar_init(smem_u32(&c.o_done[s][0]), 1);
+        mbar_init(smem_u32(&c.o_done[s][1]), 1);
+    }
+}
+__device__ __forceinline__ void mbar_inval(uint32_t bar) {
+    asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+
 template <int HD>
 __global__ void __launch_bounds__(Geo<HD>::kThreads, 1) msa_attention_kernel(const __grid_constant__ AttnArgs a) {
     using G = Geo<HD>;
@@ -697,10 +731,12 @@ __global__ void __launch_bounds__(Geo<HD>::kThreads, 1) msa_attention_kernel(con
     const int h = pair - b * a.n_heads;
     const int nk = a.n_kslots, nv_slots = a.n_vslots;
     volatile int* abort_flag = &c.abort;
+    // Row blocks that are not split start on the shared-reference pipeline (see kSharedRefLimit)
+    bool shared_ref = C == 1;
 
     if (tid == 0) SS_TR(0, 0);
 #ifdef SS_TRACE
-    __shared__ unsigned int s_launch;
+    unsigned int& s_launch = c.trace_launch;
     if (tid == 0) {
         const unsigned long long key = reinterpret_cast<unsigned long long>(a.o_main);
         s_launch = 0;
@@ -766,15 +802,9 @@ __global__ void __launch_bounds__(Geo<HD>::kThreads, 1) msa_attention_kernel(con
         if (a.gamma > 0) tma_prefetch_desc(&a.tm_vs);
     } else if (tid == 64) {                               // every other barrier (first used after the CTA-wide sync)
         for (int s = 0; s < kMaxSlots; ++s) { mbar_init(smem_u32(&c.k_empty[s]), 1); mbar_init(smem_u32(&c.v_empty[s]), 1); }
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(smem_u32(&c.s_free[s]), 1);                        // the P V commit
-            mbar_init(smem_u32(&c.s_full[0][s]), 1);
-            mbar_init(smem_u32(&c.s_full[1][s]), 1);
-            mbar_init(smem_u32(&c.p_full[s][0]), 4);                     // the warps of a warpgroup
-            mbar_init(smem_u32(&c.p_full[s][1]), 4);
-            mbar_init(smem_u32(&c.o_done[s][0]), 1);
-            mbar_init(smem_u32(&c.o_done[s][1]), 1);
-        }
+        init_tile_barriers(c, shared_ref);
+        for (int s = 0; s < 4; ++s) mbar_init(smem_u32(&c.mref_full[s]), 1);
+        for (int s = 0; s < 2; ++s) mbar_init(smem_u32(&c.drain[s]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (tid == 0) SS_TR(0, 1);
@@ -890,33 +920,40 @@ __global__ void __launch_bounds__(Geo<HD>::kThreads, 1) msa_attention_kernel(con
     RowInfo ri;
     ri.valid = false; ri.node = 0; ri.stream = 0;
 
+    // The tile loops of all roles, for either pipeline; early_k / early_v tiles have been requested already.
+    // n_requested: what a producer thread has requested in all (for the wait when the CTA starts over).
+    int n_requested = 0;
+    const uint32_t tmem_s1 = tmem + G::kOCols;            // shared reference: O, two S buffers, two P buffers of 64 columns
+    const uint32_t tmem_p1 = tmem_s1 + 2 * TK;
+    auto run_tiles = [&](auto mode_tag, const int early_k, const int early_v) {
+    constexpr bool kShared = decltype(mode_tag)::value;
     // ============================ warp 0: K producer, warp 3: V producer ==========================
     // Two rings, two threads: a K slot comes back as soon as S is queued, a V slot only after P V, and
     // neither request waits behind the other.
     if (warp == 0) {
-        if (lane == 0 && sp.n_tiles > n_early_k) {
+        if (lane == 0 && sp.n_tiles > early_k) {
             Ring rk;
             rk.start();
-            for (int i = 0; i < n_early_k; ++i) rk.advance(nk);
+            for (int i = 0; i < early_k; ++i) rk.advance(nk);
             bool ok = true;
-            for (int j = n_early_k; ok && j < sp.n_tiles; ++j) {
+            for (int j = early_k; ok && j < sp.n_tiles; ++j) {
                 ok = mbar_wait(smem_u32(&c.k_empty[rk.slot]), (rk.round - 1) & 1, abort_flag, a.status);
                 SS_TR(0, 8 + 2 * j);
-                if (ok) { load_k(j, rk.slot); rk.advance(nk); }
+                if (ok) { load_k(j, rk.slot); rk.advance(nk); n_requested = j + 1; }
             }
             // gave up: let the copies already in flight land before shared memory is reused or released
             if (!ok) for (int s = 0; s < nk; ++s) mbar_drain(smem_u32(&c.k_full[s]), (s < rk.slot ? rk.round : rk.round - 1) & 1);
         }
     } else if (warp == 3) {
-        if (lane == 0 && sp.n_tiles > n_early_v) {
+        if (lane == 0 && sp.n_tiles > early_v) {
             Ring rv;
             rv.start();
-            for (int i = 0; i < n_early_v; ++i) rv.advance(nv_slots);
+            for (int i = 0; i < early_v; ++i) rv.advance(nv_slots);
             bool ok = true;
-            for (int j = n_early_v; ok && j < sp.n_tiles; ++j) {
+            for (int j = early_v; ok && j < sp.n_tiles; ++j) {
                 ok = mbar_wait(smem_u32(&c.v_empty[rv.slot]), (rv.round - 1) & 1, abort_flag, a.status);
                 SS_TR(0, 9 + 2 * j);
-                if (ok) { load_v(j, rv.slot); rv.advance(nv_slots); }
+                if (ok) { load_v(j, rv.slot); rv.advance(nv_slots); n_requested = j + 1; }
             }
             if (!ok) for (int s = 0; s < nv_slots; ++s) mbar_drain(smem_u32(&c.v_full[s]), (s < rv.slot ? rv.round : rv.round - 1) & 1);
         }
@@ -942,14 +979,15 @@ __global__ void __launch_bounds__(Geo<HD>::kThreads, 1) msa_attention_kernel(con
                 SS_TR(1, 9 + 4 * j);
                 tc_fence_after();
                 const uint64_t dk = desc_k_major(k_base + rk.slot * G::kSlotBytes);
+                const uint32_t sd = (kShared ? tmem_s1 : tmem_s) + buf * TK;
                 #pragma unroll
                 for (int ks = 0; ks < G::kKSteps; ++ks) {
                     const uint32_t hh = ks >> 2, off = (ks & 3) * 32u;
-                    tc_mma(tmem_s + buf * TK, dq + ((hh * kQHalfBytes + off) >> 4), dk + ((hh * G::kBoxBytes + off) >> 4), G::kIdescS, ks > 0);
+                    tc_mma(sd, dq + ((hh * kQHalfBytes + off) >> 4), dk + ((hh * G::kBoxBytes + off) >> 4), G::kIdescS, ks > 0);
                 }
                 SS_TR(1, 10 + 4 * j);
                 tc_commit(smem_u32(&c.s_full[0][buf]));
-                tc_commit(smem_u32(&c.s_full[1][buf]));
+                if (!kShared) tc_commit(smem_u32(&c.s_full[1][buf]));
                 tc_commit(smem_u32(&c.k_empty[rk.slot]));                // S of tile j is queued: K may go
                 SS_TR(1, 11 + 4 * j);
             }
@@ -965,7 +1003,19 @@ __global__ void __launch_bounds__(Geo<HD>::kThreads, 1) msa_attention_kernel(con
                 if (!mbar_wait(smem_u32(&c.v_full[rv.slot]), rv.round & 1, abort_flag, a.status)) break;
                 SS_TR(2, 8 + 4 * j);
                 const uint32_t va = v_base + rv.slot * G::kSlotBytes;
-                {
+                if constexpr (kShared) {
+                    // the tile's 128 keys into the one accumulator; P is read from its own TMEM buffer
+                    const int buf = j & 1;
+                    const uint64_t dv = desc_mn_major(va, G::kBoxBytes);
+                    if (!mbar_wait(smem_u32(&c.p_full[0][buf]), (j >> 1) & 1, abort_flag, a.status)) break;
+                    SS_TR(2, 9 + 4 * j);
+                    tc_fence_after();
+                    const uint32_t pa = tmem_p1 + buf * (TK / 2);
+                    #pragma unroll
+                    for (int ks = 0; ks < TK / 16; ++ks)
+                        tc_mma_ts(tmem, pa + ks * 8u, dv + ((ks * 2048u) >> 4), G::kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
+                    tc_commit(smem_u32(&c.o_done[buf][(j >> 1) & 1]));   // P of the buffer may be overwritten
+                } else {
                     // keys 64w .. 64w+63 into the accumulator of warpgroup w; P is read from TMEM, where the
                     // warpgroup left it over the first 32 columns of its half of the S buffer
                     const int buf = j & 1;
@@ -996,10 +1046,121 @@ __global__ void __launch_bounds__(Geo<HD>::kThreads, 1) msa_attention_kernel(con
         const unsigned long long anc = ri.valid ? c.anc[ri.node] : 0ull;
         // a warp whose 32 rows are all padding skips the arithmetic but keeps the barrier protocol
         const bool warp_active = __any_sync(0xffffffffu, ri.valid);
-        const uint32_t o_addr = tmem + lane_base + wg * G::kOCols;
         Ring rv;                                       // V ring position of tile j
         rv.start();
         int v_tile = 0;
+        // V rows past the end of the sequence's keys may hold anything (even NaN patterns): P is 0 there, but
+        // 0 * NaN is NaN, so the rows [lo, hi) of tile j that lie past the end are cleared before P V reads them.
+        // Rows that only lie past this CTA's share of the keys are real data.  (false: a wait gave up)
+        auto clear_v_tail = [&](int j, int lo, int hi) {
+            const int region_left = (sp.is_cache(j) ? sp.L + sp.T : sp.n_stream) - sp.first_key(j);      // real rows in the tile
+            const int fix_lo = max(region_left, lo), fix_hi = hi;
+            if (fix_lo >= fix_hi) return true;
+            if (!mbar_wait_warp(smem_u32(&c.v_full[rv.slot]), rv.round & 1, abort_flag, a.status)) return false;
+            const uint32_t vdst = v_base + rv.slot * G::kSlotBytes;
+            constexpr int kPieceShift = G::kHalves == 2 ? 4 : 3;                  // 16-byte pieces per row: 8 per half
+            const int n_pieces = (fix_hi - fix_lo) << kPieceShift;
+            for (int i = row_in_blk; i < n_pieces; i += kBlockRows) {
+                const int r = fix_lo + (i >> kPieceShift), pc = i & ((1 << kPieceShift) - 1);
+                const uint32_t dst = vdst + (pc >> 3) * G::kBoxBytes + r * 128u + ((pc & 7) << 4);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
+            }
+            return true;
+        };
+        if constexpr (kShared) {
+            // ---- shared reference: the warpgroups take alternate tiles (warpgroup w: tiles w, w + 2, ..., all 128
+            // keys, one thread per row) from their own score buffer into their own P buffer; one accumulator.
+            // A score buffer goes back to the S issuer as soon as its scores are in registers, so the only
+            // thing a warpgroup ever waits for is its next scores.
+            const uint32_t s_addr = tmem_s1 + lane_base + wg * TK, p_addr = tmem_p1 + lane_base + wg * (TK / 2);
+            const int quad = warp & 3;
+            bool ok = true;
+            if (wg == 1 && sp.n_tiles > 0) {
+                // the reference comes from warpgroup 0's first tile
+                ok = mbar_wait_warp(smem_u32(&c.mref_full[quad]), 0, abort_flag, a.status);
+                if (ok) m_run = c.m_ref[row_in_blk];
+            }
+            for (int j = wg; ok && j < sp.n_tiles; j += 2) {
+                while (v_tile < j) { rv.advance(nv_slots); ++v_tile; }
+                if (!mbar_wait_warp(smem_u32(&c.s_full[0][wg]), n_own & 1, abort_flag, a.status)) break;
+                [[maybe_unused]] const int trole = 3 + wg;
+                [[maybe_unused]] const bool tr_on = row_in_blk == 0;
+                if (tr_on) SS_TR(trole, 8 + 6 * n_own);
+                tc_fence_after();
+                const int x = sp.first_key(j), nvk = sp.valid_keys(j);
+                const bool cache = sp.is_cache(j);
+                const bool masked = !cache || x + TK > sp.L || nvk < TK;
+                const unsigned long long vis0 = masked ? visible_mask(cache, x, nvk, sp.L, sp.gamma, ri, anc) : ~0ull;
+                const unsigned long long vis1 = masked ? visible_mask(cache, x + 64, nvk - 64, sp.L, sp.gamma, ri, anc) : ~0ull;
+                // the P buffer is free once the P V of the warpgroup's previous tile has completed
+                if (n_own > 0 && !mbar_wait_warp(smem_u32(&c.o_done[wg][(n_own - 1) & 1]), ((n_own - 1) >> 1) & 1, abort_flag, a.status)) break;
+                bool bad = false;
+                if (warp_active) {
+                    uint32_t sr[64], pk[32];
+                    if (j == 0) {
+                        // the row maximum of the first tile is the reference of the row for the whole CTA
+                        tmem_ld64(s_addr + 64, sr);
+                        tmem_wait_ld();
+                        float mx = masked ? chunk_max<true>(sr, a.scale_log2, vis1) : chunk_max<false>(sr, a.scale_log2, 0ull);
+                        tmem_ld64(s_addr, sr);
+                        tmem_wait_ld();
+                        mx = fmaxf(mx, masked ? chunk_max<true>(sr, a.scale_log2, vis0) : chunk_max<false>(sr, a.scale_log2, 0ull));
+                        m_run = mx;
+                        c.m_ref[row_in_blk] = mx;
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&c.mref_full[quad]));   // (release: the lanes' references are written)
+                        bad = ri.valid && !(mx > -INFINITY && mx < INFINITY);     // a row that sees no key here, or a NaN
+                    } else {
+                        tmem_ld64(s_addr, sr);
+                        tmem_wait_ld();
+                    }
+                    if (tr_on) SS_TR(trole, 9 + 6 * n_own);
+                    const float m_use = (m_run > -INFINITY && m_run < INFINITY) ? m_run : 0.f;
+                    float sum = masked ? chunk_exp_pack<true>(sr, a.scale_log2, m_use, vis0, pk) : chunk_exp_pack<false>(sr, a.scale_log2, m_use, 0ull, pk);
+                    tmem_st32(p_addr, pk);
+                    tmem_ld64(s_addr + 64, sr);
+                    tmem_wait_ld();
+                    // the scores are in registers: the S issuer may overwrite the buffer
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&c.s_free[wg]));
+                    if (tr_on) SS_TR(trole, 10 + 6 * n_own);
+                    sum += masked ? chunk_exp_pack<true>(sr, a.scale_log2, m_use, vis1, pk) : chunk_exp_pack<false>(sr, a.scale_log2, m_use, 0ull, pk);
+                    tmem_st32(p_addr + 32, pk);
+                    tmem_wait_st();
+                    l_run += sum;
+                    bad = bad || (ri.valid && !(sum <= kSharedRefLimit));
+                } else {
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive(smem_u32(&c.s_free[wg]));
+                        if (j == 0) mbar_arrive(smem_u32(&c.mref_full[quad]));
+                    }
+                }
+                if (__any_sync(0xffffffffu, bad)) {
+                    // the reference does not hold for some row: every role leaves its loop and the CTA starts over
+                    if (lane == 0) atomicCAS(&c.abort, 0, 2);
+                    break;
+                }
+                if (tr_on) SS_TR(trole, 11 + 6 * n_own);
+                if (!clear_v_tail(j, 0, TK)) break;
+                fence_async_smem();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&c.p_full[0][wg]));
+                if (tr_on) SS_TR(trole, 13 + 6 * n_own);
+                ++n_own;
+            }
+            // The CTA's last P V must have landed before the accumulator is read and before shared memory is reused
+            // (commits complete in order, so the last stands for all).  Its barrier has completed every earlier
+            // phase by now: this warpgroup's last P store came after the P V four tiles before the CTA's last.
+            if (sp.n_tiles > 0) {
+                const int jl = sp.n_tiles - 1;
+                mbar_wait_warp(smem_u32(&c.o_done[jl & 1][(jl >> 1) & 1]), (jl >> 2) & 1, abort_flag, a.status);
+                tc_fence_after();
+            }
+        } else {
+        const uint32_t o_addr = tmem + lane_base + wg * G::kOCols;
         for (int j = 0; j < sp.n_tiles; ++j) {
             while (v_tile < j) { rv.advance(nv_slots); ++v_tile; }
             const int buf = j & 1;
@@ -1062,22 +1223,8 @@ __global__ void __launch_bounds__(Geo<HD>::kThreads, 1) msa_attention_kernel(con
                 tmem_wait_st();
             }
             if (tr_on) SS_TR(trole, 11 + 6 * n_own);
-            // V rows past the end of the sequence's keys may hold anything (even NaN patterns): P is 0
-            // there, but 0 * NaN is NaN, so the warpgroup clears the ones its P V reads (its half of the tile).
-            // Rows that only lie past this CTA's share of the keys are real data.
-            const int region_left = (cache ? sp.L + sp.T : sp.n_stream) - x;      // real rows in the tile
-            const int fix_lo = max(region_left, wg * 64), fix_hi = wg * 64 + 64;
-            if (fix_lo < fix_hi) {
-                if (!mbar_wait_warp(smem_u32(&c.v_full[rv.slot]), rv.round & 1, abort_flag, a.status)) break;
-                const uint32_t vdst = v_base + rv.slot * G::kSlotBytes;
-                constexpr int kPieceShift = G::kHalves == 2 ? 4 : 3;              // 16-byte pieces per row: 8 per half
-                const int n_pieces = (fix_hi - fix_lo) << kPieceShift;
-                for (int i = row_in_blk; i < n_pieces; i += kBlockRows) {
-                    const int r = fix_lo + (i >> kPieceShift), pc = i & ((1 << kPieceShift) - 1);
-                    const uint32_t dst = vdst + (pc >> 3) * G::kBoxBytes + r * 128u + ((pc & 7) << 4);
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
-                }
-            }
+            // the warpgroup clears the V rows past the end that its P V reads (its half of the tile)
+            if (!clear_v_tail(j, wg * 64, wg * 64 + 64)) break;
             if (tr_on) SS_TR(trole, 12 + 6 * n_own);
             fence_async_smem();
             tc_fence_before();
@@ -1093,6 +1240,59 @@ __global__ void __launch_bounds__(Geo<HD>::kThreads, 1) msa_attention_kernel(con
             mbar_wait_warp(smem_u32(&c.o_done[wg][(n_own - 1) & 1]), ((n_own - 1) >> 1) & 1, abort_flag, a.status);
             tc_fence_after();
         }
+        }   // running maximum per warpgroup
+    }
+    };  // run_tiles
+    if (tid == 0) n_requested = n_early_k; else if (tid == 96) n_requested = n_early_v;
+    if (shared_ref) {
+        run_tiles(std::true_type{}, n_early_k, n_early_v);
+        __syncwarp();
+        tc_fence_before();
+        __syncthreads();                                  // every role has left its loop
+        tc_fence_after();
+        if (c.abort == 2) {
+            // The shared reference did not hold for some row.  What is in flight lands first: the producers wait
+            // for the last copy they requested into every slot, the MMA issuers for their last MMA; then the
+            // barriers are set up anew (all but the query tile's) and the tiles run again from the first.
+            if (tid == 0 || tid == 96) {
+                const int slots = tid == 0 ? nk : nv_slots;
+                unsigned long long* const full = tid == 0 ? c.k_full : c.v_full;
+                for (int sl = 0; sl < slots; ++sl)
+                    if (n_requested > sl) mbar_drain(smem_u32(&full[sl]), ((n_requested - 1 - sl) / slots) & 1);
+                if (tid == 0) mbar_drain(smem_u32(&c.q_full), 0);
+            } else if (tid == 32 || tid == 64) {
+                const uint32_t bar = smem_u32(&c.drain[tid == 64 ? 1 : 0]);
+                tc_commit(bar);
+                mbar_drain(bar, 0);
+            }
+            __syncwarp();
+            if (warp >= 4) { tmem_wait_ld(); tmem_wait_st(); }
+            tc_fence_before();
+            __syncthreads();
+            tc_fence_after();
+            if (tid == 0) {
+                for (int sl = 0; sl < kMaxSlots; ++sl) {
+                    unsigned long long* const ring[4] = {&c.k_full[sl], &c.k_empty[sl], &c.v_full[sl], &c.v_empty[sl]};
+                    for (int i = 0; i < 4; ++i) { mbar_inval(smem_u32(ring[i])); mbar_init(smem_u32(ring[i]), 1); }
+                }
+                for (int i = 0; i < 2; ++i) {
+                    mbar_inval(smem_u32(&c.s_free[i]));
+                    for (int k = 0; k < 2; ++k) {
+                        mbar_inval(smem_u32(&c.s_full[i][k])); mbar_inval(smem_u32(&c.p_full[i][k])); mbar_inval(smem_u32(&c.o_done[i][k]));
+                    }
+                }
+                init_tile_barriers(c, false);
+                c.abort = 0;
+                atomicAdd(a.status + 2, 1);               // diagnostics: blocks that started over
+                asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            }
+            shared_ref = false;
+            m_run = -INFINITY; l_run = 0.f; n_own = 0; n_requested = 0;
+            __syncthreads();
+            run_tiles(std::false_type{}, 0, 0);
+        }
+    } else {
+        run_tiles(std::false_type{}, n_early_k, n_early_v);
     }
     if (tid == kAuxThreads) SS_TR(5, 0);
     __syncwarp();     // the single-lane roles of warps 0..3 rejoin their warps
@@ -1101,8 +1301,9 @@ __global__ void __launch_bounds__(Geo<HD>::kThreads, 1) msa_attention_kernel(con
     // The softmax warpgroups combine the partials a row has inside the CTA.  Not split (C == 1): that
     // is the result.  Split: every CTA leaves one un-normalised partial row (O, m, l) per query row in
     // the workspace (it stays in L2) and combines its own share of the rows as they arrive from all CTAs.
-    const bool has_acc = (warp >= 4) && n_own > 0;     // otherwise the partial is (m = -inf, l = 0, O = 0)
-    const uint32_t o_addr = tmem + lane_base + (warp >= 4 ? wg : 0) * G::kOCols;
+    // (shared reference: one accumulator, which both threads of a lane read; the reference is the row's m for both)
+    const bool has_acc = (warp >= 4) && (shared_ref ? sp.n_tiles > 0 : n_own > 0);     // otherwise the partial is (m = -inf, l = 0, O = 0)
+    const uint32_t o_addr = tmem + lane_base + ((warp >= 4 && !shared_ref) ? wg : 0) * G::kOCols;
     constexpr int RP = G::kMergePitch;                                         // floats per partial row: O, m, l, pad
     constexpr uint32_t RB = RP * 4;                                            // bytes of a partial row
     constexpr int rows_cap = G::kRowsCap;                                      // partial rows per CTA
@@ -1135,7 +1336,7 @@ __global__ void __launch_bounds__(Geo<HD>::kThreads, 1) msa_attention_kernel(con
         const float w_ot = other.x != -INFINITY ? exp2f(other.x - m_out) : 0.f;
         float l_out = w_me * l_run + w_ot * other.y;
         // an accumulator that no MMA has written holds anything: it is not read
-        const bool has_ot = has_acc;
+        const bool has_ot = has_acc && !shared_ref;
         const uint32_t o_other = tmem + lane_base + (wg ^ 1) * G::kOCols;
         const int c_lo = wg == 0 ? 0 : G::kSplitCol, c_hi = wg == 0 ? G::kSplitCol : HD;
         float v[G::kSplitCol];                                                   // this thread's columns of the lane's combined partial
@@ -1299,7 +1500,7 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     // row blocks: the query tile, then the K ring and the V ring (P lives in TMEM)
     const size_t qp = static_cast<size_t>(halves) * kBlockRows * 128;
     const size_t slot = static_cast<size_t>(halves) * kTileKeys * 128;
-    int slots = static_cast<int>((kMaxDynSmem - 1024 - qp) / slot);
+    int slots = static_cast<int>((kPairMaxDynSmem - 1024 - qp) / slot);
     if (slots > 2 * kMaxSlots) slots = 2 * kMaxSlots;
     if (slots < 4) return false;
     // a K slot is held until S is queued, a V slot until P V has completed: the odd slot goes to V
@@ -1314,7 +1515,7 @@ static bool make_plan(const ss_attn_params& p, AttnPlan* plan) {
     plan->smem = bytes + 1024;
     // workspace: one partial row per (group, CTA of the group, row)
     plan->partial_bytes = c > 1 ? static_cast<size_t>(plan->groups) * c * kBlockRows * row_bytes : 0;
-    return plan->smem <= static_cast<size_t>(kMaxDynSmem);
+    return plan->smem <= static_cast<size_t>(kPairMaxDynSmem);
 }
 
 template <int HD>
@@ -1323,7 +1524,7 @@ static int32_t launch(const AttnArgs& args, const AttnPlan& plan, cudaStream_t s
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return SS_ERR_CUDA;
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        if (cudaFuncSetAttribute(msa_attention_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem) !=
+        if (cudaFuncSetAttribute(msa_attention_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairMaxDynSmem) !=
             cudaSuccess)
             return SS_ERR_CUDA;
         configured[dev] = true;

@@ -100,6 +100,10 @@ EDGE_CASES = {
                                       k_ramp=0.05),
     "growing_scores_row_blocks": dict(prefix_len=1500, n_nodes=64, gamma=4, max_depth=5, n_heads=40, head_dim=128,
                                       tree_kind="topk_growth", k_ramp=0.05),
+    # later keys exceed the first tile's scores by hundreds of nats: unsplit 128-row blocks give up the reference they
+    # share (the row maximum of the first tile) and run their tiles again with a running maximum
+    "steep_scores_row_blocks": dict(prefix_len=700, n_nodes=64, gamma=4, max_depth=5, n_heads=40, head_dim=128,
+                                    tree_kind="topk_growth", k_ramp=0.5),
     "growing_scores_split_keys": dict(prefix_len=3000, n_nodes=40, gamma=2, max_depth=4, n_heads=3, head_dim=64,
                                       k_ramp=0.03),
 }
@@ -114,6 +118,9 @@ def test_attention_edge_cases(cuda, oracle, case):
     dev = DeviceStep(st, with_lse=True)
     dev.run_attention()
     assert api.ss_status(dev.attn_ws) == 0
+    started_over = int(dev.attn_ws.view(torch.int32)[2])
+    if case == "steep_scores_row_blocks":
+        assert started_over > 0                              # the multi-stream layer's blocks did start over
     for i in range(2):
         assert_attention_close(oracle, st, st.layer(i), dev, i, check_lse=True)
 
