@@ -1092,8 +1092,6 @@ __global__ void __launch_bounds__(Geo<HD>::kThreads, 1) msa_attention_kernel(con
                 const bool masked = !cache || x + TK > sp.L || nvk < TK;
                 const unsigned long long vis0 = masked ? visible_mask(cache, x, nvk, sp.L, sp.gamma, ri, anc) : ~0ull;
                 const unsigned long long vis1 = masked ? visible_mask(cache, x + 64, nvk - 64, sp.L, sp.gamma, ri, anc) : ~0ull;
-                // the P buffer is free once the P V of the warpgroup's previous tile has completed
-                if (n_own > 0 && !mbar_wait_warp(smem_u32(&c.o_done[wg][(n_own - 1) & 1]), ((n_own - 1) >> 1) & 1, abort_flag, a.status)) break;
                 bool bad = false;
                 if (warp_active) {
                     uint32_t sr[64], pk[32];
@@ -1117,6 +1115,9 @@ __global__ void __launch_bounds__(Geo<HD>::kThreads, 1) msa_attention_kernel(con
                     if (tr_on) SS_TR(trole, 9 + 6 * n_own);
                     const float m_use = (m_run > -INFINITY && m_run < INFINITY) ? m_run : 0.f;
                     float sum = masked ? chunk_exp_pack<true>(sr, a.scale_log2, m_use, vis0, pk) : chunk_exp_pack<false>(sr, a.scale_log2, m_use, 0ull, pk);
+                    // the P buffer is free once the P V of the warpgroup's previous tile has completed
+                    if (n_own > 0 && !mbar_wait_warp(smem_u32(&c.o_done[wg][(n_own - 1) & 1]), ((n_own - 1) >> 1) & 1, abort_flag, a.status)) break;
+                    tc_fence_after();
                     tmem_st32(p_addr, pk);
                     tmem_ld64(s_addr + 64, sr);
                     tmem_wait_ld();
@@ -1131,7 +1132,9 @@ __global__ void __launch_bounds__(Geo<HD>::kThreads, 1) msa_attention_kernel(con
                     l_run += sum;
                     bad = bad || (ri.valid && !(sum <= kSharedRefLimit));
                 } else {
-                    __syncwarp();
+                    // (a warp without rows keeps the protocol, this wait included: it must see every phase of
+                    // the barrier, or the wait after the loop could take an earlier phase for the last)
+                    if (n_own > 0 && !mbar_wait_warp(smem_u32(&c.o_done[wg][(n_own - 1) & 1]), ((n_own - 1) >> 1) & 1, abort_flag, a.status)) break;
                     if (lane == 0) {
                         mbar_arrive(smem_u32(&c.s_free[wg]));
                         if (j == 0) mbar_arrive(smem_u32(&c.mref_full[quad]));
