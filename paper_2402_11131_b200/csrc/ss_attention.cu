@@ -18,13 +18,21 @@
 //   warp 1      tcgen05 issuer of S = Q K^T (128 x 128 keys x d) into one of two TMEM buffers;
 //   warp 2      tcgen05 issuer of O += P V (A = P in TMEM) into the TMEM accumulator of a warpgroup;
 //               tcgen05.commit arrives on the mbarriers that hand buffers back.
-//   warps 4..11 two softmax warpgroups, one thread per TMEM lane: of every 128-key tile warpgroup 0 takes
-//               keys 0..63 and warpgroup 1 keys 64..127, each with its own running maximum and
-//               accumulator: tcgen05.ld of 64 scores of the row, tree / stream mask from the node's
-//               64-bit ancestor word, online softmax in fp32 registers (the running maximum is only
-//               raised when it would grow by more than 2^8, which keeps the TMEM accumulator untouched
-//               on almost every tile), P as bf16 written over the first 32 of the score columns just
-//               read, from where the second MMA takes it.
+//   warps 4..11 two softmax warpgroups, one thread per TMEM lane: tcgen05.ld of the row's scores, tree /
+//               stream mask from the node's 64-bit ancestor word, exponentials and row sums in fp32
+//               registers, P as bf16 back to TMEM, from where the second MMA takes it.  Two pipelines:
+//               - a block whose keys are not split (C == 1, the long key sequences): the warpgroups take
+//                 alternate tiles against one reference per row, the maximum of the row's first tile
+//                 (any reference not absurdly far from the row's maximum gives the same result after
+//                 normalisation); one accumulator; P in TMEM buffers of its own, so a score buffer goes
+//                 back to the S issuer as soon as its scores are in registers and one tile's exponentials
+//                 run beside the other tile's MMAs.  If a later tile's exponentials would leave the range
+//                 of fp32 (a tile's row sum above 2^64), the CTA lets everything in flight land, sets its
+//                 barriers up anew and runs its tiles again on the other pipeline;
+//               - a split block (short key spans), or a block that started over: of every tile warpgroup 0
+//                 takes keys 0..63 and warpgroup 1 keys 64..127, each with its own running maximum (raised
+//                 only when it would grow by more than 2^8) and accumulator; P is written over the first
+//                 32 of the score columns just read.
 //
 // Split-KV merge.  Each CTA ends with un-normalised (m, l, O) per row, combines what it holds for a
 // row locally, and -- when the keys were split -- leaves one partial row in the workspace (it stays in
@@ -452,8 +460,9 @@ __device__ __forceinline__ float chunk_exp_pack(const uint32_t (&v)[64], float s
     unsigned long long sum2[2] = {pack_f32x2(0.f, 0.f), pack_f32x2(0.f, 0.f)};
     #pragma unroll
     for (int k = 0; k < 64; k += 2) {
+        const unsigned long long t2 = fma_f32x2(pack_f32x2(__uint_as_float(v[k]), __uint_as_float(v[k + 1])), scale2, shift2);
         float t0, t1;
-        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[k]), __uint_as_float(v[k + 1])), scale2, shift2), t0, t1);
+        unpack_f32x2(t2, t0, t1);
         float e0 = exp2f(t0), e1 = exp2f(t1);
         if (MASKED) {
             e0 = (((k < 32 ? vlo : vhi) >> (k & 31)) & 1u) ? e0 : 0.f;
