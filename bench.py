@@ -340,6 +340,8 @@ def measure(args, workload, world, rank, local_rank):
     status = api.ss_status(dev.attn_ws, stream) or api.ss_status(dev.verify_ws, stream)
     if status != 0:
         raise RuntimeError("device status %d after the timed region" % status)
+    # workspace word 2: CTAs of unsplit row blocks that gave up their shared reference and ran their tiles twice
+    started_over = int(dev.attn_ws.view(torch.int32)[2])
 
     # ---- the draft-management calls around the step (not part of it), each timed alone --------------
     draft_us = None
@@ -381,6 +383,7 @@ def measure(args, workload, world, rank, local_rank):
         "us_verify": verify_ms * 1e3, "us_compact": compact_ms * 1e3,
         "draft_management_us": draft_us,
         "mean_accept_len": float(acc.mean()),
+        "row_blocks_started_over": started_over,
         "attention_tflops": attn_flops / (attn_ms * 1e-3) / 1e12,
         "gpu_launches": launches_per_step * K,
         "clocks": clocks,
