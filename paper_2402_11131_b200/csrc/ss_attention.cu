@@ -723,7 +723,9 @@ __device__ __forceinline__ void mbar_inval(uint32_t bar) {
     asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-template <int HD>
+// SHARED: the instantiation for blocks whose keys are not split (it starts on the shared-reference pipeline and holds
+// the other one for a block that has to start over); the instantiation for split blocks holds only the other one.
+template <int HD, bool SHARED>
 __global__ void __launch_bounds__(Geo<HD>::kThreads, 1) msa_attention_kernel(const __grid_constant__ AttnArgs a) {
     using G = Geo<HD>;
     constexpr int TK = kTileKeys;
@@ -741,7 +743,7 @@ __global__ void __launch_bounds__(Geo<HD>::kThreads, 1) msa_attention_kernel(con
     const int nk = a.n_kslots, nv_slots = a.n_vslots;
     volatile int* abort_flag = &c.abort;
     // Row blocks that are not split start on the shared-reference pipeline (see kSharedRefLimit)
-    bool shared_ref = C == 1;
+    bool shared_ref = SHARED;
 
     if (tid == 0) SS_TR(0, 0);
 #ifdef SS_TRACE
@@ -1256,7 +1258,7 @@ __global__ void __launch_bounds__(Geo<HD>::kThreads, 1) msa_attention_kernel(con
     }
     };  // run_tiles
     if (tid == 0) n_requested = n_early_k; else if (tid == 96) n_requested = n_early_v;
-    if (shared_ref) {
+    if constexpr (SHARED) {
         run_tiles(std::true_type{}, n_early_k, n_early_v);
         __syncwarp();
         tc_fence_before();
@@ -1536,8 +1538,10 @@ static int32_t launch(const AttnArgs& args, const AttnPlan& plan, cudaStream_t s
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return SS_ERR_CUDA;
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        if (cudaFuncSetAttribute(msa_attention_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairMaxDynSmem) !=
-            cudaSuccess)
+        if (cudaFuncSetAttribute(msa_attention_kernel<HD, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairMaxDynSmem) !=
+                cudaSuccess ||
+            cudaFuncSetAttribute(msa_attention_kernel<HD, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairMaxDynSmem) !=
+                cudaSuccess)
             return SS_ERR_CUDA;
         configured[dev] = true;
     }
@@ -1554,7 +1558,9 @@ static int32_t launch(const AttnArgs& args, const AttnPlan& plan, cudaStream_t s
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, msa_attention_kernel<HD>, args) == cudaSuccess ? SS_OK : SS_ERR_CUDA;
+    const cudaError_t err = plan.cluster == 1 ? cudaLaunchKernelEx(&cfg, msa_attention_kernel<HD, true>, args)
+                                              : cudaLaunchKernelEx(&cfg, msa_attention_kernel<HD, false>, args);
+    return err == cudaSuccess ? SS_OK : SS_ERR_CUDA;
 }
 
 template <int HD>
