@@ -104,6 +104,11 @@ EDGE_CASES = {
     # share (the row maximum of the first tile) and run their tiles again with a running maximum
     "steep_scores_row_blocks": dict(prefix_len=700, n_nodes=64, gamma=4, max_depth=5, n_heads=40, head_dim=128,
                                     tree_kind="topk_growth", k_ramp=0.5),
+    # the same in a ragged batch (sequences dispatched longest first) and at head_dim 64 with two row blocks
+    "steep_scores_ragged_batch": dict(batch=3, prefix_len_range=(300, 1500), n_nodes=40, gamma=3, max_depth=4, n_heads=16,
+                                      head_dim=128, tree_kind="topk_growth", k_ramp=0.3),
+    "steep_scores_d64": dict(prefix_len=2000, n_nodes=64, gamma=2, max_depth=5, n_heads=48, head_dim=64,
+                             tree_kind="topk_growth", k_ramp=0.4),
     "growing_scores_split_keys": dict(prefix_len=3000, n_nodes=40, gamma=2, max_depth=4, n_heads=3, head_dim=64,
                                       k_ramp=0.03),
 }
@@ -119,7 +124,7 @@ def test_attention_edge_cases(cuda, oracle, case):
     dev.run_attention()
     assert api.ss_status(dev.attn_ws) == 0
     started_over = int(dev.attn_ws.view(torch.int32)[2])
-    if case == "steep_scores_row_blocks":
+    if case.startswith("steep_scores"):
         assert started_over > 0                              # the multi-stream layer's blocks did start over
     for i in range(2):
         assert_attention_close(oracle, st, st.layer(i), dev, i, check_lse=True)
